@@ -1,0 +1,203 @@
+/*
+ * mosaic.h - C ABI of the B200 (sm_100a) library for the data-parallel hot
+ * path of Mosaic's composite projection pruning.
+ *
+ * The path (paper Section 3.1-3.3, Algorithm 1, Section 4.1.3):
+ *   activation l2 norms per input channel  ->  weight metric w = norm*|W| (Eq. 5)
+ *   ->  projection outlier count (Eq. 6)   ->  non-uniform sparsity targets
+ *   (normalize(R_LLM) + Projection Planner, Eq. 1-2)  ->  per-row unstructured
+ *   selection + zeroing  ->  structured ranking + dense compaction.
+ *
+ * Conventions that hold for every call
+ *   - Matrices are row-major.  W is [rows = out_features, cols = in_features]
+ *     with leading dimension ldw (elements); X is [tokens, cols] with ldx.
+ *   - dtype is MOSAIC_F32 or MOSAIC_BF16 (raw IEEE bfloat16 bit patterns).
+ *   - "device" pointers are CUDA global memory of the current device; "host"
+ *     pointers are ordinary memory.  Matrix base pointers must be 16-byte
+ *     aligned and leading dimensions a multiple of 16 bytes (8 bf16 / 4 fp32
+ *     elements), otherwise MOSAIC_ERR_MISALIGNED.
+ *   - The library allocates no memory and owns none: outputs and workspaces
+ *     are the caller's.  A workspace must be 256-byte aligned and at least
+ *     the matching *_workspace_bytes() query; its contents are scratch.
+ *   - Device calls only enqueue work on `stream` (a cudaStream_t passed as
+ *     void*, NULL = default stream) and never synchronise.  Results are
+ *     deterministic: the same inputs give the same bytes, run to run.
+ *   - Every call returns MOSAIC_OK (0) or a negative mosaic_status; argument
+ *     errors are detected before anything is enqueued.  No C++ exception
+ *     crosses the boundary.
+ *   - norms[] must be >= +0 (they are l2 norms); scores are then >= +0 and
+ *     ordered by their fp32 bit patterns.  A NaN score orders above +inf.
+ */
+#ifndef MOSAIC_H_
+#define MOSAIC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MOSAIC_VERSION 100
+
+typedef enum mosaic_status {
+    MOSAIC_OK = 0,
+    MOSAIC_ERR_INVALID_ARG = -1,
+    MOSAIC_ERR_NULL_PTR = -2,
+    MOSAIC_ERR_BAD_DTYPE = -3,
+    MOSAIC_ERR_MISALIGNED = -4,
+    MOSAIC_ERR_WORKSPACE_TOO_SMALL = -5,
+    MOSAIC_ERR_ALIASING = -6,
+    MOSAIC_ERR_CUDA = -7,
+    MOSAIC_ERR_NONFINITE = -8,   /* reserved */
+    MOSAIC_ERR_INFEASIBLE = -9,  /* allocation had to clamp a target; outputs are still written */
+    MOSAIC_ERR_TIMEOUT = -10     /* reserved */
+} mosaic_status;
+
+typedef enum mosaic_dtype { MOSAIC_F32 = 0, MOSAIC_BF16 = 1 } mosaic_dtype;
+
+/* flags of mosaic_act_norms */
+#define MOSAIC_RESET_ACCUM 1 /* treat sumsq_accum as zero on entry */
+
+/* mode of mosaic_allocate_sparsity */
+#define MOSAIC_GLOBAL_NORM 0       /* normalise ranks over all N*M projections            */
+#define MOSAIC_PER_CATEGORY_NORM 1 /* normalise separately over the N entries of each m   */
+
+/* flags of mosaic_prune_structured_compact */
+#define MOSAIC_ROWS_GIVEN 1    /* row_keep_units is an input (ascending unit indices)      */
+#define MOSAIC_COLS_GIVEN 2    /* col_keep_units is an input                               */
+#define MOSAIC_RANK_ONLY 4     /* compute scores / keep lists, do not write W_out          */
+#define MOSAIC_SCORES_ONLY 8   /* compute unit_scores_out only: no ranking, no compaction  */
+#define MOSAIC_SCORES_ACCUM 16 /* add the unit scores to unit_scores_out (fp32) instead of
+                                  overwriting it: lets a caller sum the scores of coupled
+                                  projections before ranking them once                     */
+
+int mosaic_version(void);
+const char *mosaic_status_string(int status);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_act_norms - the ||A||_2 term of Eq. 5 (Section 3.3, Activation
+ * Processor / Rank Pre-Processor): per input channel j,
+ *     sumsq_accum[j] += sum_t X[t,j]^2        (fp64, exact squares)
+ * and, if norms_out != NULL,  norms_out[j] = (float) sqrt(sumsq_accum[j]).
+ * Accumulating: call once per chunk of calibration tokens; tokens == 0 is
+ * legal (only the reset / finalise parts run).
+ *   X            device, [tokens, cols], ld ldx, dtype; read only
+ *   sumsq_accum  device, [cols] fp64, in-out, caller-owned accumulator
+ *   norms_out    device, [cols] fp32, or NULL
+ *   flags        0 or MOSAIC_RESET_ACCUM
+ *   ws           device scratch, >= mosaic_act_norms_workspace_bytes(tokens, cols)
+ * ------------------------------------------------------------------------- */
+size_t mosaic_act_norms_workspace_bytes(int64_t tokens, int64_t cols);
+int mosaic_act_norms(const void *X, int64_t tokens, int64_t cols, int64_t ldx, int dtype,
+                     double *sumsq_accum, float *norms_out, int flags, void *ws, size_t ws_bytes,
+                     void *stream);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_score - Eq. 5 / Algorithm 1 line 11, materialised:
+ *     score_out[i, j] = fl32( norms[j] * |W[i, j]| )      (one fp32 multiply)
+ * For tests and small use; the pruning calls recompute scores on the fly.
+ *   W          device, [rows, cols], ld ldw, dtype; read only
+ *   norms      device, [cols] fp32
+ *   score_out  device, [rows, cols] fp32, ld = cols, 16-byte aligned
+ * ------------------------------------------------------------------------- */
+int mosaic_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                 const float *norms, float *score_out, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_outlier_ratio - Eq. 6 / Algorithm 1 lines 13-14 for one projection:
+ *     S = sum_ij (double) w_ij,  tau = (double)alpha * S / (rows*cols),
+ *     O = #{ (i,j) : (double) w_ij > tau }                  (strict)
+ *   outlier_count_out  device, 1 x int64
+ *   score_sum_out      device, 1 x fp64, or NULL
+ *   ws                 device scratch, >= mosaic_outlier_ratio_workspace_bytes()
+ * The rank R = 100*O/C (Algorithm 1 line 15) is formed on the host:
+ * mosaic_ratio_from_count.
+ * ------------------------------------------------------------------------- */
+size_t mosaic_outlier_ratio_workspace_bytes(int64_t rows, int64_t cols);
+int mosaic_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                         const float *norms, float alpha, int64_t *outlier_count_out,
+                         double *score_sum_out, void *ws, size_t ws_bytes, void *stream);
+double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_allocate_sparsity - normalize(R_LLM) (Algorithm 1 line 19) and the
+ * Projection Planner (Section 3.3 component 8; Eq. 1-2).  HOST function, all
+ * pointers are host memory, q = n*n_proj + m.
+ * The paper states only the properties (targets average to p; more outliers
+ * => pruned less).  Definition used, fp64, loops in q order:
+ *     R_q = 100*O_q/C_q;  lo = min R, hi = max R;  hi == lo -> s_q = p
+ *     r_q = (R_q-lo)/(hi-lo);  d_q = 2*lambda*r_q;  dbar = (sum_q d_q)/count
+ *     s_q = (p + dbar) - d_q, clamped to [0, 1 - 1/cols_q]
+ *     k_q = floor(s_q * cols_q)       (weights removed from every row)
+ * MOSAIC_PER_CATEGORY_NORM applies the same over the n_layers entries of each
+ * projection index m separately.  Returns MOSAIC_ERR_INFEASIBLE if a clamp
+ * fired (outputs are still complete).
+ * ------------------------------------------------------------------------- */
+int mosaic_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numels,
+                             const int64_t *cols, int n_layers, int n_proj, double p,
+                             double lambda, int mode, double *sparsity_out, int64_t *k_out);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_prune_unstructured - unstructured projection pruning (Section 4.1.3:
+ * pruned parameters are set to zero; Section 2.3: the lowest-ranking
+ * parameters are removed), selection per output row.  In every row the k
+ * entries that come first under (w_ij ascending, j ascending) become +0; all
+ * other entries keep their bits.
+ *   W_in      device, [rows, cols]; W_out device, same shape/ld; W_out may be
+ *             W_in exactly (in place); any other overlap -> MOSAIC_ERR_ALIASING
+ *   k         0 <= k <= cols
+ *   mask_out  device, [rows, ceil(cols/32)] uint32 or NULL; bit j%32 of word
+ *             j/32 is 1 for a kept entry; padding bits are 0
+ *   cols      at most 65536
+ * ------------------------------------------------------------------------- */
+size_t mosaic_prune_unstructured_workspace_bytes(int64_t rows, int64_t cols);
+int mosaic_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64_t cols,
+                              int64_t ldw, int dtype, const float *norms, int64_t k,
+                              uint32_t *mask_out, void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_prune_structured_compact - structured projection pruning (Section
+ * 4.1.3: remove the lowest-magnitude heads and channels; Section 2.3:
+ * structured pruning removes whole data structures and leaves smaller dense
+ * matrices).  A row unit is row_group consecutive rows, a column unit
+ * col_group consecutive columns (rows % row_group == 0, cols % col_group == 0).
+ *   1. unit scores: fp64 sum of w_ij over the unit, rounded once to fp32
+ *      (norms == NULL means norm = 1, i.e. sum of |W|);
+ *   2. per dimension, the (n_units - keep) units first under (score asc,
+ *      index asc) are removed; the keep list is the surviving unit indices
+ *      in ascending order;
+ *   3. W_out[a, b] = W_in[row(a), col(b)] bit for bit, dense,
+ *      [row_units_keep*row_group, col_units_keep*col_group], ld = its cols.
+ *   row_keep_units / col_keep_units  device int32 [row_units_keep] / [col_units_keep];
+ *        outputs, or inputs when the matching *_GIVEN flag is set (ascending
+ *        unit indices chosen elsewhere, e.g. shared by coupled projections;
+ *        an out-of-range given index is clamped into range)
+ *   unit_scores_out  device fp32 [rows/row_group + cols/col_group] (row units
+ *        first) or NULL
+ *   W_out   device; must not overlap W_in; ignored for RANK_ONLY / SCORES_ONLY
+ *   ws      device scratch, >= mosaic_prune_structured_compact_workspace_bytes()
+ * ------------------------------------------------------------------------- */
+size_t mosaic_prune_structured_compact_workspace_bytes(int64_t rows, int64_t cols);
+int mosaic_prune_structured_compact(const void *W_in, int64_t rows, int64_t cols, int64_t ldw,
+                                    int dtype, const float *norms, int64_t row_group,
+                                    int64_t col_group, int64_t row_units_keep,
+                                    int64_t col_units_keep, int32_t *row_keep_units,
+                                    int32_t *col_keep_units, int flags, void *W_out,
+                                    float *unit_scores_out, void *ws, size_t ws_bytes,
+                                    void *stream);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_rank_units - step 2 above on its own, for scores a caller combined
+ * itself (coupled projections share one keep list: Fig. "composite", nodes
+ * between projections are pruned as a group).
+ *   scores     device fp32 [n_units], >= +0
+ *   keep_out   device int32 [keep], ascending surviving unit indices
+ * ------------------------------------------------------------------------- */
+int mosaic_rank_units(const float *scores, int64_t n_units, int64_t keep, int32_t *keep_out,
+                      void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOSAIC_H_ */

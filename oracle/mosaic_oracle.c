@@ -1,0 +1,415 @@
+/*
+ * TEST INFRASTRUCTURE - NOT PART OF THE PRODUCT.
+ *
+ * A plain, slow, scalar CPU statement of what the hot path of Mosaic's
+ * composite projection pruning computes.  It exists so that the CUDA library
+ * can be checked element by element against something a reader can verify by
+ * eye against the paper.  It shares no source, header, table or helper with
+ * the CUDA library and must never be called from the product path.
+ *
+ * Every function is the definition written out: loops in index order, fp64
+ * for every accumulation, one fp32 multiply for the score, a full sort for
+ * every selection.  OpenMP is used only across independent outputs (columns,
+ * rows, units), so threading never changes a result.
+ *
+ * Notation follows the paper (Section 3.1-3.3):
+ *   W      one projection's weights, row-major [rows = out, cols = in]
+ *   X      calibration activations feeding that projection, row-major [T, cols]
+ *   norm_j l2 norm of column j of X                         (the ||A||_2 of Eq. 5)
+ *   w_ij   = norm_j * |W_ij|                                (Eq. 5, Alg. 1 line 11)
+ *   C      = rows*cols                                      (Alg. 1 line 13)
+ *   O      = #{ w_ij > alpha * mean(w) }                    (Eq. 6, Alg. 1 line 14)
+ *   R      = 100 * O / C                                    (Alg. 1 line 15)
+ *
+ * Parity with the authors' own program is unpinned: the paper prints no
+ * worked numeric example and leaves normalize(R_LLM) (Alg. 1 line 19)
+ * undefined; oracle_allocate_sparsity states the reading taken.  Everything
+ * else here is pinned by the CPU tests against brute force in exact rational
+ * arithmetic, closed forms and invariants.
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -fopenmp -shared -fPIC
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+enum { ORACLE_F32 = 0, ORACLE_BF16 = 1 };
+
+/* Element idx of a buffer of the given type, widened exactly to fp32. */
+static float load_elem(const void *base, int64_t idx, int dtype)
+{
+    if (dtype == ORACLE_F32)
+        return ((const float *)base)[idx];
+    uint32_t bits = (uint32_t)((const uint16_t *)base)[idx] << 16; /* bf16 = top half of fp32 */
+    float f;
+    memcpy(&f, &bits, sizeof f);
+    return f;
+}
+
+static uint32_t float_bits(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    return u;
+}
+
+/* Eq. 5 for one element: a single round-to-nearest fp32 multiply. */
+static float weight_metric(float norm_j, float w)
+{
+    float a = fabsf(w);
+    float s = norm_j * a; /* built with -ffp-contract=off: never fused or widened */
+    return s;
+}
+
+/*
+ * Ordering key of a score.  Scores are >= +0, so their fp32 bit patterns
+ * order like the values; a NaN score (non-finite input, not covered by the
+ * paper) is given the largest key so it is selected last.
+ */
+static uint32_t score_key(float s)
+{
+    return (s != s) ? 0xFFFFFFFFu : float_bits(s);
+}
+
+/* ------------------------------------------------------------------ */
+/* Activation norms: the ||A||_2 term of Eq. 5 (Section 3.3, RC 3-4).  */
+/* ------------------------------------------------------------------ */
+
+/*
+ * sumsq[j] += sum_t X[t,j]^2: for every column j the squares are added one by
+ * one in t order, in fp64 (each square of a bf16/fp32 value is exact in fp64).
+ * Columns are independent; they are walked a block at a time only so that
+ * memory is read along rows.
+ */
+void oracle_act_sumsq(const void *X, int64_t tokens, int64_t cols, int64_t ldx,
+                      int dtype, double *sumsq)
+{
+    const int64_t block = 64;
+#pragma omp parallel for schedule(static)
+    for (int64_t j0 = 0; j0 < cols; j0 += block) {
+        int64_t j1 = j0 + block < cols ? j0 + block : cols;
+        for (int64_t t = 0; t < tokens; ++t)
+            for (int64_t j = j0; j < j1; ++j) {
+                double x = (double)load_elem(X, t * ldx + j, dtype);
+                sumsq[j] = sumsq[j] + x * x;
+            }
+    }
+}
+
+/* norm[j] = (float) sqrt(sumsq[j]) */
+void oracle_norm_finalize(const double *sumsq, int64_t cols, float *norms)
+{
+    for (int64_t j = 0; j < cols; ++j)
+        norms[j] = (float)sqrt(sumsq[j]);
+}
+
+/*
+ * Certification of the norms of one X against summation order: ok[j] = 1 iff
+ * the fp32 norm of column j is the same for the sequential fp64 sum, for an
+ * extended-precision (long double) sum, and for that sum perturbed by
+ * +-tokens*2^-52 relative - i.e. no admissible fp64 summation order can
+ * change the rounded result.  Returns the number of columns NOT certified.
+ */
+int64_t oracle_norm_certify(const void *X, int64_t tokens, int64_t cols, int64_t ldx,
+                            int dtype, uint8_t *ok)
+{
+    int64_t bad = 0;
+    double eps = (double)tokens * ldexp(1.0, -52);
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+    for (int64_t j = 0; j < cols; ++j) {
+        double s = 0.0;
+        long double e = 0.0L;
+        for (int64_t t = 0; t < tokens; ++t) {
+            double x = (double)load_elem(X, t * ldx + j, dtype);
+            s = s + x * x;
+            e = e + (long double)x * (long double)x;
+        }
+        float n0 = (float)sqrt(s);
+        float n1 = (float)sqrt((double)e);
+        float n2 = (float)sqrt((double)e * (1.0 - eps));
+        float n3 = (float)sqrt((double)e * (1.0 + eps));
+        int good = (float_bits(n0) == float_bits(n1)) && (float_bits(n1) == float_bits(n2)) &&
+                   (float_bits(n1) == float_bits(n3));
+        if (ok)
+            ok[j] = (uint8_t)good;
+        bad += good ? 0 : 1;
+    }
+    return bad;
+}
+
+/* ------------------------------------------------------------------ */
+/* Weight metric, Eq. 5 / Alg. 1 line 11, materialised.                */
+/* ------------------------------------------------------------------ */
+void oracle_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                  const float *norms, float *score /* [rows, cols] */)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j)
+            score[i * cols + j] = weight_metric(norms[j], load_elem(W, i * ldw + j, dtype));
+}
+
+/* ------------------------------------------------------------------ */
+/* Projection outlier statistic, Eq. 6 / Alg. 1 lines 13-15.           */
+/* ------------------------------------------------------------------ */
+/*
+ * sum   = sum_i sum_j (double) w_ij          (row-major order, fp64)
+ * tau   = (double)alpha * (sum / C)          (kept in fp64)
+ * O     = #{ (double) w_ij > tau }           (strict)
+ * certified = 1 iff O is unchanged when tau is moved by +-C*2^-52 relative,
+ *             i.e. no admissible fp64 summation order changes the count.
+ */
+void oracle_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                          const float *norms, float alpha, int64_t *outlier_count,
+                          double *score_sum, double *ratio_percent, int *certified)
+{
+    double sum = 0.0;
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j)
+            sum = sum + (double)weight_metric(norms[j], load_elem(W, i * ldw + j, dtype));
+
+    double C = (double)(rows * cols);
+    double mean = sum / C;
+    double tau = (double)alpha * mean;
+    double eps = C * ldexp(1.0, -52);
+    double tau_lo = tau * (1.0 - eps), tau_hi = tau * (1.0 + eps);
+
+    int64_t O = 0, O_lo = 0, O_hi = 0;
+#pragma omp parallel for schedule(static) reduction(+ : O, O_lo, O_hi)
+    for (int64_t i = 0; i < rows; ++i)
+        for (int64_t j = 0; j < cols; ++j) {
+            double s = (double)weight_metric(norms[j], load_elem(W, i * ldw + j, dtype));
+            O += (s > tau);
+            O_lo += (s > tau_lo);
+            O_hi += (s > tau_hi);
+        }
+    if (outlier_count) *outlier_count = O;
+    if (score_sum) *score_sum = sum;
+    if (ratio_percent) *ratio_percent = 100.0 * (double)O / C;
+    if (certified) *certified = (O == O_lo && O == O_hi);
+}
+
+/* ------------------------------------------------------------------ */
+/* normalize(R_LLM) + Projection Planner (Alg. 1 line 19; Section 3.3  */
+/* component 8; Eq. 1-2).                                              */
+/* ------------------------------------------------------------------ */
+/*
+ * The paper fixes only the properties: the targets average to p (Eq. 1-2,
+ * Projection Planner), and a projection with more outliers is pruned less
+ * (Section 3.1).  Reading taken: min-max normalise the ranks R_q = 100*O_q/C_q
+ * to r_q in [0,1]; give each projection the deviation d_q = 2*lambda*r_q;
+ * s_q = p + mean(d) - d_q.  Then mean(s) = p, s decreases in R, and
+ * max(s)-min(s) = 2*lambda.  mode 0 normalises over all N*M entries, mode 1
+ * separately over the N entries of each projection category m.
+ * s is clamped to [0, 1 - 1/cols_q]; k_q = floor(s_q * cols_q) weights are
+ * removed from every row.  Returns 0, or 1 if any clamp was applied.
+ */
+int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numels,
+                             const int64_t *cols, int n_layers, int n_proj, double p,
+                             double lambda, int mode, double *sparsity, int64_t *k_out)
+{
+    int total = n_layers * n_proj;
+    int clamped = 0;
+    double *R = (double *)malloc(sizeof(double) * (size_t)total);
+    for (int q = 0; q < total; ++q)
+        R[q] = 100.0 * (double)outlier_counts[q] / (double)numels[q];
+
+    int n_groups = (mode == 1) ? n_proj : 1;
+    for (int g = 0; g < n_groups; ++g) {
+        /* members of this normalisation group, in q order */
+        int first = (mode == 1) ? g : 0;
+        int step = (mode == 1) ? n_proj : 1;
+        int count = (mode == 1) ? n_layers : total;
+
+        double lo = R[first], hi = R[first];
+        for (int c = 0, q = first; c < count; ++c, q += step) {
+            if (R[q] < lo) lo = R[q];
+            if (R[q] > hi) hi = R[q];
+        }
+        if (hi == lo) {
+            for (int c = 0, q = first; c < count; ++c, q += step)
+                sparsity[q] = p;
+            continue;
+        }
+        double dsum = 0.0;
+        for (int c = 0, q = first; c < count; ++c, q += step) {
+            double r = (R[q] - lo) / (hi - lo);
+            double d = 2.0 * lambda * r;
+            dsum = dsum + d;
+        }
+        double dbar = dsum / (double)count;
+        for (int c = 0, q = first; c < count; ++c, q += step) {
+            double r = (R[q] - lo) / (hi - lo);
+            double d = 2.0 * lambda * r;
+            sparsity[q] = (p + dbar) - d;
+        }
+    }
+    for (int q = 0; q < total; ++q) {
+        double smax = 1.0 - 1.0 / (double)cols[q];
+        if (sparsity[q] < 0.0) { sparsity[q] = 0.0; clamped = 1; }
+        if (sparsity[q] > smax) { sparsity[q] = smax; clamped = 1; }
+        k_out[q] = (int64_t)floor(sparsity[q] * (double)cols[q]);
+    }
+    free(R);
+    return clamped;
+}
+
+/* ------------------------------------------------------------------ */
+/* Unstructured projection pruning (Section 4.1.3: "masked by setting  */
+/* their weights to zero"; Section 2.3: the lowest-ranking parameters   */
+/* are removed), per output row.                                        */
+/* ------------------------------------------------------------------ */
+typedef struct { uint32_t key; int64_t idx; } keyed_t;
+
+static int keyed_cmp(const void *a, const void *b)
+{
+    const keyed_t *x = (const keyed_t *)a, *y = (const keyed_t *)b;
+    if (x->key != y->key) return x->key < y->key ? -1 : 1;
+    if (x->idx != y->idx) return x->idx < y->idx ? -1 : 1;
+    return 0;
+}
+
+/*
+ * In every row the k entries that come first under (w_ij ascending, j
+ * ascending) are set to +0; all others keep their input bits.  mask (optional)
+ * is [rows, ceil(cols/32)] words, bit j%32 of word j/32 = 1 for a kept entry,
+ * padding bits 0.  W_out may be W_in.
+ */
+void oracle_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64_t cols,
+                               int64_t ldw, int dtype, const float *norms, int64_t k,
+                               uint32_t *mask)
+{
+    int64_t words = (cols + 31) / 32;
+#pragma omp parallel
+    {
+        keyed_t *order = (keyed_t *)malloc(sizeof(keyed_t) * (size_t)cols);
+        uint8_t *pruned = (uint8_t *)malloc((size_t)cols);
+#pragma omp for schedule(static)
+        for (int64_t i = 0; i < rows; ++i) {
+            for (int64_t j = 0; j < cols; ++j) {
+                order[j].key = score_key(weight_metric(norms[j], load_elem(W_in, i * ldw + j, dtype)));
+                order[j].idx = j;
+            }
+            qsort(order, (size_t)cols, sizeof(keyed_t), keyed_cmp);
+            memset(pruned, 0, (size_t)cols);
+            for (int64_t r = 0; r < k; ++r)
+                pruned[order[r].idx] = 1;
+
+            if (mask)
+                for (int64_t w = 0; w < words; ++w)
+                    mask[i * words + w] = 0;
+            for (int64_t j = 0; j < cols; ++j) {
+                if (dtype == ORACLE_F32) {
+                    uint32_t v = ((const uint32_t *)W_in)[i * ldw + j];
+                    ((uint32_t *)W_out)[i * ldw + j] = pruned[j] ? 0u : v;
+                } else {
+                    uint16_t v = ((const uint16_t *)W_in)[i * ldw + j];
+                    ((uint16_t *)W_out)[i * ldw + j] = pruned[j] ? (uint16_t)0 : v;
+                }
+                if (mask && !pruned[j])
+                    mask[i * words + j / 32] |= (uint32_t)1 << (j % 32);
+            }
+        }
+        free(order);
+        free(pruned);
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* Structured projection pruning (Section 4.1.3: remove the            */
+/* lowest-magnitude heads and channels; Section 2.3: structured         */
+/* pruning removes whole data structures, leaving smaller dense         */
+/* matrices).                                                           */
+/* ------------------------------------------------------------------ */
+/*
+ * Unit scores.  A row unit u is the row_group consecutive rows
+ * [u*row_group, (u+1)*row_group); a column unit likewise.  The score of a
+ * unit is the fp64 sum, in row-major order, of w_ij over its elements,
+ * rounded once to fp32.  norms == NULL means norm_j = 1 (pure magnitude).
+ */
+void oracle_unit_scores(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                        const float *norms, int64_t row_group, int64_t col_group,
+                        float *row_scores /* [rows/row_group] */,
+                        float *col_scores /* [cols/col_group] */)
+{
+    int64_t n_ru = rows / row_group, n_cu = cols / col_group;
+#pragma omp parallel for schedule(static)
+    for (int64_t u = 0; u < n_ru; ++u) {
+        double s = 0.0;
+        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i)
+            for (int64_t j = 0; j < cols; ++j)
+                s = s + (double)weight_metric(norms ? norms[j] : 1.0f, load_elem(W, i * ldw + j, dtype));
+        row_scores[u] = (float)s;
+    }
+#pragma omp parallel for schedule(static)
+    for (int64_t v = 0; v < n_cu; ++v) {
+        double s = 0.0;
+        for (int64_t i = 0; i < rows; ++i)
+            for (int64_t j = v * col_group; j < (v + 1) * col_group; ++j)
+                s = s + (double)weight_metric(norms ? norms[j] : 1.0f, load_elem(W, i * ldw + j, dtype));
+        col_scores[v] = (float)s;
+    }
+}
+
+/*
+ * Of n_units units, the (n_units - keep) that come first under (score
+ * ascending, index ascending) are removed; keep_list receives the surviving
+ * unit indices in ascending order.
+ */
+void oracle_rank_units(const float *scores, int64_t n_units, int64_t keep, int32_t *keep_list)
+{
+    keyed_t *order = (keyed_t *)malloc(sizeof(keyed_t) * (size_t)n_units);
+    uint8_t *removed = (uint8_t *)calloc((size_t)n_units, 1);
+    for (int64_t u = 0; u < n_units; ++u) {
+        order[u].key = score_key(scores[u]);
+        order[u].idx = u;
+    }
+    qsort(order, (size_t)n_units, sizeof(keyed_t), keyed_cmp);
+    for (int64_t r = 0; r < n_units - keep; ++r)
+        removed[order[r].idx] = 1;
+    int64_t out = 0;
+    for (int64_t u = 0; u < n_units; ++u)
+        if (!removed[u])
+            keep_list[out++] = (int32_t)u;
+    free(order);
+    free(removed);
+}
+
+/*
+ * Dense compaction: Wc[a, b] = W[row(a), col(b)] bit for bit, where row(a)
+ * walks the kept row units in list order (row_group rows each) and col(b) the
+ * kept column units.  Wc is [n_rk*row_group, n_ck*col_group], ld = its cols.
+ */
+void oracle_compact(const void *W, int64_t ldw, int dtype, const int32_t *row_keep, int64_t n_rk,
+                    int64_t row_group, const int32_t *col_keep, int64_t n_ck, int64_t col_group,
+                    void *Wc)
+{
+    int64_t out_cols = n_ck * col_group;
+    size_t esz = (dtype == ORACLE_F32) ? 4 : 2;
+#pragma omp parallel for schedule(static)
+    for (int64_t a = 0; a < n_rk * row_group; ++a) {
+        int64_t i = (int64_t)row_keep[a / row_group] * row_group + a % row_group;
+        for (int64_t b = 0; b < out_cols; ++b) {
+            int64_t j = (int64_t)col_keep[b / col_group] * col_group + b % col_group;
+            memcpy((char *)Wc + (size_t)(a * out_cols + b) * esz,
+                   (const char *)W + (size_t)(i * ldw + j) * esz, esz);
+        }
+    }
+}
+
+int oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}
