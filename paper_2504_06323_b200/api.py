@@ -1,0 +1,283 @@
+"""Thin Python binding of libmosaic.so (the C ABI declared in include/mosaic.h).
+
+Argument marshalling only: every function takes torch tensors that already
+live on the CUDA device (torch is used for device memory and streams), passes
+their raw pointers and sizes through ctypes, and raises `MosaicError` on a
+non-zero status.  All arithmetic of the method runs inside the library's CUDA
+kernels; there is no CPU fallback - if the library cannot be loaded the import
+of a function here fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmosaic.so")
+
+F32, BF16 = 0, 1
+RESET_ACCUM = 1
+GLOBAL_NORM, PER_CATEGORY_NORM = 0, 1
+ROWS_GIVEN, COLS_GIVEN, RANK_ONLY, SCORES_ONLY, SCORES_ACCUM = 1, 2, 4, 8, 16
+OK, ERR_INFEASIBLE = 0, -9
+
+# every symbol include/mosaic.h declares
+SYMBOLS = (
+    "mosaic_version", "mosaic_status_string",
+    "mosaic_act_norms_workspace_bytes", "mosaic_act_norms",
+    "mosaic_score",
+    "mosaic_outlier_ratio_workspace_bytes", "mosaic_outlier_ratio", "mosaic_ratio_from_count",
+    "mosaic_allocate_sparsity",
+    "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
+    "mosaic_prune_structured_compact_workspace_bytes", "mosaic_prune_structured_compact",
+    "mosaic_rank_units",
+)
+
+
+class MosaicError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libmosaic.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2504_06323_b200.build` "
+                "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        i64, vp, sz, ci, dbl, flt = C.c_int64, C.c_void_p, C.c_size_t, C.c_int, C.c_double, C.c_float
+        L.mosaic_version.restype = ci
+        L.mosaic_status_string.restype = C.c_char_p
+        L.mosaic_status_string.argtypes = [ci]
+        L.mosaic_act_norms_workspace_bytes.restype = sz
+        L.mosaic_act_norms_workspace_bytes.argtypes = [i64, i64]
+        L.mosaic_act_norms.restype = ci
+        L.mosaic_act_norms.argtypes = [vp, i64, i64, i64, ci, vp, vp, ci, vp, sz, vp]
+        L.mosaic_score.restype = ci
+        L.mosaic_score.argtypes = [vp, i64, i64, i64, ci, vp, vp, vp]
+        L.mosaic_outlier_ratio_workspace_bytes.restype = sz
+        L.mosaic_outlier_ratio_workspace_bytes.argtypes = [i64, i64]
+        L.mosaic_outlier_ratio.restype = ci
+        L.mosaic_outlier_ratio.argtypes = [vp, i64, i64, i64, ci, vp, flt, vp, vp, vp, sz, vp]
+        L.mosaic_ratio_from_count.restype = dbl
+        L.mosaic_ratio_from_count.argtypes = [i64, i64]
+        L.mosaic_allocate_sparsity.restype = ci
+        L.mosaic_allocate_sparsity.argtypes = [vp, vp, vp, ci, ci, dbl, dbl, ci, vp, vp]
+        L.mosaic_prune_unstructured_workspace_bytes.restype = sz
+        L.mosaic_prune_unstructured_workspace_bytes.argtypes = [i64, i64]
+        L.mosaic_prune_unstructured.restype = ci
+        L.mosaic_prune_unstructured.argtypes = [vp, vp, i64, i64, i64, ci, vp, i64, vp, vp, sz, vp]
+        L.mosaic_prune_structured_compact_workspace_bytes.restype = sz
+        L.mosaic_prune_structured_compact_workspace_bytes.argtypes = [i64, i64]
+        L.mosaic_prune_structured_compact.restype = ci
+        L.mosaic_prune_structured_compact.argtypes = [vp, i64, i64, i64, ci, vp, i64, i64, i64, i64, vp, vp, ci, vp,
+                                                      vp, vp, sz, vp]
+        L.mosaic_rank_units.restype = ci
+        L.mosaic_rank_units.argtypes = [vp, i64, i64, vp, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().mosaic_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str, allow=()):
+    if status != OK and status not in allow:
+        raise MosaicError(status, what)
+    return status
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.float32:
+        return F32
+    raise TypeError(f"unsupported dtype {t.dtype}: the library takes float32 or bfloat16")
+
+
+def _dev(t: torch.Tensor, name: str, dtype=None, ndim=None) -> torch.Tensor:
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise TypeError(f"{name} must be a CUDA tensor (no CPU path exists)")
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
+    if ndim is not None and t.dim() != ndim:
+        raise ValueError(f"{name} must have {ndim} dims")
+    return t
+
+
+def _mat(t: torch.Tensor, name: str):
+    _dev(t, name, ndim=2)
+    if t.stride(1) != 1:
+        raise ValueError(f"{name} must be row-major (unit stride along columns)")
+    return t.data_ptr(), t.shape[0], t.shape[1], (t.stride(0) if t.shape[0] > 1 else max(t.stride(0), t.shape[1]))
+
+
+def _ptr(t):
+    return None if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int | None:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream or None
+
+
+class Workspace:
+    """A caller-owned, growable scratch buffer (the library itself allocates nothing)."""
+
+    def __init__(self, device="cuda"):
+        self.device = torch.device(device)
+        self.buf = None
+
+    def get(self, nbytes: int) -> tuple[int, int]:
+        nbytes = max(int(nbytes), 256)
+        if self.buf is None or self.buf.numel() < nbytes:
+            self.buf = torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+        assert self.buf.data_ptr() % 256 == 0
+        return self.buf.data_ptr(), self.buf.numel()
+
+
+_default_ws: dict[int, Workspace] = {}
+
+
+def _ws(ws: Workspace | None, device) -> Workspace:
+    if ws is not None:
+        return ws
+    idx = torch.device(device).index
+    idx = torch.cuda.current_device() if idx is None else idx
+    if idx not in _default_ws:
+        _default_ws[idx] = Workspace(torch.device("cuda", idx))
+    return _default_ws[idx]
+
+
+# --------------------------------------------------------------------------- calls
+def mosaic_version() -> int:
+    return int(lib().mosaic_version())
+
+
+def mosaic_act_norms(X: torch.Tensor, sumsq_accum: torch.Tensor, norms_out: torch.Tensor | None = None,
+                     flags: int = 0, ws: Workspace | None = None, stream=None) -> None:
+    """sumsq_accum[j] += sum_t X[t,j]^2 (fp64); optionally norms_out = sqrt (Eq. 5's norm term)."""
+    xp, tokens, cols, ldx = _mat(X, "X")
+    _dev(sumsq_accum, "sumsq_accum", torch.float64)
+    if sumsq_accum.numel() != cols or (norms_out is not None and norms_out.numel() != cols):
+        raise ValueError("sumsq_accum / norms_out must have one entry per column of X")
+    if norms_out is not None:
+        _dev(norms_out, "norms_out", torch.float32)
+    L = lib()
+    wp, wn = _ws(ws, X.device).get(L.mosaic_act_norms_workspace_bytes(tokens, cols))
+    _check(L.mosaic_act_norms(xp, tokens, cols, ldx, _dtype_code(X), sumsq_accum.data_ptr(), _ptr(norms_out),
+                              int(flags), wp, wn, _stream(stream)), "mosaic_act_norms")
+
+
+def mosaic_score(W: torch.Tensor, norms: torch.Tensor, score_out: torch.Tensor, stream=None) -> None:
+    """score_out[i,j] = norms[j] * |W[i,j]| in fp32 (Eq. 5, materialised)."""
+    p, rows, cols, ldw = _mat(W, "W")
+    _dev(norms, "norms", torch.float32)
+    _dev(score_out, "score_out", torch.float32)
+    if norms.numel() != cols or tuple(score_out.shape) != (rows, cols) or not score_out.is_contiguous():
+        raise ValueError("norms must be [cols] and score_out a contiguous [rows, cols]")
+    _check(lib().mosaic_score(p, rows, cols, ldw, _dtype_code(W), norms.data_ptr(), score_out.data_ptr(),
+                              _stream(stream)), "mosaic_score")
+
+
+def mosaic_outlier_ratio(W: torch.Tensor, norms: torch.Tensor, alpha: float, outlier_count_out: torch.Tensor,
+                         score_sum_out: torch.Tensor | None = None, ws: Workspace | None = None, stream=None) -> None:
+    """Eq. 6: outlier_count_out[0] = #{score > alpha*mean(score)}; score_sum_out[0] = fp64 sum of scores."""
+    p, rows, cols, ldw = _mat(W, "W")
+    _dev(norms, "norms", torch.float32)
+    _dev(outlier_count_out, "outlier_count_out", torch.int64)
+    if score_sum_out is not None:
+        _dev(score_sum_out, "score_sum_out", torch.float64)
+    if norms.numel() != cols:
+        raise ValueError("norms must be [cols]")
+    L = lib()
+    wp, wn = _ws(ws, W.device).get(L.mosaic_outlier_ratio_workspace_bytes(rows, cols))
+    _check(L.mosaic_outlier_ratio(p, rows, cols, ldw, _dtype_code(W), norms.data_ptr(), float(alpha),
+                                  outlier_count_out.data_ptr(), _ptr(score_sum_out), wp, wn, _stream(stream)),
+           "mosaic_outlier_ratio")
+
+
+def mosaic_ratio_from_count(outlier_count: int, numel: int) -> float:
+    return float(lib().mosaic_ratio_from_count(int(outlier_count), int(numel)))
+
+
+def mosaic_allocate_sparsity(outlier_counts, numels, cols, n_layers: int, n_proj: int, p: float,
+                             lam: float = 0.08, mode: int = GLOBAL_NORM):
+    """Host call: (sparsity[N*M] fp64, k[N*M] int64, infeasible flag) from the outlier counts."""
+    n = n_layers * n_proj
+    I64 = C.c_int64 * n
+    oc, ne, cl = I64(*[int(v) for v in outlier_counts]), I64(*[int(v) for v in numels]), I64(*[int(v) for v in cols])
+    s, k = (C.c_double * n)(), I64()
+    st = _check(lib().mosaic_allocate_sparsity(C.addressof(oc), C.addressof(ne), C.addressof(cl), n_layers, n_proj,
+                                               float(p), float(lam), int(mode), C.addressof(s), C.addressof(k)),
+                "mosaic_allocate_sparsity", allow=(ERR_INFEASIBLE,))
+    return list(s), list(k), st == ERR_INFEASIBLE
+
+
+def mosaic_prune_unstructured(W_in: torch.Tensor, W_out: torch.Tensor, norms: torch.Tensor, k: int,
+                              mask_out: torch.Tensor | None = None, ws: Workspace | None = None, stream=None) -> None:
+    """Per row, zero the k entries first under (score asc, column asc); optional keep bitmask."""
+    p, rows, cols, ldw = _mat(W_in, "W_in")
+    po, r2, c2, ld2 = _mat(W_out, "W_out")
+    if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or (rows > 1 and ld2 != ldw):
+        raise ValueError("W_out must match W_in in shape, dtype and leading dimension")
+    _dev(norms, "norms", torch.float32)
+    if norms.numel() != cols:
+        raise ValueError("norms must be [cols]")
+    if mask_out is not None:
+        _dev(mask_out, "mask_out", torch.int32)
+        if tuple(mask_out.shape) != (rows, (cols + 31) // 32) or not mask_out.is_contiguous():
+            raise ValueError("mask_out must be a contiguous int32 [rows, ceil(cols/32)]")
+    _check(lib().mosaic_prune_unstructured(p, po, rows, cols, ldw, _dtype_code(W_in), norms.data_ptr(), int(k),
+                                           _ptr(mask_out), None, 0, _stream(stream)), "mosaic_prune_unstructured")
+
+
+def mosaic_prune_structured_compact(W_in: torch.Tensor, norms: torch.Tensor | None, row_group: int, col_group: int,
+                                    row_units_keep: int, col_units_keep: int, row_keep_units: torch.Tensor | None,
+                                    col_keep_units: torch.Tensor | None, flags: int = 0,
+                                    W_out: torch.Tensor | None = None, unit_scores_out: torch.Tensor | None = None,
+                                    ws: Workspace | None = None, stream=None) -> None:
+    """Unit scores -> ranked keep lists -> dense compacted W_out (see include/mosaic.h)."""
+    p, rows, cols, ldw = _mat(W_in, "W_in")
+    if norms is not None:
+        _dev(norms, "norms", torch.float32)
+    for t, nm, n in ((row_keep_units, "row_keep_units", row_units_keep), (col_keep_units, "col_keep_units", col_units_keep)):
+        if t is not None:
+            _dev(t, nm, torch.int32)
+            if t.numel() < n:
+                raise ValueError(f"{nm} is shorter than the number of kept units")
+    if W_out is not None:
+        _dev(W_out, "W_out", W_in.dtype)
+        if not W_out.is_contiguous() or W_out.numel() < row_units_keep * row_group * col_units_keep * col_group:
+            raise ValueError("W_out must be contiguous and hold the compacted matrix")
+    if unit_scores_out is not None:
+        _dev(unit_scores_out, "unit_scores_out", torch.float32)
+        if unit_scores_out.numel() < rows // row_group + cols // col_group:
+            raise ValueError("unit_scores_out too short")
+    L = lib()
+    wp, wn = _ws(ws, W_in.device).get(L.mosaic_prune_structured_compact_workspace_bytes(rows, cols))
+    _check(L.mosaic_prune_structured_compact(p, rows, cols, ldw, _dtype_code(W_in), _ptr(norms), int(row_group),
+                                             int(col_group), int(row_units_keep), int(col_units_keep),
+                                             _ptr(row_keep_units), _ptr(col_keep_units), int(flags), _ptr(W_out),
+                                             _ptr(unit_scores_out), wp, wn, _stream(stream)),
+           "mosaic_prune_structured_compact")
+
+
+def mosaic_rank_units(scores: torch.Tensor, keep: int, keep_out: torch.Tensor, stream=None) -> None:
+    """Ascending indices of the `keep` units that survive removal of the lowest-scored ones."""
+    _dev(scores, "scores", torch.float32)
+    _dev(keep_out, "keep_out", torch.int32)
+    if keep_out.numel() < keep:
+        raise ValueError("keep_out too short")
+    _check(lib().mosaic_rank_units(scores.data_ptr(), scores.numel(), int(keep), keep_out.data_ptr(), _stream(stream)),
+           "mosaic_rank_units")

@@ -1,0 +1,116 @@
+// Host-only entry points and argument validation shared by the device calls.
+#include <math.h>
+
+#include "common.cuh"
+
+namespace mosaic {
+
+int sm_count() {
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        (void)cudaGetLastError();
+        return 148;
+    }
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            (void)cudaGetLastError();
+            n = 148;
+        }
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+int check_matrix(const void* p, int64_t rows, int64_t cols, int64_t ld, int dtype) {
+    if (dtype != MOSAIC_F32 && dtype != MOSAIC_BF16) return MOSAIC_ERR_BAD_DTYPE;
+    if (rows < 0 || cols <= 0 || ld < cols) return MOSAIC_ERR_INVALID_ARG;
+    if (p == nullptr) return MOSAIC_ERR_NULL_PTR;
+    const int64_t per16 = 16 / (int64_t)elem_size(dtype);
+    if ((reinterpret_cast<uintptr_t>(p) & 15u) != 0 || (ld % per16) != 0) return MOSAIC_ERR_MISALIGNED;
+    return MOSAIC_OK;
+}
+
+}  // namespace mosaic
+
+extern "C" {
+
+int mosaic_version(void) { return MOSAIC_VERSION; }
+
+const char* mosaic_status_string(int status) {
+    switch (status) {
+        case MOSAIC_OK: return "ok";
+        case MOSAIC_ERR_INVALID_ARG: return "invalid argument";
+        case MOSAIC_ERR_NULL_PTR: return "null pointer";
+        case MOSAIC_ERR_BAD_DTYPE: return "unsupported dtype";
+        case MOSAIC_ERR_MISALIGNED: return "pointer or leading dimension not 16-byte aligned";
+        case MOSAIC_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case MOSAIC_ERR_ALIASING: return "input and output overlap";
+        case MOSAIC_ERR_CUDA: return "CUDA error";
+        case MOSAIC_ERR_NONFINITE: return "non-finite input";
+        case MOSAIC_ERR_INFEASIBLE: return "sparsity target clamped";
+        case MOSAIC_ERR_TIMEOUT: return "device wait timed out";
+        default: return "unknown status";
+    }
+}
+
+double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel) {
+    // Algorithm 1 line 15: R = O / C * 100
+    return 100.0 * (double)outlier_count / (double)numel;
+}
+
+// normalize(R_LLM) + Projection Planner; see mosaic.h for the definition.
+int mosaic_allocate_sparsity(const int64_t* outlier_counts, const int64_t* numels, const int64_t* cols,
+                             int n_layers, int n_proj, double p, double lambda, int mode,
+                             double* sparsity_out, int64_t* k_out) {
+    if (!outlier_counts || !numels || !cols || !sparsity_out || !k_out) return MOSAIC_ERR_NULL_PTR;
+    if (n_layers <= 0 || n_proj <= 0 || !(p >= 0.0 && p < 1.0) || !(lambda >= 0.0)) return MOSAIC_ERR_INVALID_ARG;
+    if (mode != MOSAIC_GLOBAL_NORM && mode != MOSAIC_PER_CATEGORY_NORM) return MOSAIC_ERR_INVALID_ARG;
+    const int total = n_layers * n_proj;
+    for (int q = 0; q < total; ++q)
+        if (numels[q] <= 0 || cols[q] <= 0 || outlier_counts[q] < 0 || outlier_counts[q] > numels[q])
+            return MOSAIC_ERR_INVALID_ARG;
+
+    const int n_groups = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_proj : 1;
+    const int stride = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_proj : 1;
+    const int members = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_layers : total;
+    for (int g = 0; g < n_groups; ++g) {
+        double lo = 0.0, hi = 0.0;
+        for (int c = 0; c < members; ++c) {
+            const int q = g + c * stride;
+            const double R = mosaic_ratio_from_count(outlier_counts[q], numels[q]);
+            if (c == 0 || R < lo) lo = R;
+            if (c == 0 || R > hi) hi = R;
+        }
+        if (hi == lo) {
+            for (int c = 0; c < members; ++c) sparsity_out[g + c * stride] = p;
+            continue;
+        }
+        const double range = hi - lo;
+        double dsum = 0.0;
+        for (int c = 0; c < members; ++c) {
+            const int q = g + c * stride;
+            const double r = (mosaic_ratio_from_count(outlier_counts[q], numels[q]) - lo) / range;
+            const double d = 2.0 * lambda * r;
+            dsum = dsum + d;
+        }
+        const double dbar = dsum / (double)members;
+        for (int c = 0; c < members; ++c) {
+            const int q = g + c * stride;
+            const double r = (mosaic_ratio_from_count(outlier_counts[q], numels[q]) - lo) / range;
+            const double d = 2.0 * lambda * r;
+            sparsity_out[q] = (p + dbar) - d;
+        }
+    }
+    int status = MOSAIC_OK;
+    for (int q = 0; q < total; ++q) {
+        const double smax = 1.0 - 1.0 / (double)cols[q];
+        if (sparsity_out[q] < 0.0) { sparsity_out[q] = 0.0; status = MOSAIC_ERR_INFEASIBLE; }
+        if (sparsity_out[q] > smax) { sparsity_out[q] = smax; status = MOSAIC_ERR_INFEASIBLE; }
+        k_out[q] = (int64_t)floor(sparsity_out[q] * (double)cols[q]);
+    }
+    return status;
+}
+
+}  // extern "C"

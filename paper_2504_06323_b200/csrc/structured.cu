@@ -1,0 +1,343 @@
+// mosaic_prune_structured_compact / mosaic_rank_units: structured projection
+// pruning (Section 4.1.3; Section 2.3) - unit scores, exact ranking of units,
+// dense compaction.
+//
+//   scores : row sums (one warp per row, fp64, fixed butterfly) and column sums
+//            (the two-stage column reduction shared with the activation norms),
+//            then one fp64 sum per unit over its rows / columns in index order,
+//            rounded once to fp32.
+//   rank   : one CTA per dimension; 4 x 8-bit radix select on the fp32 score
+//            bits finds the threshold key and tie quota; an ordered block scan
+//            then emits the ascending keep list (ties: lowest index removed
+//            first).
+//   compact: one CTA per output row; each thread gathers 8 output elements
+//            through the kept-column map and stores 16 bytes.
+#include "colreduce.cuh"
+
+namespace mosaic {
+
+constexpr int kRankThreads = 1024;
+
+struct StructWs {  // carve-up of the caller's workspace
+    double* row_sum;      // [rows]
+    double* col_partial;  // [splits, cols]
+    float* scores;        // [n_ru + n_cu]
+    size_t bytes;
+};
+
+static StructWs struct_ws(void* base, int64_t rows, int64_t cols) {
+    StructWs w;
+    char* p = static_cast<char*>(base);
+    size_t off = 0;
+    w.row_sum = reinterpret_cast<double*>(p + off);
+    off += align_up(sizeof(double) * (size_t)rows, 256);
+    const ColSplit cs = col_split_plan(rows, cols);
+    w.col_partial = reinterpret_cast<double*>(p + off);
+    off += align_up(sizeof(double) * (size_t)cs.splits * (size_t)cols, 256);
+    w.scores = reinterpret_cast<float*>(p + off);
+    off += align_up(sizeof(float) * (size_t)(rows + cols), 256);
+    w.bytes = off;
+    return w;
+}
+
+// One warp per row: fp64 sum of the weight metric along the row.
+template <int DT>
+__global__ void __launch_bounds__(256) row_sum_kernel(const void* __restrict__ W, int64_t rows, int64_t cols, int64_t ldw,
+                                                       const float* __restrict__ norms, double* __restrict__ row_sum) {
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t nvec = (cols + kVec - 1) / kVec;
+    for (int64_t row = warp; row < rows; row += nwarps) {
+        double acc = 0.0;
+        for (int64_t v = lane; v < nvec; v += 32) {
+            Raw8<DT> r;
+            const int64_t c0 = v * kVec;
+            load_vec<DT, true>(r, W, row * ldw, c0, cols);
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) {
+                const float n = (c0 + e < cols) ? (norms ? norms[c0 + e] : 1.0f) : 0.0f;
+                acc += (double)__fmul_rn(n, r.abs_f32(e));
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) row_sum[row] = acc;
+    }
+}
+
+// Unit score = fp64 sum of the unit's row sums (or of its columns' split partials), -> fp32.
+__global__ void unit_score_kernel(const double* __restrict__ row_sum, int64_t n_ru, int64_t row_group,
+                                  const double* __restrict__ col_partial, int splits, int64_t cols, int64_t n_cu,
+                                  int64_t col_group, float* __restrict__ out, int accumulate) {
+    const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u >= n_ru + n_cu) return;
+    double s = 0.0;
+    if (u < n_ru) {
+        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i) s += row_sum[i];
+    } else {
+        const int64_t v = u - n_ru;
+        for (int64_t c = v * col_group; c < (v + 1) * col_group; ++c) {
+            double cs = 0.0;
+            for (int p = 0; p < splits; ++p) cs += col_partial[(int64_t)p * cols + c];
+            s += cs;
+        }
+    }
+    const float f = (float)s;
+    out[u] = accumulate ? __fadd_rn(out[u], f) : f;
+}
+
+__device__ __forceinline__ uint32_t unit_key(float s) { return (s != s) ? 0xFFFFFFFFu : __float_as_uint(s); }
+
+// Keep list of one dimension: remove the (n - keep) units first under (score, index).
+__device__ void rank_units_block(const float* __restrict__ scores, int64_t n, int64_t keep, int32_t* __restrict__ keep_out) {
+    __shared__ uint32_t hist[256];
+    __shared__ uint32_t warp_tot[2][32];
+    __shared__ uint32_t sel_bin, sel_rank, sel_cnt;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int64_t remove = n - keep;
+    uint32_t T = 0u;
+    int64_t q = 0, n_eq = 0;  // q of the n_eq units with key == T are removed
+    if (remove > 0) {
+        uint32_t prefix = 0u, pmask = 0u;
+        int64_t rank = remove;
+        for (int shift = 24; shift >= 0; shift -= 8) {
+            if (tid < 256) hist[tid] = 0u;
+            __syncthreads();
+            for (int64_t u = tid; u < n; u += kRankThreads) {
+                const uint32_t key = unit_key(scores[u]);
+                if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFFu], 1u);
+            }
+            __syncthreads();
+            if (tid == 0) {
+                int64_t cum = 0;
+                for (int b = 0; b < 256; ++b) {
+                    if (rank <= cum + (int64_t)hist[b]) {
+                        sel_bin = (uint32_t)b;
+                        sel_rank = (uint32_t)(rank - cum);
+                        sel_cnt = hist[b];
+                        break;
+                    }
+                    cum += hist[b];
+                }
+            }
+            __syncthreads();
+            prefix |= sel_bin << shift;
+            pmask |= 0xFFu << shift;
+            rank = sel_rank;
+            n_eq = sel_cnt;
+            __syncthreads();
+        }
+        T = prefix;
+        q = rank;
+    }
+    // ordered emission, 1024 units per step
+    int64_t eq_before = 0, kept_before = 0;
+    for (int64_t base = 0; base < n; base += kRankThreads) {
+        const int64_t u = base + tid;
+        uint32_t is_eq = 0u, key = 0u;
+        if (u < n) {
+            key = unit_key(scores[u]);
+            is_eq = (remove > 0 && key == T) ? 1u : 0u;
+        }
+        // scan of the tie indicator
+        uint32_t incl = is_eq;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) warp_tot[0][wid] = incl;
+        __syncthreads();
+        uint32_t eq_excl = incl - is_eq, eq_total = 0u;
+        for (int w = 0; w < kRankThreads / 32; ++w) {
+            const uint32_t t = warp_tot[0][w];
+            if (w < wid) eq_excl += t;
+            eq_total += t;
+        }
+        uint32_t kept = 0u;
+        if (u < n) {
+            if (remove == 0) kept = 1u;
+            else if (key > T) kept = 1u;
+            else if (key == T) kept = (eq_before + (int64_t)eq_excl >= q) ? 1u : 0u;
+        }
+        uint32_t kincl = kept;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, kincl, o);
+            if (lane >= o) kincl += v;
+        }
+        if (lane == 31) warp_tot[1][wid] = kincl;
+        __syncthreads();
+        uint32_t k_excl = kincl - kept, k_total = 0u;
+        for (int w = 0; w < kRankThreads / 32; ++w) {
+            const uint32_t t = warp_tot[1][w];
+            if (w < wid) k_excl += t;
+            k_total += t;
+        }
+        if (kept) {
+            const int64_t pos = kept_before + (int64_t)k_excl;
+            if (pos < keep) keep_out[pos] = (int32_t)u;
+        }
+        eq_before += eq_total;
+        kept_before += k_total;
+        __syncthreads();
+    }
+    (void)n_eq;
+}
+
+// blockIdx.x == 0 ranks the row units, 1 the column units (either may be skipped).
+__global__ void __launch_bounds__(kRankThreads) rank_kernel(const float* row_scores, int64_t n_ru, int64_t row_keep,
+                                                             int32_t* row_out, const float* col_scores, int64_t n_cu,
+                                                             int64_t col_keep, int32_t* col_out) {
+    if (blockIdx.x == 0) {
+        if (row_out) rank_units_block(row_scores, n_ru, row_keep, row_out);
+    } else {
+        if (col_out) rank_units_block(col_scores, n_cu, col_keep, col_out);
+    }
+}
+
+// Dense gather.  grid.x = output rows; threads walk output vectors of 8 elements.
+template <int DT>
+__global__ void __launch_bounds__(256) compact_kernel(const void* __restrict__ W, int64_t ldw, const int32_t* __restrict__ row_keep,
+                                                       int64_t n_ru, int64_t row_group, const int32_t* __restrict__ col_keep,
+                                                       int64_t n_cu, int64_t col_group, int64_t out_cols, void* __restrict__ out) {
+    constexpr int esz = (DT == MOSAIC_F32) ? 4 : 2;
+    const int64_t a = blockIdx.x;
+    int64_t ru = row_keep[a / row_group];
+    ru = ru < 0 ? 0 : (ru >= n_ru ? n_ru - 1 : ru);
+    const int64_t src_row = ru * row_group + a % row_group;
+    const int64_t nvec = (out_cols + kVec - 1) / kVec;
+    const bool vec_ok = (out_cols % kVec) == 0;   // every output row then starts 16-byte aligned
+    for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+        Raw8<DT> r;
+        r.clear();
+        const int64_t b0 = v * kVec;
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+            const int64_t b = b0 + e;
+            if (b < out_cols) {
+                int64_t cu = (col_group == 1) ? (int64_t)col_keep[b] : (int64_t)col_keep[b / col_group];
+                cu = cu < 0 ? 0 : (cu >= n_cu ? n_cu - 1 : cu);
+                const int64_t j = (col_group == 1) ? cu : cu * col_group + b % col_group;
+                r.set_scalar(e, W, src_row * ldw + j);
+            }
+        }
+        if (vec_ok) {
+            r.store((char*)out + (a * out_cols + b0) * esz);
+        } else {
+#pragma unroll
+            for (int e = 0; e < kVec; ++e)
+                if (b0 + e < out_cols) r.put_scalar(e, out, a * out_cols + b0 + e);
+        }
+    }
+}
+
+}  // namespace mosaic
+
+using namespace mosaic;
+
+extern "C" size_t mosaic_prune_structured_compact_workspace_bytes(int64_t rows, int64_t cols) {
+    if (rows <= 0 || cols <= 0) return 256;
+    return struct_ws(nullptr, rows, cols).bytes;
+}
+
+extern "C" int mosaic_rank_units(const float* scores, int64_t n_units, int64_t keep, int32_t* keep_out, void* stream) {
+    if (!scores || (!keep_out && keep > 0)) return MOSAIC_ERR_NULL_PTR;
+    if (n_units <= 0 || keep < 0 || keep > n_units || n_units > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    if (keep == 0) return MOSAIC_OK;
+    rank_kernel<<<1, kRankThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, n_units, keep, keep_out, nullptr, 0, 0,
+                                                                          nullptr);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                                               const float* norms, int64_t row_group, int64_t col_group,
+                                               int64_t row_units_keep, int64_t col_units_keep, int32_t* row_keep_units,
+                                               int32_t* col_keep_units, int flags, void* W_out, float* unit_scores_out,
+                                               void* ws, size_t ws_bytes, void* stream) {
+    int rc = check_matrix(W_in, rows, cols, ldw, dtype);
+    if (rc != MOSAIC_OK) return rc;
+    const int known = MOSAIC_ROWS_GIVEN | MOSAIC_COLS_GIVEN | MOSAIC_RANK_ONLY | MOSAIC_SCORES_ONLY | MOSAIC_SCORES_ACCUM;
+    if (rows == 0 || (flags & ~known) || row_group <= 0 || col_group <= 0 || rows % row_group || cols % col_group)
+        return MOSAIC_ERR_INVALID_ARG;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    const int64_t n_ru = rows / row_group, n_cu = cols / col_group;
+    const bool scores_only = flags & MOSAIC_SCORES_ONLY;
+    const bool rank_only = flags & MOSAIC_RANK_ONLY;
+    const bool rows_given = flags & MOSAIC_ROWS_GIVEN, cols_given = flags & MOSAIC_COLS_GIVEN;
+    if ((flags & MOSAIC_SCORES_ACCUM) && !unit_scores_out) return MOSAIC_ERR_NULL_PTR;
+    if (scores_only && !unit_scores_out) return MOSAIC_ERR_NULL_PTR;
+    if (!scores_only) {
+        if (row_units_keep < 1 || row_units_keep > n_ru || col_units_keep < 1 || col_units_keep > n_cu)
+            return MOSAIC_ERR_INVALID_ARG;
+        if (!row_keep_units || !col_keep_units) return MOSAIC_ERR_NULL_PTR;
+        if ((reinterpret_cast<uintptr_t>(row_keep_units) & 3u) || (reinterpret_cast<uintptr_t>(col_keep_units) & 3u))
+            return MOSAIC_ERR_MISALIGNED;
+    }
+    const bool need_scores = scores_only || unit_scores_out || !(rows_given && cols_given);
+    const int64_t out_rows = row_units_keep * row_group, out_cols = col_units_keep * col_group;
+    if (!scores_only && !rank_only) {
+        if (!W_out) return MOSAIC_ERR_NULL_PTR;
+        if (reinterpret_cast<uintptr_t>(W_out) & 15u) return MOSAIC_ERR_MISALIGNED;
+        const size_t in_span = ((size_t)(rows - 1) * (size_t)ldw + (size_t)cols) * elem_size(dtype);
+        const size_t out_span = (size_t)out_rows * (size_t)out_cols * elem_size(dtype);
+        const char *a = static_cast<const char*>(W_in), *b = static_cast<const char*>(W_out);
+        if (a < b + out_span && b < a + in_span) return MOSAIC_ERR_ALIASING;
+    }
+    if ((reinterpret_cast<uintptr_t>(norms) & 3u) || (reinterpret_cast<uintptr_t>(unit_scores_out) & 3u))
+        return MOSAIC_ERR_MISALIGNED;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    StructWs w{};
+    if (need_scores) {
+        if (!ws) return MOSAIC_ERR_NULL_PTR;
+        if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
+        if (ws_bytes < mosaic_prune_structured_compact_workspace_bytes(rows, cols)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+        w = struct_ws(ws, rows, cols);
+        const ColSplit cs = col_split_plan(rows, cols);
+        int64_t rblocks = (rows + 7) / 8;
+        const int64_t cap = (int64_t)sm_count() * 8;
+        if (rblocks > cap) rblocks = cap;
+        dim3 cgrid((unsigned)((cols + kColTile - 1) / kColTile), (unsigned)cs.splits);
+        if (dtype == MOSAIC_BF16) {
+            row_sum_kernel<MOSAIC_BF16><<<(unsigned)rblocks, 256, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_sum);
+            MOSAIC_LAUNCH_CHECK();
+            col_partial_kernel<MOSAIC_BF16, COL_SCORE><<<cgrid, kColTile, 0, st>>>(W_in, rows, cols, ldw, norms,
+                                                                                   cs.rows_per_split, w.col_partial);
+        } else {
+            row_sum_kernel<MOSAIC_F32><<<(unsigned)rblocks, 256, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_sum);
+            MOSAIC_LAUNCH_CHECK();
+            col_partial_kernel<MOSAIC_F32, COL_SCORE><<<cgrid, kColTile, 0, st>>>(W_in, rows, cols, ldw, norms,
+                                                                                  cs.rows_per_split, w.col_partial);
+        }
+        MOSAIC_LAUNCH_CHECK();
+        // with SCORES_ACCUM the running totals live in the caller's array; ranking then uses those
+        float* dst = (flags & MOSAIC_SCORES_ACCUM) ? unit_scores_out : w.scores;
+        const int64_t nu = n_ru + n_cu;
+        unit_score_kernel<<<(unsigned)((nu + 127) / 128), 128, 0, st>>>(w.row_sum, n_ru, row_group, w.col_partial, cs.splits,
+                                                                       cols, n_cu, col_group, dst,
+                                                                       (flags & MOSAIC_SCORES_ACCUM) ? 1 : 0);
+        MOSAIC_LAUNCH_CHECK();
+        if (unit_scores_out && dst != unit_scores_out)
+            MOSAIC_CUDA_TRY(cudaMemcpyAsync(unit_scores_out, dst, sizeof(float) * (size_t)nu, cudaMemcpyDeviceToDevice, st));
+        w.scores = dst;
+    }
+    if (scores_only) return MOSAIC_OK;
+
+    if (!(rows_given && cols_given)) {
+        rank_kernel<<<2, kRankThreads, 0, st>>>(w.scores, n_ru, row_units_keep, rows_given ? nullptr : row_keep_units,
+                                                w.scores + n_ru, n_cu, col_units_keep, cols_given ? nullptr : col_keep_units);
+        MOSAIC_LAUNCH_CHECK();
+    }
+    if (rank_only) return MOSAIC_OK;
+
+    if (dtype == MOSAIC_BF16)
+        compact_kernel<MOSAIC_BF16><<<(unsigned)out_rows, 256, 0, st>>>(W_in, ldw, row_keep_units, n_ru, row_group,
+                                                                       col_keep_units, n_cu, col_group, out_cols, W_out);
+    else
+        compact_kernel<MOSAIC_F32><<<(unsigned)out_rows, 256, 0, st>>>(W_in, ldw, row_keep_units, n_ru, row_group,
+                                                                      col_keep_units, n_cu, col_group, out_cols, W_out);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}

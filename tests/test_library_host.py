@@ -1,0 +1,91 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every symbol the
+header declares, validates arguments before touching the device, and its host
+function mosaic_allocate_sparsity agrees bit for bit with the oracle."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2504_06323_b200 import api, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return api.lib()
+
+
+def header_symbols():
+    text = open(os.path.join(ROOT, "include", "mosaic.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mosaic_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = header_symbols()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(lib, n), n
+    assert set(api.SYMBOLS) == set(names)
+    assert lib.mosaic_version() == 100
+
+
+def test_status_strings(lib):
+    seen = set()
+    for s in range(0, -11, -1):
+        txt = api.status_string(s)
+        assert txt and txt != "unknown status"
+        seen.add(txt)
+    assert len(seen) == 11
+    assert api.status_string(-99) == "unknown status"
+
+
+def test_argument_validation_needs_no_device(lib):
+    # every one of these is rejected before any CUDA call is made
+    assert lib.mosaic_act_norms(None, 4, 4, 4, 7, None, None, 0, None, 0, None) == -3       # bad dtype
+    assert lib.mosaic_act_norms(None, 4, 4, 4, 0, None, None, 0, None, 0, None) == -2       # null accum
+    assert lib.mosaic_score(None, 4, 4, 4, 1, None, None, None) == -2
+    assert lib.mosaic_score(16, 4, 4, 3, 1, 16, 16, None) == -1                              # ld < cols
+    assert lib.mosaic_score(8, 4, 8, 8, 1, 16, 16, None) == -4                               # misaligned base
+    assert lib.mosaic_score(16, 4, 8, 12, 1, 16, 16, None) == -4                             # ld not 16 B multiple
+    assert lib.mosaic_prune_unstructured(16, 16, 4, 8, 8, 1, 16, 9, None, None, 0, None) == -1   # k > cols
+    assert lib.mosaic_prune_unstructured(16, 32, 4, 8, 8, 1, 16, 1, None, None, 0, None) == -6   # partial overlap
+    assert lib.mosaic_outlier_ratio(16, 4, 8, 8, 1, 16, 5.0, 16, None, 256, 16, None) == -5      # workspace too small
+    assert lib.mosaic_prune_structured_compact(16, 4, 8, 8, 1, None, 3, 1, 1, 1, 16, 16, 0, 4096, None, 256, 1 << 20,
+                                               None) == -1                                   # rows % row_group
+    assert lib.mosaic_rank_units(16, 4, 5, 16, None) == -1                                   # keep > n
+    assert lib.mosaic_ratio_from_count(3, 200) == 1.5
+    assert lib.mosaic_act_norms_workspace_bytes(262144, 4096) % 256 == 0
+
+
+@pytest.mark.parametrize("mode", [api.GLOBAL_NORM, api.PER_CATEGORY_NORM])
+@pytest.mark.parametrize("p,lam", [(0.5, 0.08), (0.8, 0.15), (0.1, 0.0), (0.7, 0.3)])
+def test_allocate_sparsity_bit_exact_vs_oracle(lib, mode, p, lam):
+    rng = np.random.default_rng(42)
+    for N, M in [(1, 7), (32, 7), (40, 7), (3, 2)]:
+        numel = rng.integers(1 << 16, 1 << 26, N * M)
+        O = (numel * rng.random(N * M) * 0.02).astype(np.int64)
+        cols = rng.choice([256, 688, 4096, 5120, 11008, 14336], N * M)
+        s_ref, k_ref, clamp_ref = oracle.allocate_sparsity(O, numel, cols, N, M, p, lam, mode)
+        s, k, clamp = api.mosaic_allocate_sparsity(O, numel, cols, N, M, p, lam, mode)
+        assert np.array_equal(np.array(s).view(np.uint64), s_ref.view(np.uint64))     # bit-exact fp64
+        assert list(k) == list(k_ref) and clamp == clamp_ref
+
+
+def test_allocate_sparsity_errors(lib):
+    with pytest.raises(api.MosaicError):
+        api.mosaic_allocate_sparsity([1], [10], [8], 1, 1, 1.0)          # p must be < 1
+    with pytest.raises(api.MosaicError):
+        api.mosaic_allocate_sparsity([11], [10], [8], 1, 1, 0.5)         # more outliers than elements
+    s, k, infeasible = api.mosaic_allocate_sparsity([0, 50], [100, 100], [64, 64], 1, 2, 0.95, 0.2)
+    assert infeasible and k[0] == 63
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    with pytest.raises(TypeError):
+        api.mosaic_score(torch.zeros(4, 8), torch.zeros(8), torch.zeros(4, 8))
