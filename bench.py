@@ -1,0 +1,426 @@
+#!/usr/bin/env python
+"""Benchmark of the Mosaic pruning hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl native|reference]
+
+A step is one pass of the whole path over a LLaMA-7B-shaped model (32 layers,
+bf16, 128 x 2048 calibration tokens per projection input): activation norms
+for every projection input, outlier count of every projection, the host
+allocation of the 224 sparsity targets, and the per-row unstructured
+selection + zeroing (+ keep bitmask) of every projection at 50 % average
+sparsity.  The metric is weight GB/s: bytes of weights scored and pruned per
+second of step time.  One JSON line is printed by rank 0.
+
+With N > 1 (torchrun, one process per GPU) every rank owns 32 layers of a
+32*N-layer model (weak scaling); the only exchange is one all_gather of the
+outlier counts between the two phases.
+
+--impl reference times the CPU oracle (as it stands) on the host cores over a
+bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2504_06323_b200 import workloads as wl  # noqa: E402
+from paper_2504_06323_b200.workloads import PROJECTIONS  # noqa: E402
+
+METRIC = "weight_GBps_scored_and_pruned"
+UNIT = "GB/s"
+
+# DRAM traffic per launch of the dominant kernel from an ncu capture (bytes read + written
+# divided by the bytes of X the launch reduces); see profiles/.  None until captured.
+NCU_TRAFFIC_RATIO = {"col_partial_kernel": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled every 200 ms while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "200", "-f", self.path], stdout=subprocess.DEVNULL, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm = [float(r[0]) for r in rows if len(r) >= 7]
+            if sm:
+                busy = [s for s, r in zip(sm, rows) if float(r[2]) > 250.0] or sm
+                out["sm_mhz"] = statistics.median(busy)
+                out["sm_max_mhz"] = float(rows[0][1])
+                names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+                out["reasons"] = [n for i, n in enumerate(names) if any(r[3 + i].strip() == "Active" for r in rows)]
+                out["samples"] = len(sm)
+        except Exception:
+            pass
+        return out
+
+
+# --------------------------------------------------------------------------- CPU oracle sample
+def oracle_sample_inputs(cfg, frac_div: int, device):
+    """1/frac_div of one layer: tokens/frac_div calibration tokens per input and rows/frac_div rows
+    of each of the seven projections (so activation and weight work keep the model's ratio)."""
+    T = cfg.tokens // frac_div
+    X = {xk: wl.to_numpy(wl.gen_activation(cfg, 0, xk, device, tokens=T)) for xk in cfg.x_keys()}
+    W = {}
+    for pr in PROJECTIONS:
+        rows, cols = cfg.shape(pr)
+        W[pr] = wl.to_numpy(wl.gen_weight(cfg, 0, pr, device, shape=(max(rows // frac_div, 1), cols)))
+    return X, W
+
+
+def oracle_sample_step(cfg, X, W):
+    """The path on the sample, oracle calls only.  Returns weight bytes processed."""
+    import oracle
+    norms = {xk: oracle.act_norms(x, cfg.dtype) for xk, x in X.items()}
+    counts, numels, cols = [], [], []
+    for pr in PROJECTIONS:
+        r = oracle.outlier_ratio(W[pr], norms[cfg.x_key(pr)], cfg.alpha, cfg.dtype)
+        counts.append(r["count"])
+        numels.append(r["numel"])
+        cols.append(W[pr].shape[1])
+    _, k, _ = oracle.allocate_sparsity(counts, numels, cols, 1, len(PROJECTIONS), cfg.p, cfg.lam)
+    for m, pr in enumerate(PROJECTIONS):
+        oracle.prune_unstructured(W[pr], norms[cfg.x_key(pr)], int(k[m]), cfg.dtype)
+    return sum(w.size * w.itemsize for w in W.values())
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    device = "cuda" if torch.cuda.is_available() else "cpu"
+    frac_div = 32
+    X, W = oracle_sample_inputs(cfg, frac_div, device)
+    for _ in range(args.warmup):
+        oracle_sample_step(cfg, X, W)
+    t0 = time.perf_counter()
+    nbytes = 0
+    for _ in range(args.steps):
+        nbytes += oracle_sample_step(cfg, X, W)
+    dt = time.perf_counter() - t0
+    value = nbytes / dt / 1e9
+    sample = f"1/{frac_div} of one layer per step: {cfg.tokens // frac_div} tokens per input, rows/{frac_div} of each projection"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "llama7b: 32 layers, hidden 4096, MLP 11008, bf16, 128x2048 calibration tokens, "
+                               "unstructured 50% (oracle on a bounded sample)", "inputs": "larger than L2"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------- native arm
+def run_native(args, cfg):
+    import torch.distributed as dist
+    from paper_2504_06323_b200 import api, build, driver
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if not os.path.exists(api.LIB_PATH):
+        if rank == 0:
+            build.build_library()
+        if world > 1:
+            dist.barrier()
+    api.lib()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    n_layers = args.layers or cfg.n_layers
+    total_cfg = wl.scaled(cfg, n_layers=n_layers * world)            # weak scaling: each rank owns n_layers layers
+    mine = driver.layers_of_rank(total_cfg.n_layers, rank, world)
+    st = driver.alloc_model(total_cfg, dev, mine)
+    # One layer's calibration activations, resident in HBM and reused for every layer
+    # (12.2 GB for the 7B shape: far larger than L2; a whole model's 391 GB would not fit).
+    X = driver.make_activations(cfg, 0, dev, tokens=args.tokens or cfg.tokens)
+    M = len(PROJECTIONS)
+    w_bytes = sum(st.W[l, p].numel() * cfg.itemsize for l in mine for p in PROJECTIONS)
+    x_bytes_layer = sum(x.numel() * cfg.itemsize for x in X.values())
+
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+
+    def step(record=False):
+        launches = 0
+        if record: ev[0].record()
+        for layer in mine:
+            launches += 2 * driver.accumulate_norms(st, layer, X)
+        if record: ev[1].record()
+        for layer in mine:
+            launches += 2 * driver.count_outliers(st, layer)
+        if record: ev[2].record()
+        counts = driver.exchange_counts(st.counts, total_cfg.n_layers, rank, world)
+        _, k, _ = driver.plan_sparsity(total_cfg, counts)
+        if record: ev[3].record()
+        for layer in mine:
+            launches += driver.prune_unstructured_layer(st, layer, k)
+        if record: ev[4].record()
+        return launches
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    phase_ms = [0.0, 0.0, 0.0, 0.0]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    launches = 0
+    phase_events = []
+    for _ in range(args.steps):
+        launches += step(record=False)
+    end.record()
+    barrier()
+    total_ms = start.elapsed_time(end)
+    # phase breakdown on separate (untimed) steps so that event bookkeeping does not sit in the timed region
+    for _ in range(3):
+        step(record=True)
+        torch.cuda.synchronize()
+        for i in range(4):
+            phase_ms[i] += ev[i].elapsed_time(ev[i + 1]) / 3.0
+    clocks = sampler.stop() if rank == 0 else None
+
+    t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_per_step = t.item() / args.steps
+    value = w_bytes * world / (ms_per_step * 1e-3) / 1e9
+
+    # ---- end to end from pinned host buffers (weights and activations in, pruned weights out)
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, cfg, total_cfg, st, mine, dev, rank, world, barrier)
+
+    # ---- CPU oracle on a bounded sample (rank 0, N = 1 only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        import oracle
+        frac_div, reps = 2, 4
+        Xs, Ws = oracle_sample_inputs(cfg, frac_div, dev)
+        t0 = time.perf_counter()
+        nb = sum(oracle_sample_step(cfg, Xs, Ws) for _ in range(reps))
+        dt = time.perf_counter() - t0
+        cpu = {"value": nb / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{reps} passes over 1/{frac_div} of one layer: {cfg.tokens // frac_div} calibration tokens "
+                         f"per input and rows/{frac_div} of each of the 7 projections ({nb / 1e6:.1f} MB of weights "
+                         f"in {dt:.1f} s)"}
+        del Xs, Ws
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    peak, peak_kind = measured_peaks()
+    n_act_launch = len(mine) * len(X)
+    act_bytes = x_bytes_layer * len(mine)
+    act_gbs = act_bytes / (phase_ms[0] * 1e-3) / 1e9
+    ratio = NCU_TRAFFIC_RATIO["col_partial_kernel"]
+    roofline = {
+        "kernel": "col_partial_kernel<bf16, square> (activation norms)", "bound": "hbm", "achieved": act_gbs,
+        "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": act_gbs / peak,
+        "traffic": None if ratio is None else ratio * act_bytes / n_act_launch,
+        "algorithmic_bytes_per_launch": act_bytes / n_act_launch, "launches_per_step": n_act_launch,
+        "avg_launch_ms": phase_ms[0] / n_act_launch,
+    }
+    outl_gbs = w_bytes / (phase_ms[1] * 1e-3) / 1e9
+    prune_gbs = w_bytes * 4.125 / 2 / (phase_ms[3] * 1e-3) / 1e9
+    weight_pass_ms = phase_ms[1] + phase_ms[2] + phase_ms[3]
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": f"{cfg.name}: {n_layers} layers/GPU, hidden {cfg.hidden}, MLP {cfg.intermediate}, bf16 "
+                               f"Student-t weights, {args.tokens or cfg.tokens} calibration tokens per projection input "
+                               f"(one layer's activations resident and reused by every layer), alpha {cfg.alpha}, "
+                               f"unstructured p={cfg.p}, lambda={cfg.lam}",
+                   "inputs": "larger than L2 (25.1 GB per step vs 126 MB)", "parallelism": f"layers sharded over {world} GPU(s)"},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+        "roofline": roofline, "cpu_baseline": cpu,
+        "phases_ms": {"act_norms": phase_ms[0], "outlier_ratio": phase_ms[1], "counts_d2h_allocate": phase_ms[2],
+                      "prune_unstructured": phase_ms[3]},
+        "weight_pass": {"ms": weight_pass_ms, "weight_GBps": w_bytes / (weight_pass_ms * 1e-3) / 1e9,
+                        "compulsory_GBps": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9,
+                        "frac_of_peak": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / peak,
+                        "frac_of_8TBps": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / 8000.0},
+        "roofline_other": [
+            {"kernel": "score_sum_kernel + outlier_count_kernel", "bound": "hbm", "achieved": outl_gbs, "peak": peak,
+             "unit": "GB/s", "frac": outl_gbs / peak, "algorithmic_bytes": "2 B/weight"},
+            {"kernel": "prune_rows_kernel", "bound": "hbm", "achieved": prune_gbs, "peak": peak, "unit": "GB/s",
+             "frac": prune_gbs / peak, "algorithmic_bytes": "4.125 B/weight"}],
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, cfg, total_cfg, st, mine, dev, rank, world, barrier):
+    """Same step, but every input starts in pinned host memory and the pruned weights end there:
+    weights H2D once per step, calibration activations streamed H2D in token chunks through two
+    device staging slots (copy stream) while the previous chunk is reduced (compute stream),
+    counts D2H, allocation, pruning, pruned weights D2H."""
+    import torch.distributed as dist
+    from paper_2504_06323_b200 import api, driver
+    M = len(PROJECTIONS)
+    tokens = args.tokens or cfg.tokens
+    chunk = min(args.e2e_chunk, tokens)
+    n_chunks = (tokens + chunk - 1) // chunk
+    host_x = {xk: torch.randn(chunk, cfg.x_cols(xk), dtype=torch.float32).to(cfg.torch_dtype).pin_memory()
+              for xk in cfg.x_keys()}
+    stage = {xk: [torch.empty(chunk, cfg.x_cols(xk), dtype=cfg.torch_dtype, device=dev) for _ in range(2)]
+             for xk in cfg.x_keys()}
+    host_w = {key: torch.empty(w.shape, dtype=w.dtype).pin_memory() for key, w in st.W.items()}
+    for key, w in st.W.items():
+        host_w[key].copy_(w)
+    host_out = {key: torch.empty(w.shape, dtype=w.dtype).pin_memory() for key, w in st.W.items()}
+    copy_s = torch.cuda.Stream(dev)
+    comp_s = torch.cuda.current_stream(dev)
+    h2d = sum(w.numel() * w.element_size() for w in host_w.values()) + \
+        len(mine) * n_chunks * sum(x.numel() * x.element_size() for x in host_x.values())
+    d2h = sum(w.numel() * w.element_size() for w in host_out.values()) + st.counts.numel() * 8
+    free_ev = {(xk, s): None for xk in host_x for s in range(2)}
+
+    def e2e_step():
+        with torch.cuda.stream(copy_s):
+            for key in st.W:
+                st.W[key].copy_(host_w[key], non_blocking=True)
+            w_ready = torch.cuda.Event()
+            w_ready.record(copy_s)
+        i = 0
+        for layer in mine:
+            for c in range(n_chunks):
+                slot = i % 2
+                i += 1
+                t = min(chunk, tokens - c * chunk)
+                for xk in host_x:
+                    if free_ev[xk, slot] is not None:
+                        copy_s.wait_event(free_ev[xk, slot])
+                    with torch.cuda.stream(copy_s):
+                        stage[xk][slot][:t].copy_(host_x[xk][:t], non_blocking=True)
+                        ready = torch.cuda.Event()
+                        ready.record(copy_s)
+                    comp_s.wait_event(ready)
+                    api.mosaic_act_norms(stage[xk][slot][:t], st.sumsq[layer, xk],
+                                         st.norms[layer, xk] if c == n_chunks - 1 else None,
+                                         api.RESET_ACCUM if c == 0 else 0, st.ws)
+                    done = torch.cuda.Event()
+                    done.record(comp_s)
+                    free_ev[xk, slot] = done
+        comp_s.wait_event(w_ready)
+        for layer in mine:
+            driver.count_outliers(st, layer)
+        counts = driver.exchange_counts(st.counts, total_cfg.n_layers, rank, world)
+        _, k, _ = driver.plan_sparsity(total_cfg, counts)
+        for layer in mine:
+            driver.prune_unstructured_layer(st, layer, k)
+            done = torch.cuda.Event()
+            done.record(comp_s)
+            copy_s.wait_event(done)
+            with torch.cuda.stream(copy_s):
+                for pr in PROJECTIONS:
+                    host_out[layer, pr].copy_(st.W_out[layer, pr], non_blocking=True)
+        fin = torch.cuda.Event()
+        fin.record(copy_s)
+        comp_s.wait_event(fin)
+
+    for _ in range(args.e2e_warmup):
+        e2e_step()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = t.item() / args.e2e_steps
+    w_bytes = sum(w.numel() * w.element_size() for w in host_w.values())
+    return {"value": w_bytes * world / (ms * 1e-3) / 1e9, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": ms, "steps": args.e2e_steps, "warmup": args.e2e_warmup,
+            "note": "weights + calibration activations from pinned host memory, pruned weights back to it"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="native", choices=["native", "reference"])
+    ap.add_argument("--config", default="llama7b")
+    ap.add_argument("--layers", type=int, default=0, help="layers per GPU (default: the model's)")
+    ap.add_argument("--tokens", type=int, default=0, help="calibration tokens (default: the config's)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=1)
+    ap.add_argument("--e2e-warmup", type=int, default=1)
+    ap.add_argument("--e2e-chunk", type=int, default=16384)
+    args = ap.parse_args()
+    cfg = wl.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_native(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

@@ -197,6 +197,15 @@ int mosaic_prune_structured_compact(const void *W_in, int64_t rows, int64_t cols
 int mosaic_rank_units(const float *scores, int64_t n_units, int64_t keep, int32_t *keep_out,
                       void *stream);
 
+/* ---------------------------------------------------------------------------
+ * mosaic_sum_unit_scores - dst[u] = fl32(dst[u] + src[u]) for u < n_units: adds
+ * the unit scores of a coupled projection to a running total before one
+ * ranking (same Fig. "composite" grouping; e.g. MLP channel c = row c of
+ * gate and up plus column c of down).  dst, src: device fp32, may not overlap
+ * partially.
+ * ------------------------------------------------------------------------- */
+int mosaic_sum_unit_scores(float *dst, const float *src, int64_t n_units, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,7 +32,7 @@ SYMBOLS = (
     "mosaic_allocate_sparsity",
     "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
     "mosaic_prune_structured_compact_workspace_bytes", "mosaic_prune_structured_compact",
-    "mosaic_rank_units",
+    "mosaic_rank_units", "mosaic_sum_unit_scores",
 )
 
 
@@ -83,6 +83,8 @@ def lib() -> C.CDLL:
                                                       vp, vp, sz, vp]
         L.mosaic_rank_units.restype = ci
         L.mosaic_rank_units.argtypes = [vp, i64, i64, vp, vp]
+        L.mosaic_sum_unit_scores.restype = ci
+        L.mosaic_sum_unit_scores.argtypes = [vp, vp, i64, vp]
         _lib = L
     return _lib
 
@@ -281,3 +283,13 @@ def mosaic_rank_units(scores: torch.Tensor, keep: int, keep_out: torch.Tensor, s
         raise ValueError("keep_out too short")
     _check(lib().mosaic_rank_units(scores.data_ptr(), scores.numel(), int(keep), keep_out.data_ptr(), _stream(stream)),
            "mosaic_rank_units")
+
+
+def mosaic_sum_unit_scores(dst: torch.Tensor, src: torch.Tensor, stream=None) -> None:
+    """dst[u] += src[u] in fp32: running total of the unit scores of coupled projections."""
+    _dev(dst, "dst", torch.float32)
+    _dev(src, "src", torch.float32)
+    if dst.numel() != src.numel() or not dst.is_contiguous() or not src.is_contiguous():
+        raise ValueError("dst and src must be contiguous and of equal length")
+    _check(lib().mosaic_sum_unit_scores(dst.data_ptr(), src.data_ptr(), dst.numel(), _stream(stream)),
+           "mosaic_sum_unit_scores")

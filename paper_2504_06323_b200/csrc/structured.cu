@@ -86,6 +86,11 @@ __global__ void unit_score_kernel(const double* __restrict__ row_sum, int64_t n_
     out[u] = accumulate ? __fadd_rn(out[u], f) : f;
 }
 
+__global__ void sum_scores_kernel(float* __restrict__ dst, const float* __restrict__ src, int64_t n) {
+    const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < n) dst[u] = __fadd_rn(dst[u], src[u]);
+}
+
 __device__ __forceinline__ uint32_t unit_key(float s) { return (s != s) ? 0xFFFFFFFFu : __float_as_uint(s); }
 
 // Keep list of one dimension: remove the (n - keep) units first under (score, index).
@@ -247,6 +252,17 @@ extern "C" int mosaic_rank_units(const float* scores, int64_t n_units, int64_t k
     if (keep == 0) return MOSAIC_OK;
     rank_kernel<<<1, kRankThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, n_units, keep, keep_out, nullptr, 0, 0,
                                                                           nullptr);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_sum_unit_scores(float* dst, const float* src, int64_t n_units, void* stream) {
+    if (!dst || !src) return MOSAIC_ERR_NULL_PTR;
+    if (n_units < 0) return MOSAIC_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dst) & 3u) || (reinterpret_cast<uintptr_t>(src) & 3u)) return MOSAIC_ERR_MISALIGNED;
+    if (dst != src && dst < src + n_units && src < dst + n_units) return MOSAIC_ERR_ALIASING;
+    if (n_units == 0) return MOSAIC_OK;
+    sum_scores_kernel<<<(unsigned)((n_units + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(dst, src, n_units);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }

@@ -1,0 +1,234 @@
+"""Runs the pruning hot path over a whole LLaMA-shaped model.
+
+Host-side orchestration only: it owns the device buffers (through torch),
+decides the order of the library calls, moves the <= N*M outlier counts to the
+host for the allocation, and - when several processes each own a share of the
+layers - exchanges those counts.  All arithmetic happens inside the library.
+
+Two phases separated by one tiny global dependency:
+  phase A (per projection, independent): activation norms, outlier counts;
+  host: every projection's count is needed before any target is known
+        (normalize(R_LLM) ranks each projection against all others);
+  phase B (per projection, independent): unstructured selection + zeroing,
+        and / or structured ranking + compaction.
+The phase-A result (counts) does not depend on the pruning target p, so one
+calibration serves any number of targets.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import torch
+
+from . import api
+from .workloads import PROJECTIONS, ModelConfig, gen_activation, gen_weight
+
+
+def layers_of_rank(n_layers: int, rank: int, world: int) -> list[int]:
+    """Round-robin ownership of whole layers (coupled structured units stay inside a layer)."""
+    return [l for l in range(n_layers) if l % world == rank]
+
+
+def exchange_counts(local_counts: torch.Tensor, n_layers: int, rank: int, world: int, group=None) -> list[int]:
+    """All ranks' outlier counts in global (layer, projection) order.
+
+    local_counts: int64 [len(layers_of_rank) * M], host or device.  With world == 1
+    this is only the device->host read.  Otherwise one all_gather of equal-sized int64
+    blocks (layers are padded to the largest share) - the only data-path exchange.
+    """
+    M = len(PROJECTIONS)
+    mine = layers_of_rank(n_layers, rank, world)
+    assert local_counts.numel() == len(mine) * M
+    if world == 1:
+        return [int(v) for v in local_counts.cpu().tolist()]
+    import torch.distributed as dist
+    share = (n_layers + world - 1) // world
+    block = torch.full((share * M,), -1, dtype=torch.int64, device=local_counts.device)
+    block[: local_counts.numel()] = local_counts
+    out = [torch.empty_like(block) for _ in range(world)]
+    dist.all_gather(out, block, group=group)
+    counts = [0] * (n_layers * M)
+    for r in range(world):
+        vals = out[r].cpu().tolist()
+        for i, layer in enumerate(layers_of_rank(n_layers, r, world)):
+            counts[layer * M:(layer + 1) * M] = [int(v) for v in vals[i * M:(i + 1) * M]]
+    return counts
+
+
+def plan_sparsity(cfg: ModelConfig, counts: list[int], p: float | None = None, lam: float | None = None,
+                  mode: int = api.GLOBAL_NORM, n_layers: int | None = None):
+    """normalize(R_LLM) + Projection Planner through the library's host call."""
+    n_layers = cfg.n_layers if n_layers is None else n_layers
+    numels, cols = [], []
+    for _ in range(n_layers):
+        for pr in PROJECTIONS:
+            r, c = cfg.shape(pr)
+            numels.append(r * c)
+            cols.append(c)
+    return api.mosaic_allocate_sparsity(counts, numels, cols, n_layers, len(PROJECTIONS),
+                                        cfg.p if p is None else p, cfg.lam if lam is None else lam, mode)
+
+
+@dataclass
+class ModelState:
+    cfg: ModelConfig
+    device: torch.device
+    layers: list[int]                                  # global ids of the layers this process owns
+    W: dict = field(default_factory=dict)              # (layer, proj) -> weights
+    W_out: dict = field(default_factory=dict)          # (layer, proj) -> pruned weights
+    mask: dict = field(default_factory=dict)           # (layer, proj) -> keep bitmask
+    sumsq: dict = field(default_factory=dict)          # (layer, x_key) -> fp64 accumulator
+    norms: dict = field(default_factory=dict)          # (layer, x_key) -> fp32 norms
+    counts: torch.Tensor | None = None                 # int64 [len(layers)*M]
+    ws: api.Workspace | None = None
+
+    def q_local(self, layer: int, proj: str) -> int:
+        return self.layers.index(layer) * len(PROJECTIONS) + PROJECTIONS.index(proj)
+
+
+def alloc_model(cfg: ModelConfig, device="cuda", layers: list[int] | None = None, outputs: bool = True,
+                masks: bool = True, generate: bool = True) -> ModelState:
+    """Allocate (and fill with the seeded synthetic weights) the buffers of the owned layers."""
+    device = torch.device(device)
+    st = ModelState(cfg, device, list(range(cfg.n_layers)) if layers is None else list(layers))
+    st.ws = api.Workspace(device)
+    st.counts = torch.zeros(len(st.layers) * len(PROJECTIONS), dtype=torch.int64, device=device)
+    for layer in st.layers:
+        for pr in PROJECTIONS:
+            rows, cols = cfg.shape(pr)
+            st.W[layer, pr] = gen_weight(cfg, layer, pr, device) if generate else \
+                torch.empty(rows, cols, dtype=cfg.torch_dtype, device=device)
+            if outputs:
+                st.W_out[layer, pr] = torch.empty(rows, cols, dtype=cfg.torch_dtype, device=device)
+            if masks:
+                st.mask[layer, pr] = torch.empty(rows, (cols + 31) // 32, dtype=torch.int32, device=device)
+        for xk in cfg.x_keys():
+            c = cfg.x_cols(xk)
+            st.sumsq[layer, xk] = torch.zeros(c, dtype=torch.float64, device=device)
+            st.norms[layer, xk] = torch.empty(c, dtype=torch.float32, device=device)
+    return st
+
+
+def make_activations(cfg: ModelConfig, layer: int, device="cuda", tokens: int | None = None) -> dict:
+    """One layer's calibration activations, one tensor per distinct projection input."""
+    return {xk: gen_activation(cfg, layer, xk, device, tokens) for xk in cfg.x_keys()}
+
+
+# ------------------------------------------------------------------ phase A
+def accumulate_norms(st: ModelState, layer: int, X: dict, first: bool = True, last: bool = True) -> int:
+    """Add one chunk of calibration tokens per input; `last` also finalises the fp32 norms.
+    Returns the number of library calls made."""
+    n = 0
+    for xk, x in X.items():
+        api.mosaic_act_norms(x, st.sumsq[layer, xk], st.norms[layer, xk] if last else None,
+                             api.RESET_ACCUM if first else 0, st.ws)
+        n += 1
+    return n
+
+
+def count_outliers(st: ModelState, layer: int, alpha: float | None = None) -> int:
+    cfg = st.cfg
+    a = cfg.alpha if alpha is None else alpha
+    for pr in PROJECTIONS:
+        q = st.q_local(layer, pr)
+        api.mosaic_outlier_ratio(st.W[layer, pr], st.norms[layer, cfg.x_key(pr)], a, st.counts[q:q + 1], None, st.ws)
+    return len(PROJECTIONS)
+
+
+# ------------------------------------------------------------------ phase B
+def prune_unstructured_layer(st: ModelState, layer: int, k_global: list[int], in_place: bool = False) -> int:
+    cfg = st.cfg
+    M = len(PROJECTIONS)
+    for m, pr in enumerate(PROJECTIONS):
+        W = st.W[layer, pr]
+        out = W if in_place else st.W_out[layer, pr]
+        api.mosaic_prune_unstructured(W, out, st.norms[layer, cfg.x_key(pr)], int(k_global[layer * M + m]),
+                                      st.mask.get((layer, pr)), st.ws)
+    return M
+
+
+def _scores(W, norms, row_group, col_group, out, accumulate, ws):
+    flags = api.SCORES_ONLY | (api.SCORES_ACCUM if accumulate else 0)
+    api.mosaic_prune_structured_compact(W, norms, row_group, col_group, 0, 0, None, None, flags, None, out, ws)
+
+
+def prune_structured_coupled_layer(st: ModelState, layer: int, frac: float, source: dict | None = None,
+                                   use_norms: bool = True) -> dict:
+    """Structured stage with the projections of a layer coupled the way the model's shapes require
+    (Fig. "composite": nodes between projections are pruned as a group):
+      * MLP channel c = row c of gate and up + column c of down, scored by the sum of the three;
+      * attention unit = one KV head with its query heads: rows of q (n_rep*head_dim), k and v
+        (head_dim), columns of o (n_rep*head_dim), scored by the sum of the four;
+      * the hidden (residual) dimension is never removed.
+    floor(frac * n_units) units are removed.  `source` gives the matrices to read (the masked
+    weights in composite mode); returns {"W": {proj: compacted}, "mlp_keep", "attn_keep"}.
+    """
+    cfg, dev, ws = st.cfg, st.device, st.ws
+    src = {pr: (source[pr] if source is not None else st.W[layer, pr]) for pr in PROJECTIONS}
+    nrm = {pr: (st.norms[layer, cfg.x_key(pr)] if use_norms else None) for pr in PROJECTIONS}
+    hd, n_kv = cfg.head_dim, cfg.n_kv_heads
+    n_rep = cfg.n_heads // n_kv
+    h, it = cfg.hidden, cfg.intermediate
+    out: dict = {"W": {}}
+
+    # MLP channels
+    s_gu = torch.empty(it + h, dtype=torch.float32, device=dev)       # row units first, then column units
+    s_d = torch.empty(h + it, dtype=torch.float32, device=dev)
+    _scores(src["gate"], nrm["gate"], 1, 1, s_gu, False, ws)
+    _scores(src["up"], nrm["up"], 1, 1, s_gu, True, ws)
+    _scores(src["down"], nrm["down"], 1, 1, s_d, False, ws)
+    total = s_gu[:it]                                                 # (gate + up) + down, fp32
+    api.mosaic_sum_unit_scores(total, s_d[h:])
+    keep_n = it - int(frac * it)
+    ch = torch.empty(keep_n, dtype=torch.int32, device=dev)
+    api.mosaic_rank_units(total, keep_n, ch)
+    all_h = torch.arange(h, dtype=torch.int32, device=dev)
+    given = api.ROWS_GIVEN | api.COLS_GIVEN
+    for pr in ("gate", "up"):
+        o = torch.empty(keep_n, h, dtype=cfg.torch_dtype, device=dev)
+        api.mosaic_prune_structured_compact(src[pr], None, 1, 1, keep_n, h, ch, all_h, given, o, None, ws)
+        out["W"][pr] = o
+    o = torch.empty(h, keep_n, dtype=cfg.torch_dtype, device=dev)
+    api.mosaic_prune_structured_compact(src["down"], None, 1, 1, h, keep_n, all_h, ch, given, o, None, ws)
+    out["W"]["down"] = o
+    out["mlp_keep"] = ch
+
+    # attention KV groups
+    gq = n_rep * hd
+    s_q = torch.empty(n_kv + h, dtype=torch.float32, device=dev)
+    s_k = torch.empty(n_kv + h, dtype=torch.float32, device=dev)
+    s_o = torch.empty(h + n_kv, dtype=torch.float32, device=dev)
+    _scores(src["q"], nrm["q"], gq, 1, s_q, False, ws)
+    _scores(src["k"], nrm["k"], hd, 1, s_k, False, ws)
+    _scores(src["v"], nrm["v"], hd, 1, s_k, True, ws)
+    _scores(src["o"], nrm["o"], 1, gq, s_o, False, ws)
+    tot_a = s_q[:n_kv]                                                # (q + (k + v)) + o, fp32
+    api.mosaic_sum_unit_scores(tot_a, s_k[:n_kv])
+    api.mosaic_sum_unit_scores(tot_a, s_o[h:])
+    keep_a = n_kv - int(frac * n_kv)
+    grp = torch.empty(keep_a, dtype=torch.int32, device=dev)
+    api.mosaic_rank_units(tot_a, keep_a, grp)
+    for pr, g in (("q", gq), ("k", hd), ("v", hd)):
+        o = torch.empty(keep_a * g, h, dtype=cfg.torch_dtype, device=dev)
+        api.mosaic_prune_structured_compact(src[pr], None, g, 1, keep_a, h, grp, all_h, given, o, None, ws)
+        out["W"][pr] = o
+    o = torch.empty(h, keep_a * gq, dtype=cfg.torch_dtype, device=dev)
+    api.mosaic_prune_structured_compact(src["o"], None, 1, gq, h, keep_a, all_h, grp, given, o, None, ws)
+    out["W"]["o"] = o
+    out["attn_keep"] = grp
+    return out
+
+
+def prune_structured_independent(st: ModelState, layer: int, proj: str, frac: float, use_norms: bool = True):
+    """Every projection on its own: remove floor(frac*rows) rows and floor(frac*cols) columns
+    (group 1) and write the dense compacted matrix.  Returns (W_compact, row_keep, col_keep)."""
+    cfg, dev = st.cfg, st.device
+    W = st.W[layer, proj]
+    rows, cols = W.shape
+    kr, kc = rows - int(frac * rows), cols - int(frac * cols)
+    rk = torch.empty(kr, dtype=torch.int32, device=dev)
+    ck = torch.empty(kc, dtype=torch.int32, device=dev)
+    out = torch.empty(kr, kc, dtype=cfg.torch_dtype, device=dev)
+    api.mosaic_prune_structured_compact(W, st.norms[layer, cfg.x_key(proj)] if use_norms else None, 1, 1, kr, kc, rk,
+                                        ck, 0, out, None, st.ws)
+    return out, rk, ck

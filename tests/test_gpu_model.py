@@ -1,0 +1,141 @@
+"""GPU parity of the whole path over a model, driver vs oracle pipeline: the five
+workload configurations (the tiny one at full size, the LLaMA-shaped ones scaled
+down so the oracle finishes in seconds but every row still spans several tiles
+and ragged tails)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import oracle_pipeline as op
+from paper_2504_06323_b200 import api, driver, workloads as wl
+from paper_2504_06323_b200.workloads import PROJECTIONS
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def bits_equal(a, b):
+    a, b = np.ascontiguousarray(a), np.ascontiguousarray(b)
+    return a.shape == b.shape and a.dtype == b.dtype and np.array_equal(a.view(np.uint8), b.view(np.uint8))
+
+
+def small(name, **kw):
+    base = wl.CONFIGS[name]
+    d = dict(n_layers=2, hidden=512, n_heads=8, n_kv_heads=8, head_dim=64, intermediate=1376, tokens=3000)
+    d.update(kw)
+    return wl.scaled(base, **d)
+
+
+def run_phase_a(cfg):
+    st = driver.alloc_model(cfg, DEV)
+    Wh, Xh = {}, {}
+    for layer in st.layers:
+        X = driver.make_activations(cfg, layer, DEV)
+        # two chunks through the accumulating call
+        cut = cfg.tokens // 3
+        driver.accumulate_norms(st, layer, {k: v[:cut] for k, v in X.items()}, first=True, last=False)
+        driver.accumulate_norms(st, layer, {k: v[cut:] for k, v in X.items()}, first=False, last=True)
+        driver.count_outliers(st, layer)
+        for xk, x in X.items():
+            Xh[layer, xk] = wl.to_numpy(x)
+        for pr in PROJECTIONS:
+            Wh[layer, pr] = wl.to_numpy(st.W[layer, pr])
+    counts = driver.exchange_counts(st.counts, cfg.n_layers, 0, 1)
+    norms_ref, counts_ref = op.phase_a(cfg, Wh, Xh, st.layers)
+    for key, n in st.norms.items():
+        ok = oracle.norm_certify(Xh[key], cfg.dtype)
+        got = n.cpu().numpy()
+        np.testing.assert_allclose(got, norms_ref[key], rtol=1e-5)
+        assert ok.all(), "re-seed: a column sits on an fp32 rounding boundary"
+        assert bits_equal(got, norms_ref[key])
+    assert counts == counts_ref
+    return st, Wh, Xh, norms_ref, counts
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", None), ("llama7b", {}), ("llama2_13b", dict(hidden=640, n_heads=10, n_kv_heads=10,
+                                                                                        intermediate=1728))])
+def test_unstructured_model(name, kw):
+    cfg = wl.CONFIGS[name] if kw is None else small(name, **kw)
+    st, Wh, Xh, norms_ref, counts = run_phase_a(cfg)
+    sweep = cfg.extra.get("p_sweep", (cfg.p,))
+    prev = {}
+    for p in sweep:
+        s, k, infeasible = driver.plan_sparsity(cfg, counts, p=p)
+        s_ref, k_ref, inf_ref = op.plan(cfg, counts, cfg.n_layers, p=p)
+        assert np.array_equal(np.array(s).view(np.uint64), s_ref.view(np.uint64)) and list(k) == list(k_ref)
+        assert infeasible == inf_ref
+        assert abs(np.mean(s) - p) < 1e-12                      # targets average to p
+        assert len(set(k)) > 1                                  # allocation is non-uniform
+        for layer in st.layers:
+            driver.prune_unstructured_layer(st, layer, k)
+            ref = op.unstructured(cfg, Wh, norms_ref, layer, k_ref)
+            for pr in PROJECTIONS:
+                assert bits_equal(wl.to_numpy(st.W_out[layer, pr]), ref[pr][0]), (layer, pr)
+                m = st.mask[layer, pr].cpu().numpy().view(np.uint32)
+                assert bits_equal(m, ref[pr][1]), (layer, pr)
+                if (layer, pr) in prev:
+                    assert ((m & ~prev[layer, pr]) == 0).all()  # masks nested across the sweep
+                prev[layer, pr] = m
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", None), ("llama3_8b", dict(hidden=640, n_heads=10, n_kv_heads=5, head_dim=64, intermediate=1728))])
+def test_composite_model(name, kw):
+    cfg = wl.CONFIGS[name] if kw is None else small(name, **kw)
+    frac = cfg.extra.get("structured_frac", 0.2)
+    st, Wh, Xh, norms_ref, counts = run_phase_a(cfg)
+    _, k, _ = driver.plan_sparsity(cfg, counts)
+    for layer in st.layers:
+        driver.prune_unstructured_layer(st, layer, k)
+        masked = {pr: st.W_out[layer, pr] for pr in PROJECTIONS}
+        got = driver.prune_structured_coupled_layer(st, layer, frac, source=masked)
+        ref_u = op.unstructured(cfg, Wh, norms_ref, layer, k)
+        ref = op.structured_coupled(cfg, {pr: ref_u[pr][0] for pr in PROJECTIONS}, norms_ref, layer, frac)
+        assert bits_equal(got["mlp_keep"].cpu().numpy(), ref["mlp_keep"])
+        assert bits_equal(got["attn_keep"].cpu().numpy(), ref["attn_keep"])
+        assert len(ref["mlp_keep"]) == cfg.intermediate - int(frac * cfg.intermediate)
+        for pr in PROJECTIONS:
+            assert bits_equal(wl.to_numpy(got["W"][pr]), ref["W"][pr]), (layer, pr)
+
+
+@pytest.mark.parametrize("frac", [0.1, 0.3, 0.5])
+def test_structured_independent_model(frac):
+    cfg = small("llama7b_structured", n_layers=1)
+    st, Wh, Xh, norms_ref, counts = run_phase_a(cfg)
+    for pr in PROJECTIONS:
+        out, rk, ck = driver.prune_structured_independent(st, 0, pr, frac)
+        ref, rk_ref, ck_ref = op.structured_independent(cfg, Wh[0, pr], norms_ref[0, cfg.x_key(pr)], frac)
+        assert bits_equal(rk.cpu().numpy(), rk_ref) and bits_equal(ck.cpu().numpy(), ck_ref)
+        rows, cols = cfg.shape(pr)
+        assert tuple(out.shape) == (rows - int(frac * rows), cols - int(frac * cols))
+        assert bits_equal(wl.to_numpy(out), ref)
+
+
+def test_full_size_rows_sampled_against_oracle():
+    # the headline launch configuration: full LLaMA-7B projection shapes, checked on sampled rows
+    cfg = wl.CONFIGS["llama7b"]
+    for pr in ("q", "gate", "down"):
+        rows, cols = cfg.shape(pr)
+        W = wl.gen_weight(cfg, 0, pr, DEV)
+        g = torch.Generator(device="cpu").manual_seed(rows + cols)
+        norms = (torch.rand(cols, generator=g) * 500 + 100).to(DEV)
+        norms[wl.outlier_columns(cfg, 0, cfg.x_key(pr), cols, cfg.x_outlier_frac).to(DEV)] *= 100
+        out = torch.empty_like(W)
+        mask = torch.empty(rows, (cols + 31) // 32, dtype=torch.int32, device=DEV)
+        k = cols // 2
+        api.mosaic_prune_unstructured(W, out, norms, k, mask)
+        cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+        ssum = torch.zeros(1, dtype=torch.float64, device=DEV)
+        api.mosaic_outlier_ratio(W, norms, cfg.alpha, cnt, ssum)
+        sample = torch.randperm(rows, generator=g)[:48].sort().values
+        Ws, nh = wl.to_numpy(W[sample.to(DEV)]), norms.cpu().numpy()
+        ref_W, ref_mask = oracle.prune_unstructured(Ws, nh, k, "bf16")
+        assert bits_equal(wl.to_numpy(out[sample.to(DEV)]), ref_W)
+        assert bits_equal(mask[sample.to(DEV)].cpu().numpy().view(np.uint32), ref_mask)
+        # properties that hold at any size
+        kept = mask.cpu().numpy().view(np.uint8)
+        assert (np.unpackbits(kept, axis=1).sum(1) == cols - k).all()
+        assert int((out == 0).sum().item()) >= rows * k
+        ref = oracle.outlier_ratio(wl.to_numpy(W), nh, cfg.alpha, "bf16")     # whole matrix: a second or two
+        assert ref["certified"] and cnt.item() == ref["count"]
+        np.testing.assert_allclose(ssum.item(), ref["sum"], rtol=1e-12)
