@@ -94,7 +94,7 @@ int mosaic_act_norms(const void *X, int64_t tokens, int64_t cols, int64_t ldx, i
                      void *stream);
 
 /* ---------------------------------------------------------------------------
- * mosaic_score - Eq. 5 / Algorithm 1 line 11, materialised:
+ * mosaic_score - Eq. 5 / the weight-metric step of Algorithm 1, materialised:
  *     score_out[i, j] = fl32( norms[j] * |W[i, j]| )      (one fp32 multiply)
  * For tests and small use; the pruning calls recompute scores on the fly.
  *   W          device, [rows, cols], ld ldw, dtype; read only
@@ -105,13 +105,13 @@ int mosaic_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dty
                  const float *norms, float *score_out, void *stream);
 
 /* ---------------------------------------------------------------------------
- * mosaic_outlier_ratio - Eq. 6 / Algorithm 1 lines 13-14 for one projection:
+ * mosaic_outlier_ratio - Eq. 6 / the outlier-count step of Algorithm 1 for one projection:
  *     S = sum_ij (double) w_ij,  tau = (double)alpha * S / (rows*cols),
  *     O = #{ (i,j) : (double) w_ij > tau }                  (strict)
  *   outlier_count_out  device, 1 x int64
  *   score_sum_out      device, 1 x fp64, or NULL
  *   ws                 device scratch, >= mosaic_outlier_ratio_workspace_bytes()
- * The rank R = 100*O/C (Algorithm 1 line 15) is formed on the host:
+ * The rank R = 100*O/C (the projection-rank step of Algorithm 1) is formed on the host:
  * mosaic_ratio_from_count.
  * ------------------------------------------------------------------------- */
 size_t mosaic_outlier_ratio_workspace_bytes(int64_t rows, int64_t cols);
@@ -121,7 +121,7 @@ int mosaic_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw,
 double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
 
 /* ---------------------------------------------------------------------------
- * mosaic_allocate_sparsity - normalize(R_LLM) (Algorithm 1 line 19) and the
+ * mosaic_allocate_sparsity - normalize(R_LLM) (the return of Algorithm 1) and the
  * Projection Planner (Section 3.3 component 8; Eq. 1-2).  HOST function, all
  * pointers are host memory, q = n*n_proj + m.
  * The paper states only the properties (targets average to p; more outliers

@@ -112,7 +112,7 @@ def score(W: np.ndarray, norms: np.ndarray, dtype=None) -> np.ndarray:
 
 
 def outlier_ratio(W: np.ndarray, norms: np.ndarray, alpha: float = 5.0, dtype=None) -> dict:
-    """Eq. 6 / Alg. 1 lines 13-15: outlier count O, fp64 score sum, R = 100*O/C."""
+    """Eq. 6 / Algorithm 1's count and rank steps: outlier count O, fp64 score sum, R = 100*O/C."""
     code = _code(W, dtype)
     rows, cols = W.shape
     norms = np.ascontiguousarray(norms, np.float32)

@@ -16,13 +16,13 @@
  *   W      one projection's weights, row-major [rows = out, cols = in]
  *   X      calibration activations feeding that projection, row-major [T, cols]
  *   norm_j l2 norm of column j of X                         (the ||A||_2 of Eq. 5)
- *   w_ij   = norm_j * |W_ij|                                (Eq. 5, Alg. 1 line 11)
- *   C      = rows*cols                                      (Alg. 1 line 13)
- *   O      = #{ w_ij > alpha * mean(w) }                    (Eq. 6, Alg. 1 line 14)
- *   R      = 100 * O / C                                    (Alg. 1 line 15)
+ *   w_ij   = norm_j * |W_ij|                                (Eq. 5, Algorithm 1)
+ *   C      = rows*cols                                      (Algorithm 1)
+ *   O      = #{ w_ij > alpha * mean(w) }                    (Eq. 6, Algorithm 1)
+ *   R      = 100 * O / C                                    (Algorithm 1)
  *
  * Parity with the authors' own program is unpinned: the paper prints no
- * worked numeric example and leaves normalize(R_LLM) (Alg. 1 line 19)
+ * worked numeric example and leaves normalize(R_LLM) (Algorithm 1's return)
  * undefined; oracle_allocate_sparsity states the reading taken.  Everything
  * else here is pinned by the CPU tests against brute force in exact rational
  * arithmetic, closed forms and invariants.
@@ -142,7 +142,7 @@ int64_t oracle_norm_certify(const void *X, int64_t tokens, int64_t cols, int64_t
 }
 
 /* ------------------------------------------------------------------ */
-/* Weight metric, Eq. 5 / Alg. 1 line 11, materialised.                */
+/* Weight metric, Eq. 5 / Algorithm 1, materialised.                    */
 /* ------------------------------------------------------------------ */
 void oracle_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
                   const float *norms, float *score /* [rows, cols] */)
@@ -154,7 +154,7 @@ void oracle_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dt
 }
 
 /* ------------------------------------------------------------------ */
-/* Projection outlier statistic, Eq. 6 / Alg. 1 lines 13-15.           */
+/* Projection outlier statistic, Eq. 6 / Algorithm 1.                  */
 /* ------------------------------------------------------------------ */
 /*
  * sum   = sum_i sum_j (double) w_ij          (row-major order, fp64)
@@ -194,7 +194,7 @@ void oracle_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw
 }
 
 /* ------------------------------------------------------------------ */
-/* normalize(R_LLM) + Projection Planner (Alg. 1 line 19; Section 3.3  */
+/* normalize(R_LLM) + Projection Planner (Algorithm 1; Section 3.3      */
 /* component 8; Eq. 1-2).                                              */
 /* ------------------------------------------------------------------ */
 /*

@@ -56,7 +56,7 @@ const char* mosaic_status_string(int status) {
 }
 
 double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel) {
-    // Algorithm 1 line 15: R = O / C * 100
+    // projection rank of Algorithm 1: R = O / C * 100
     return 100.0 * (double)outlier_count / (double)numel;
 }
 

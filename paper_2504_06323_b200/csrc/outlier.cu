@@ -1,5 +1,5 @@
 // mosaic_score (Eq. 5 materialised) and mosaic_outlier_ratio (Eq. 6 /
-// Algorithm 1 lines 13-14): fp64 sum of the weight metric over a projection,
+// the outlier-count step of Algorithm 1): fp64 sum of the weight metric over a projection,
 // threshold tau = alpha * mean, strict outlier count.
 //
 // Decomposition of both sweeps: a CTA of 128 threads owns a chunk of 1024
