@@ -222,6 +222,52 @@ def test_prune_writes_only_its_outputs():
     assert (mbuf[0] == 0x5A5A5A5A).all() and (mbuf[-1] == 0x5A5A5A5A).all()
 
 
+def _check_prune(W, norms, k, dtype):
+    out, mask = run_prune(W, norms, k)
+    ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, dtype)
+    assert_bits_equal(host(out), ref_W)
+    assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("rows,cols", [(2500, 4096), (1300, 5120), (700, 11008), (640, 14336)])
+def test_prune_many_rows_per_cta(dtype, rows, cols):
+    # more rows than resident CTAs: every CTA carries its threshold estimate from row to row
+    W = make(rows, cols, dtype, seed=rows + cols, heavy=False)
+    norms = norms_for(cols, 31)
+    for k in (cols // 2, cols // 10):
+        _check_prune(W, norms, k, dtype)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_prune_rows_of_very_different_scale(dtype):
+    # consecutive rows of a CTA differ by orders of magnitude, some are constant, some all zero,
+    # some half zero: the carried estimate is useless and every fallback of the selection runs
+    rows, cols = 3000, 4096
+    W = make(rows, cols, dtype, seed=77, heavy=True).clone()
+    g = torch.Generator(device="cpu").manual_seed(78)
+    scale = torch.exp2(torch.randint(-20, 21, (rows, 1), generator=g).float()).to(DEV)
+    W = (W.float() * scale).to(W.dtype)
+    W[5::97] = 0.0
+    W[7::89] = 0.125
+    W[11::83, ::2] = 0.0
+    W[13::79, 100:] = -3.0
+    norms = norms_for(cols, 32)
+    for k in (1, 1500, 2048, 4000, 4096):
+        _check_prune(W, norms, k, dtype)
+
+
+def test_prune_already_pruned_matrix():
+    # half of every row is exactly zero (a matrix pruned before): thousands of tied keys at +0
+    rows, cols = 1200, 4096
+    W = make(rows, cols, "bf16", seed=91)
+    norms = norms_for(cols, 33)
+    half, _ = run_prune(W, norms, 2048)
+    half = half.contiguous()
+    for k in (100, 2047, 2048, 2049, 3000):
+        _check_prune(half, norms, k, "bf16")
+
+
 # ------------------------------------------------------------------ structured
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("rows,cols,rg,cg,fr,fc", [(256, 688, 1, 1, 0.3, 0.3), (512, 1024, 64, 1, 0.25, 0.5),
