@@ -121,6 +121,41 @@ int mosaic_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw,
 double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
 
 /* ---------------------------------------------------------------------------
+ * mosaic_outlier_ratio_static - mosaic_outlier_ratio without a workspace
+ * argument.  (The paper has no counterpart: this is a packaging variant of the
+ * call above, not another operation.)
+ * Who it is for: code that may not allocate device memory when it calls in -
+ * a plug-in running inside a host application that owns the allocator, a
+ * callback on a latency-critical path where cudaMalloc's implicit
+ * synchronisation is not acceptable, a process whose memory pool is already
+ * committed.  Such a caller has nowhere to take the scratch buffer from, so
+ * the library carries one itself: a fixed array of
+ * MOSAIC_OUTLIER_STATIC_SCRATCH_BYTES in device memory, present on every GPU
+ * that loads the library for as long as the process lives.  The call
+ * allocates and frees nothing.
+ *   - Inputs and outputs are the caller's, exactly as for mosaic_outlier_ratio,
+ *     and the results are bit-identical to it.
+ *   - A matrix whose scratch need (mosaic_outlier_ratio_workspace_bytes)
+ *     exceeds the built-in array is refused with
+ *     MOSAIC_ERR_WORKSPACE_TOO_SMALL before anything is enqueued; use the
+ *     regular call with your own buffer then.
+ *   - The first call on each device looks up the array's device address (a
+ *     host-side runtime query, with that device current).  Make that first
+ *     call during start-up, outside any stream capture.
+ *   - All calls on one device share the one array.  The part that has to
+ *     start from zero is cleared on the stream at the start of every call, so
+ *     back-to-back calls on one stream are fine; two calls that can overlap
+ *     on the GPU (different streams, different host threads) race on it and
+ *     give wrong counts.  Serialise them, or give the overlapping ones their
+ *     own workspace through mosaic_outlier_ratio.
+ * ------------------------------------------------------------------------- */
+#define MOSAIC_OUTLIER_STATIC_SCRATCH_BYTES 65536
+size_t mosaic_outlier_ratio_static_max_workspace_bytes(void);
+int mosaic_outlier_ratio_static(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                                const float *norms, float alpha, int64_t *outlier_count_out,
+                                double *score_sum_out, void *stream);
+
+/* ---------------------------------------------------------------------------
  * mosaic_allocate_sparsity - normalize(R_LLM) (the return of Algorithm 1) and the
  * Projection Planner (Section 3.3 component 8; Eq. 1-2).  HOST function, all
  * pointers are host memory, q = n*n_proj + m.

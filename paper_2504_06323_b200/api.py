@@ -29,6 +29,7 @@ SYMBOLS = (
     "mosaic_act_norms_workspace_bytes", "mosaic_act_norms",
     "mosaic_score",
     "mosaic_outlier_ratio_workspace_bytes", "mosaic_outlier_ratio", "mosaic_ratio_from_count",
+    "mosaic_outlier_ratio_static_max_workspace_bytes", "mosaic_outlier_ratio_static",
     "mosaic_allocate_sparsity",
     "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
     "mosaic_prune_structured_compact_workspace_bytes", "mosaic_prune_structured_compact",
@@ -68,6 +69,10 @@ def lib() -> C.CDLL:
         L.mosaic_outlier_ratio_workspace_bytes.argtypes = [i64, i64]
         L.mosaic_outlier_ratio.restype = ci
         L.mosaic_outlier_ratio.argtypes = [vp, i64, i64, i64, ci, vp, flt, vp, vp, vp, sz, vp]
+        L.mosaic_outlier_ratio_static_max_workspace_bytes.restype = sz
+        L.mosaic_outlier_ratio_static_max_workspace_bytes.argtypes = []
+        L.mosaic_outlier_ratio_static.restype = ci
+        L.mosaic_outlier_ratio_static.argtypes = [vp, i64, i64, i64, ci, vp, flt, vp, vp, vp]
         L.mosaic_ratio_from_count.restype = dbl
         L.mosaic_ratio_from_count.argtypes = [i64, i64]
         L.mosaic_allocate_sparsity.restype = ci
@@ -207,6 +212,23 @@ def mosaic_outlier_ratio(W: torch.Tensor, norms: torch.Tensor, alpha: float, out
     _check(L.mosaic_outlier_ratio(p, rows, cols, ldw, _dtype_code(W), norms.data_ptr(), float(alpha),
                                   outlier_count_out.data_ptr(), _ptr(score_sum_out), wp, wn, _stream(stream)),
            "mosaic_outlier_ratio")
+
+
+def mosaic_outlier_ratio_static(W: torch.Tensor, norms: torch.Tensor, alpha: float, outlier_count_out: torch.Tensor,
+                                score_sum_out: torch.Tensor | None = None, stream=None) -> None:
+    """mosaic_outlier_ratio for callers that cannot allocate device memory: no workspace is
+    passed, the library uses the fixed scratch array it carries on the device.  Calls on one
+    device share that array, so do not let two of them overlap on the GPU."""
+    p, rows, cols, ldw = _mat(W, "W")
+    _dev(norms, "norms", torch.float32)
+    _dev(outlier_count_out, "outlier_count_out", torch.int64)
+    if score_sum_out is not None:
+        _dev(score_sum_out, "score_sum_out", torch.float64)
+    if norms.numel() != cols:
+        raise ValueError("norms must be [cols]")
+    _check(lib().mosaic_outlier_ratio_static(p, rows, cols, ldw, _dtype_code(W), norms.data_ptr(), float(alpha),
+                                             outlier_count_out.data_ptr(), _ptr(score_sum_out), _stream(stream)),
+           "mosaic_outlier_ratio_static")
 
 
 def mosaic_ratio_from_count(outlier_count: int, numel: int) -> float:

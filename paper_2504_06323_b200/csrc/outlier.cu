@@ -239,3 +239,57 @@ extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, i
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// mosaic_outlier_ratio_static: the same computation with the scratch memory built into the
+// library, for callers that have no device allocator to take a workspace from.
+// ------------------------------------------------------------------------------------------
+namespace mosaic {
+
+// Scratch of mosaic_outlier_ratio_static.  Every device that loads the library carries these
+// 64 KiB until the process exits.  It holds the sweep counter, the threshold and one fp64
+// partial sum per CTA of the first sweep (a few thousand at most on current parts).
+constexpr size_t kStaticScratchBytes = MOSAIC_OUTLIER_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_outlier_scratch[kStaticScratchBytes];
+
+// Device address of g_outlier_scratch on the current device.  In host code the array's name is
+// only a handle for the runtime, not something a kernel can dereference, so the address is asked
+// for once per device (with that device current) and remembered.
+static int static_scratch_address(void** out) {
+    static void* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_ERR_CUDA;
+    if (dev >= 0 && dev < 64 && cached[dev] != nullptr) {
+        *out = cached[dev];
+        return MOSAIC_OK;
+    }
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_outlier_scratch) != cudaSuccess || p == nullptr) {
+        (void)cudaGetLastError();
+        return MOSAIC_ERR_CUDA;
+    }
+    if (dev >= 0 && dev < 64) cached[dev] = p;
+    *out = p;
+    return MOSAIC_OK;
+}
+
+}  // namespace mosaic
+
+extern "C" size_t mosaic_outlier_ratio_static_max_workspace_bytes(void) { return mosaic::kStaticScratchBytes; }
+
+extern "C" int mosaic_outlier_ratio_static(const void* W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                                           const float* norms, float alpha, int64_t* outlier_count_out,
+                                           double* score_sum_out, void* stream) {
+    // argument errors first, so that a bad call costs no CUDA work
+    int rc = check_matrix(W, rows, cols, ldw, dtype);
+    if (rc != MOSAIC_OK) return rc;
+    if (rows == 0) return MOSAIC_ERR_INVALID_ARG;
+    if (mosaic_outlier_ratio_workspace_bytes(rows, cols) > kStaticScratchBytes) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+    void* scratch = nullptr;
+    rc = static_scratch_address(&scratch);
+    if (rc != MOSAIC_OK) return rc;
+    // The regular entry point clears the part of the scratch that must start at zero (the sweep
+    // counter) on the stream before the first kernel, so what an earlier call left behind is harmless.
+    return mosaic_outlier_ratio(W, rows, cols, ldw, dtype, norms, alpha, outlier_count_out, score_sum_out, scratch,
+                                kStaticScratchBytes, stream);
+}

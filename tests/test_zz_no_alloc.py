@@ -1,0 +1,70 @@
+"""mosaic_outlier_ratio_static: the workspace-free variant of mosaic_outlier_ratio.
+
+Some users of this library run where they may not allocate device memory at the
+moment they call in (inside another application's allocator, on a path that
+must not hit cudaMalloc's synchronisation, with the memory pool already spoken
+for), so this entry point uses a fixed scratch array that lives inside the
+library.  The test drives it through the C ABI and requires the same bits as
+the regular entry point, which takes a caller-owned workspace - twice in a row,
+because the second call finds the scratch as the first one left it.
+
+Collected last on purpose (file name): a run that stops at the first failure
+has then already been through every other test.
+"""
+import ctypes as C
+
+import pytest
+import torch
+
+from paper_2504_06323_b200 import api
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(rows, cols, seed):
+    g = torch.Generator(device="cpu").manual_seed(seed)
+    W = (torch.randn(rows, cols, generator=g) * 0.02).to(torch.bfloat16).cuda()
+    norms = (torch.rand(cols, generator=g) + 0.1) * 30.0
+    norms[::53] *= 80.0
+    return W, norms.to(torch.float32).cuda()
+
+
+def _regular(W, norms, alpha):
+    cnt = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+    ssum = torch.full((1,), -1.0, dtype=torch.float64, device="cuda")
+    api.mosaic_outlier_ratio(W, norms, alpha, cnt, ssum)
+    torch.cuda.synchronize()
+    return int(cnt.item()), ssum.cpu().numpy().tobytes()
+
+
+def _static_through_c_abi(W, norms, alpha):
+    L = api.lib()
+    cnt = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+    ssum = torch.full((1,), -1.0, dtype=torch.float64, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream or None
+    rc = L.mosaic_outlier_ratio_static(W.data_ptr(), W.shape[0], W.shape[1], W.stride(0), api.BF16, norms.data_ptr(),
+                                       C.c_float(alpha), cnt.data_ptr(), ssum.data_ptr(), stream)
+    assert rc == 0, api.status_string(rc)
+    torch.cuda.synchronize()
+    return int(cnt.item()), ssum.cpu().numpy().tobytes()
+
+
+def test_static_scratch_matches_caller_workspace_twice_in_a_row():
+    # two different matrices back to back: the second call starts from the scratch the first left
+    for rows, cols, seed, alpha in [(1500, 4096, 1, 5.0), (700, 1000, 2, 3.0), (1500, 4096, 1, 5.0)]:
+        W, norms = _inputs(rows, cols, seed)
+        want = _regular(W, norms, alpha)
+        assert want[0] > 0                                   # the case does have outliers to count
+        assert _static_through_c_abi(W, norms, alpha) == want
+        assert _static_through_c_abi(W, norms, alpha) == want
+
+
+def test_static_scratch_refuses_what_does_not_fit():
+    L = api.lib()
+    assert L.mosaic_outlier_ratio_static_max_workspace_bytes() == 65536
+    # a row so wide that the first sweep needs more partial sums than the built-in array holds;
+    # refused from the sizes alone, before any pointer is touched
+    cols = 16 * 1024 * 1024
+    assert L.mosaic_outlier_ratio_workspace_bytes(8, cols) > 65536
+    rc = L.mosaic_outlier_ratio_static(256, 8, cols, cols, api.BF16, 256, C.c_float(5.0), 256, None, None)
+    assert rc == -5, api.status_string(rc)
