@@ -4,37 +4,41 @@
 // projection pruning; weight metric of Eq. 5).
 //
 // One CTA works on one row at a time and walks rows blockIdx.x, +gridDim.x, ...
-// Thread t owns the vectors v*NT + t (8 adjacent columns each), so the norms of
-// its columns live in registers for the whole kernel and the row is read from
-// HBM exactly once: the raw weights stay in registers across the selection, and
-// the next row of the CTA is already in flight (a second register set) while
-// the current one is selected.  Scores are >= +0, so the fp32 bit pattern is an
-// order preserving unsigned key.
+// Thread t owns the vectors v*nt + t (8 adjacent columns each).  A row is read
+// from HBM exactly once and the next row of the CTA is already in flight while
+// the current one is selected.  Scores are >= +0, so the fp32 bit pattern of a
+// score is an order preserving unsigned key.  The result of the selection is
+// the exact k-th smallest key T of the row plus the tie quota q (how many
+// entries equal to T are pruned, lowest column first).
 //
-// The result is the exact k-th smallest key T of the row plus the tie quota q
-// (how many entries equal to T are pruned, lowest column first).  Three ways to
-// get there, all exact, tried in order of cost:
+// Rows of one projection share the norms and k, so their thresholds are close.
+// Every kernel here therefore first tries a *window* [lo, lo + 2^w) of key
+// space that should contain T: it counts the keys below lo, builds a histogram
+// of the few keys inside, and only those take part in the selection.  A window
+// comes from the previous rows of the CTA or, without one or after a miss,
+// from the matching quantile of one key per thread.  The full radix select over
+// all keys (digits of 11, 10 and 10 bits) remains as the exact fallback; all
+// paths give the same bits.
 //
-//   1. tracked window.  Rows of one projection share the norms and k, so their
-//      thresholds are close.  With a running estimate c of T the CTA counts the
-//      keys below lo = c - 2^20 and collects the keys inside [lo, lo + 2^21) in
-//      a shared-memory list (a few percent of the row).  If the k-th key lies in
-//      the window, one warp finishes the selection on the list alone with an
-//      8-bit-digit radix select.
-//   2. sampled window.  Without an estimate (first row of a CTA) or after a
-//      miss, the CTA selects the matching quantile of one key per thread and
-//      opens a 2^23 window around it.
-//   3. full radix select over all keys with shared-memory histograms: digits of
-//      11, 10 and 10 bits (bits 30..20, 19..10, 9..0; bit 31 is 0 for every
-//      valid key).  Always succeeds.
-//
-// If q is all of the ties the row is finished with a plain compare; otherwise a
-// block-wide ordered prefix count over the columns prunes the q lowest-indexed
-// ties.
-#include "common.cuh"
+// Two kernels:
+//   prune_rows_bf16_kernel  bf16 rows of 2048..16384 columns.  For a fixed
+//       window the test "score key below lo" is, per column j, a test of the
+//       weight's 15 magnitude bits against a bf16 bit pattern A_lo[j], because
+//       the score norm_j*|w| is monotone in |w|.  The thresholds of the thread's
+//       columns live in registers (two 16-bit lanes per word), and a row is
+//       classified two weights per integer subtract, without ever forming the
+//       scores.  The thresholds are conservative (computed with an approximate
+//       reciprocal and widened by two bf16 steps); the weights that fall
+//       between A_lo[j] and A_hi[j] - a few percent of the row - are the
+//       candidates, and only they get an exact fp32 score.
+//   prune_rows_kernel       any dtype, any shape; scores of all entries in fp32.
+#include "select.cuh"
 
 #ifndef MOSAIC_PRUNE_MINB_2X256
-#define MOSAIC_PRUNE_MINB_2X256 4
+#define MOSAIC_PRUNE_MINB_2X256 3
+#endif
+#ifndef MOSAIC_FAST_MAX_CTAS
+#define MOSAIC_FAST_MAX_CTAS 8
 #endif
 
 namespace mosaic {
@@ -48,147 +52,13 @@ __device__ unsigned long long g_prune_stats[8];
 #define MOSAIC_STAT_ADD(i, n) do { } while (0)
 #endif
 
-constexpr int kBins1 = 2048;      // first digit of the full select: bits 30..20
-constexpr int kBins23 = 1024;     // second / third digit
 constexpr int kListCap = kBins1;  // candidate list shares the histogram's storage
-constexpr int kTrackBits = 21;    // width (log2, in key units) of the tracked window
+constexpr int kTrackBits = 21;    // width (log2, in key units) of a window carried from row to row
 constexpr int kSampleBits = 23;   // width of the window around a sampled quantile
-
-struct SelectResult {
-    uint32_t bin, rank, count;
-};
 
 struct RowSelect {   // hand-over between warp 0 and the CTA during a window attempt
     uint32_t ok, T, q, n_eq, lo, bin;
 };
-
-// Block-wide: find the bin b with  cum(b-1) < rank <= cum(b)  in hist[0..NB), clear the
-// histogram for the next pass, and return (b, rank - cum(b-1), hist[b]).
-template <int NT, int NB>
-__device__ __forceinline__ SelectResult find_bin(uint32_t* hist, uint32_t* warp_tot, SelectResult* sel, uint32_t rank) {
-    constexpr int BPT = (NB + NT - 1) / NT;
-    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    uint32_t local[BPT];
-    uint32_t sum = 0;
-#pragma unroll
-    for (int i = 0; i < BPT; ++i) {
-        const int b = tid * BPT + i;
-        local[i] = (b < NB) ? hist[b] : 0u;
-        if (b < NB) hist[b] = 0u;
-        sum += local[i];
-    }
-    uint32_t incl = sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += n;
-    }
-    if (lane == 31) warp_tot[wid] = incl;
-    __syncthreads();
-    uint32_t base = incl - sum;
-    for (int w = 0; w < wid; ++w) base += warp_tot[w];
-    if (base < rank && rank <= base + sum) {
-#pragma unroll
-        for (int i = 0; i < BPT; ++i) {
-            if (rank <= base + local[i]) {
-                sel->bin = (uint32_t)(tid * BPT + i);
-                sel->rank = rank - base;
-                sel->count = local[i];
-                break;
-            }
-            base += local[i];
-        }
-    }
-    __syncthreads();
-    return *sel;
-}
-
-// Block-wide exclusive prefix of a per-thread count, in thread order.  Returns the
-// exclusive prefix; *total receives the block total.
-template <int NT>
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t* warp_tot, uint32_t* total) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    uint32_t incl = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += n;
-    }
-    __syncthreads();
-    if (lane == 31) warp_tot[wid] = incl;
-    __syncthreads();
-    uint32_t base = incl - v, tot = 0;
-    for (int w = 0; w < NT / 32; ++w) {
-        const uint32_t t = warp_tot[w];
-        if (w < wid) base += t;
-        tot += t;
-    }
-    *total = tot;
-    return base;
-}
-
-// One warp: the r-th smallest (1 <= r <= L) of list[0..L), whose entries all lie in
-// [lo, lo + 2^w).  Radix select on d = key - lo with 8-bit digits from the top and a
-// 256-bin histogram private to the warp.  Returns false if no bin holds the rank (a
-// caller error, or keys outside the window); then nothing is written.
-__device__ __forceinline__ bool warp_select(const uint32_t* list, uint32_t L, uint32_t lo, int w, uint32_t r,
-                                            uint32_t* whist, uint32_t* T, uint32_t* q, uint32_t* n_eq) {
-    const int lane = threadIdx.x & 31;
-    uint32_t prefix = 0u, cnt = 0u;
-    int top = w;   // low bits of d still undetermined
-    while (top > 0) {
-        const int nb = top >= 8 ? 8 : top;
-        const int s = top - nb;
-        const uint32_t dmask = (1u << nb) - 1u;
-        uint4* wh4 = reinterpret_cast<uint4*>(whist);
-        wh4[lane * 2] = make_uint4(0u, 0u, 0u, 0u);
-        wh4[lane * 2 + 1] = make_uint4(0u, 0u, 0u, 0u);
-        __syncwarp();
-        for (uint32_t i = lane; i < L; i += 32) {
-            const uint32_t d = list[i] - lo;
-            if ((d >> top) == prefix) atomicAdd(&whist[(d >> s) & dmask], 1u);
-        }
-        __syncwarp();
-        const uint4 a = wh4[lane * 2], b = wh4[lane * 2 + 1];
-        const uint32_t c[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-        uint32_t sum = 0u;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) sum += c[i];
-        uint32_t incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-            if (lane >= o) incl += n;
-        }
-        uint32_t base = incl - sum;
-        const bool mine = base < r && r <= base + sum;
-        const unsigned m = __ballot_sync(0xFFFFFFFFu, mine);
-        if (m == 0u) return false;
-        uint32_t bin = 0u, rank = 0u, count = 0u;
-        if (mine) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                if (count == 0u && r <= base + c[i]) {
-                    bin = (uint32_t)(lane * 8 + i);
-                    rank = r - base;
-                    count = c[i];
-                }
-                base += c[i];
-            }
-        }
-        const int src = __ffs(m) - 1;
-        bin = __shfl_sync(0xFFFFFFFFu, bin, src);
-        r = __shfl_sync(0xFFFFFFFFu, rank, src);
-        cnt = __shfl_sync(0xFFFFFFFFu, count, src);
-        prefix = (prefix << nb) | bin;
-        top = s;
-        __syncwarp();
-    }
-    *T = lo + prefix;
-    *q = r;
-    *n_eq = cnt;
-    return true;
-}
 
 // V = vectors per thread, NT = threads per CTA; V*NT*8 >= cols.
 template <int DT, int V, int NT, int MINB>
@@ -390,103 +260,20 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
                 }
             }
             if (!done) {
-                // full radix select over all keys
                 MOSAIC_STAT(5);
-                for (int b = tid; b < kBins1; b += NT) buf[b] = 0u;
+                for (int b = tid; b < kBins1; b += NT) buf[b] = 0u;   // the list may have left entries
                 __syncthreads();
-#pragma unroll
-                for (int v = 0; v < V; ++v)
-#pragma unroll
-                    for (int e = 0; e < kVec; ++e) {
-                        atomicAdd(&buf[key_of(v, e) >> 20], 1u);
-                    }
-                __syncthreads();
-                SelectResult r = find_bin<NT, kBins1>(buf, warp_tot, &sel3, uk);
-                uint32_t prefix = r.bin << 20;
-#pragma unroll
-                for (int v = 0; v < V; ++v)
-#pragma unroll
-                    for (int e = 0; e < kVec; ++e) {
-                        const uint32_t key = key_of(v, e);
-                        if ((key & 0xFFF00000u) == prefix) atomicAdd(&buf[(key >> 10) & 0x3FFu], 1u);
-                    }
-                __syncthreads();
-                r = find_bin<NT, kBins23>(buf, warp_tot, &sel3, r.rank);
-                prefix |= r.bin << 10;
-#pragma unroll
-                for (int v = 0; v < V; ++v)
-#pragma unroll
-                    for (int e = 0; e < kVec; ++e) {
-                        const uint32_t key = key_of(v, e);
-                        if ((key & 0xFFFFFC00u) == prefix) atomicAdd(&buf[key & 0x3FFu], 1u);
-                    }
-                __syncthreads();
-                r = find_bin<NT, kBins23>(buf, warp_tot, &sel3, r.rank);
-                T = prefix | r.bin;
-                q = r.rank;      // entries equal to T that are pruned (1 <= q <= n_eq)
-                n_eq = r.count;
+                radix_select_row<V>(key_of, uk, buf, warp_tot, &sel3, NT, &T, &q, &n_eq);
             }
             center = have_center ? (uint32_t)(((uint64_t)center + T) >> 1) : T;
             have_center = true;
         }
 
-        // prune flags: key < T, and every key == T when all ties go
         uint32_t pruned[V];
-        const uint32_t below = (q == n_eq) ? T + 1u : T;   // T < 2^31
 #pragma unroll
-        for (int v = 0; v < V; ++v) {
-            pruned[v] = 0u;
-            if (k > 0) {
-#pragma unroll
-                for (int e = 0; e < kVec; ++e) pruned[v] |= (key_of(v, e) < below) ? (1u << e) : 0u;
-            }
-        }
-        if (k > 0 && q != n_eq) {
-            // ties at the threshold: prune the q lowest-indexed entries equal to T
-            uint32_t before = 0u;  // ties in earlier vector slots (all threads)
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                uint32_t eq = 0u;
-#pragma unroll
-                for (int e = 0; e < kVec; ++e) eq |= (key_of(v, e) == T) ? (1u << e) : 0u;
-                uint32_t total;
-                uint32_t idx = before + block_excl_scan<NT>(__popc(eq), warp_tot, &total);
-#pragma unroll
-                for (int e = 0; e < kVec; ++e)
-                    if (eq & (1u << e)) {
-                        if (idx < q) pruned[v] |= (1u << e);
-                        ++idx;
-                    }
-                before += total;
-            }
-        }
-
-        // write W' and the keep bitmask
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const int vec = v * NT + tid;
-            const int c0 = vec * kVec;
-            if (vec < nvec) {
-#pragma unroll
-                for (int e = 0; e < kVec; ++e)
-                    if (pruned[v] & (1u << e)) raw[v].zero(e);
-                if (c0 + kVec <= cols) {
-                    raw[v].store((char*)W_out + (row_off + c0) * (DT == MOSAIC_F32 ? 4 : 2));
-                } else {
-#pragma unroll
-                    for (int e = 0; e < kVec; ++e)
-                        if (c0 + e < cols) raw[v].put_scalar(e, W_out, row_off + c0 + e);
-                }
-            }
-            if (mask_bytes != nullptr && vec < mask_row_bytes) {
-                uint32_t keep = 0u;
-                if (vec < nvec) {
-                    const int nvalid = (cols - c0 < kVec) ? cols - c0 : kVec;
-                    keep = ~pruned[v] & ((1u << nvalid) - 1u);
-                }
-                mask_bytes[row * mask_row_bytes + vec] = (uint8_t)keep;
-            }
-        }
+        for (int v = 0; v < V; ++v) pruned[v] = 0u;
+        if (k > 0) prune_flags<V>(key_of, T, q, n_eq, warp_tot, NT, pruned);
+        store_row<DT, V>(raw, pruned, W_out, row_off, cols, nvec, NT, mask_bytes, row * mask_row_bytes, mask_row_bytes);
     }
 }
 
