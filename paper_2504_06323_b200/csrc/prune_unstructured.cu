@@ -277,6 +277,434 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// bf16 rows, classified in the bf16 domain
+// ---------------------------------------------------------------------------------------------
+constexpr int kFastV = 4;          // vectors (of 8 columns) per thread
+constexpr int kWinBins = 1024;     // histogram over the top 10 bits of a window
+constexpr int kBinListCap = 512;   // keys of one histogram bin that warp 0 will rank; also the sample size limit
+
+__device__ __forceinline__ float rcp_approx(float x) {   // relative error <= 2^-23 for normal x
+    float r;
+    asm("rcp.approx.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "l"(gmem)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+__device__ __forceinline__ void sts_u16_zero(void* smem) {
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "h"((unsigned short)0) : "memory");
+}
+
+// A word holds two bf16 weights.  With x = word | 0x80008000 (sign bits forced on, so each 16-bit
+// lane is 0x8000 + magnitude) and A two 16-bit thresholds <= 0x8000, the lanes of x - A never
+// borrow from each other and bit 15 / bit 31 of the difference is set iff magnitude >= threshold.
+// comb_flags gathers those two bits of the four words of a vector into one word: word i's low
+// weight (element 2i) lands on bit 15-i, its high weight (element 2i+1) on bit 31-i.
+__device__ __forceinline__ uint32_t comb_flags(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3) {
+    return (t0 & 0x80008000u) | ((t1 >> 1) & 0x40004000u) | ((t2 >> 2) & 0x20002000u) | ((t3 >> 3) & 0x10001000u);
+}
+__device__ __forceinline__ int flag_elem(int b) {   // flag bit of comb_flags -> element 0..7 of the vector
+    const int half = b >> 4;
+    const int i = (15 | (half << 4)) - b;
+    return (i << 1) | half;
+}
+
+// The slow, always-exact treatment of one row held in shared memory: full radix select, ordered
+// ties, store.  Returns the row's threshold key.  hist[0..kBins1) must be zero; it is zero after.
+template <int V>
+__device__ __noinline__ uint32_t generic_row_bf16(const uint4* my_vecs, int nt, const float* __restrict__ norms, int cols,
+                                                  int nvec, uint32_t k, uint32_t* hist, uint32_t* warp_tot,
+                                                  SelectResult* sel3, void* W_out, int64_t row_off, uint8_t* mask_bytes,
+                                                  int64_t mask_off, int mask_row_bytes) {
+    const int tid = threadIdx.x;
+    Raw8<MOSAIC_BF16> raw[V];
+    float nrm[V][kVec];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int vec = v * nt + tid;
+        if (vec < nvec) {
+            const uint4 u = my_vecs[v * nt];
+            raw[v].w[0] = u.x; raw[v].w[1] = u.y; raw[v].w[2] = u.z; raw[v].w[3] = u.w;
+        } else {
+            raw[v].clear();
+        }
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+            const int c = vec * kVec + e;
+            nrm[v][e] = (c < cols) ? __ldg(norms + c) : __int_as_float(0x7F800000);
+        }
+    }
+    auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))); };
+    uint32_t T, q, n_eq, pruned[V];
+    radix_select_row<V>(key_of, k, hist, warp_tot, sel3, nt, &T, &q, &n_eq);
+    prune_flags<V>(key_of, T, q, n_eq, warp_tot, nt, pruned);
+    store_row<MOSAIC_BF16, V>(raw, pruned, W_out, row_off, cols, nvec, nt, mask_bytes, mask_off, mask_row_bytes);
+    return T;
+}
+
+// cols % 8 == 0, 0 < k < cols, blockDim.x = nt a multiple of 32 with kFastV*nt*8 >= cols and nt <= cols/8;
+// dynamic shared memory: 2 * kFastV * nt * 16 bytes.
+template <int MAXNT, int MINB>
+__global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint16_t* W_in, uint16_t* W_out, int64_t rows,
+                                                                       int cols, int64_t ldw,
+                                                                       const float* __restrict__ norms, int k,
+                                                                       uint8_t* __restrict__ mask_bytes, int mask_row_bytes) {
+    constexpr int V = kFastV;
+    extern __shared__ __align__(16) uint4 rowbuf[];      // [2][V][nt]: the row being selected and the next one
+    __shared__ __align__(16) uint32_t buf[kBins1];       // window histogram + one key per bin, or the full select's histogram
+    __shared__ __align__(16) uint32_t whist[256];        // warp 0's digit histogram
+    __shared__ uint32_t coarse[32];                      // window histogram summed over groups of 32 bins
+    __shared__ uint32_t list[kBinListCap];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ uint32_t red[32];
+    __shared__ uint32_t n_list;
+    __shared__ SelectResult sel3;
+    __shared__ RowSelect sel;
+    __shared__ uint8_t spread[16];                       // bits abcd -> 0a0b0c0d
+
+    const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = nt >> 5;
+    const int nvec = cols >> 3;
+    const uint32_t uk = (uint32_t)k;
+    uint32_t* hist = buf;
+    uint32_t* slot = buf + kWinBins;
+
+    for (int b = tid; b < kBins1; b += nt) buf[b] = 0u;
+    if (tid < 32) coarse[tid] = 0u;
+    if (tid < 16) spread[tid] = (uint8_t)((tid & 1) | ((tid & 2) << 1) | ((tid & 4) << 2) | ((tid & 8) << 3));
+    if (tid == 0) n_list = 0u;
+    bool fin = true;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+            const int c = (v * nt + tid) * kVec + e;
+            if (c < cols) {
+                const float n = __ldg(norms + c);
+                fin = fin && (n >= 0.0f) && (n <= 3.402823466e38f);
+            }
+        }
+    // The bf16-domain classification needs scores that are monotone in |w| for every column:
+    // true for finite norms >= 0.  Otherwise every row takes the exact slow path.
+    const bool all_finite = __syncthreads_and(fin ? 1 : 0) != 0;
+
+    auto prefetch = [&](int slot_idx, int64_t row) {
+        const uint16_t* src = W_in + row * ldw;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int vec = v * nt + tid;
+            if (vec < nvec) cp_async16(&rowbuf[(slot_idx * V + v) * nt + tid], src + (int64_t)vec * kVec);
+        }
+        cp_async_commit();
+    };
+
+    // ---- window state: [win_lo, win_lo + 2^win_w) and the thread's per-column thresholds
+    uint32_t Alo[V][4], Ahi[V][4];
+    uint32_t win_lo = 0u;
+    int win_w = 0;
+    bool win_valid = false;
+
+    // Thresholds of the window of width 2^w centred on `center`.  For column j with norm n:
+    //   magnitude bits a <  Alo  =>  score key < lo      (surely pruned once T >= lo)
+    //   magnitude bits a >= Ahi  =>  score key >= hi     (surely kept once T < hi)
+    // With x = l/n, the estimate x' = l * rcp(n) is within 2^-22 of x and g = top 16 bits of x' is
+    // the bf16 pattern just below or at x'.  Patterns <= g-2 are more than one bf16 step (2^-8)
+    // below x, so their product with n rounds below l; patterns >= g+2 are above x.  Alo = g-2 and
+    // Ahi = g+2 keep an extra step in hand.  The window is refused where products could be
+    // subnormal (lo < 2^24) or overflow, and columns whose norm is outside [2^-100, 2^100] get
+    // thresholds that make every weight a candidate (norm 0: every finite weight scores 0).
+    auto set_window = [&](uint32_t center, int w) {
+        const uint32_t half = 1u << (w - 1);
+        win_valid = false;
+        if (center < (1u << 24) + half) return;
+        const uint32_t lo = center - half;
+        if (lo > 0x7F7FFFFFu - (1u << w)) return;
+        const float flo = __uint_as_float(lo), fhi = __uint_as_float(lo + (1u << w));
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t al[2], ah[2];
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int c = (v * nt + tid) * kVec + 2 * i + h;
+                    al[h] = 0u;   // past the end of the row: never below, never a candidate
+                    ah[h] = 0u;
+                    if (c < cols) {
+                        const float n = __ldg(norms + c);
+                        if (n == 0.0f) {
+                            al[h] = 0x7F80u;
+                            ah[h] = 0x7F82u;
+                        } else if (!(n >= 0x1p-100f && n <= 0x1p100f)) {
+                            al[h] = 0u;
+                            ah[h] = 0x8000u;
+                        } else {
+                            const float r = rcp_approx(n);
+                            const uint32_t gl = __float_as_uint(__fmul_rn(flo, r)) >> 16;
+                            const uint32_t gh = __float_as_uint(__fmul_rn(fhi, r)) >> 16;
+                            al[h] = gl > 2u ? gl - 2u : 0u;
+                            ah[h] = gh + 2u;
+                        }
+                    }
+                }
+                Alo[v][i] = al[0] | (al[1] << 16);
+                Ahi[v][i] = ah[0] | (ah[1] << 16);
+            }
+        win_lo = lo;
+        win_w = w;
+        win_valid = true;
+    };
+
+    // Exact score key of element e of the thread's vector v of the row in buffer `cur`.
+    auto cand_key = [&](int cur, int v, int e) -> uint32_t {
+        const uint16_t* p = reinterpret_cast<const uint16_t*>(&rowbuf[(cur * V + v) * nt + tid]);
+        const uint32_t a = ((uint32_t)p[e] & 0x7FFFu) << 16;
+        return __float_as_uint(__fmul_rn(__ldg(norms + (v * nt + tid) * kVec + e), __uint_as_float(a)));
+    };
+
+    // Key of the matching quantile of one key per thread (element 0 of vector 0), or 0.
+    auto sample_center = [&](int cur) -> uint32_t {
+        list[tid] = cand_key(cur, 0, 0);
+        __syncthreads();
+        if (wid == 0) {
+            uint32_t r_s = (uint32_t)(((uint64_t)uk * (uint32_t)nt + (uint32_t)cols / 2u) / (uint32_t)cols);
+            r_s = r_s < 1u ? 1u : (r_s > (uint32_t)nt ? (uint32_t)nt : r_s);
+            uint32_t t = 0u, qq = 0u, ne = 0u;
+            const bool ok = warp_select(list, (uint32_t)nt, 0u, 31, r_s, whist, &t, &qq, &ne);
+            if (lane == 0) {
+                sel.ok = ok ? 1u : 0u;
+                sel.lo = t;
+            }
+        }
+        __syncthreads();
+        return sel.ok != 0u ? sel.lo : 0u;
+    };
+
+    // One attempt on the current window.  0: row finished and stored (T_out set); 1: the k-th key
+    // is outside the window; 2: the row needs the slow path (ties to split by column, bin overflow).
+    auto fast_attempt = [&](int cur, int64_t row, uint32_t& T_out) -> int {
+        const uint32_t lo = win_lo, width = 1u << win_w;
+        const int shift = win_w - 10;
+        uint32_t cand[V], keepf[V];   // flag words (comb_flags layout): candidates; weights not surely below lo
+        uint32_t below = 0u;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const uint4 r = rowbuf[(cur * V + v) * nt + tid];
+            const uint32_t x0 = r.x | 0x80008000u, x1 = r.y | 0x80008000u, x2 = r.z | 0x80008000u, x3 = r.w | 0x80008000u;
+            keepf[v] = comb_flags(x0 - Alo[v][0], x1 - Alo[v][1], x2 - Alo[v][2], x3 - Alo[v][3]);
+            const uint32_t above = comb_flags(x0 - Ahi[v][0], x1 - Ahi[v][1], x2 - Ahi[v][2], x3 - Ahi[v][3]);
+            cand[v] = keepf[v] & ~above;
+            below += 8u - (uint32_t)__popc(keepf[v]);
+        }
+        // exact scores of the candidates: below lo, or into the window histogram
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            uint32_t c = cand[v];
+            while (c) {
+                const int b = __ffs(c) - 1;
+                c &= c - 1u;
+                const uint32_t key = cand_key(cur, v, flag_elem(b));
+                const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
+                if (d < width) {
+                    const uint32_t bin = d >> shift;
+                    atomicAdd(&hist[bin], 1u);
+                    atomicAdd(&coarse[bin >> 5], 1u);
+                    slot[bin] = key;
+                } else {
+                    below += d >> 31;
+                }
+            }
+        }
+        below = __reduce_add_sync(0xFFFFFFFFu, below);
+        if (lane == 0) red[wid] = below;
+        __syncthreads();
+        if (wid == 0) {
+            const uint32_t n_below = __reduce_add_sync(0xFFFFFFFFu, (lane < nwarps) ? red[lane] : 0u);
+            const uint32_t cc = coarse[lane];
+            uint32_t incl = cc;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            const uint32_t base = n_below + incl - cc;
+            const unsigned m = __ballot_sync(0xFFFFFFFFu, base < uk && uk <= base + cc);
+            bool ok = m != 0u;
+            uint32_t bin = 0u, r_bin = 0u, n_bin = 0u;
+            if (ok) {
+                const int seg = __ffs(m) - 1;
+                const uint32_t seg_base = __shfl_sync(0xFFFFFFFFu, base, seg);
+                const uint32_t f = hist[seg * 32 + lane];
+                uint32_t fi = f;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, fi, o);
+                    if (lane >= o) fi += n;
+                }
+                const uint32_t fb = seg_base + fi - f;
+                const unsigned m2 = __ballot_sync(0xFFFFFFFFu, fb < uk && uk <= fb + f);
+                ok = m2 != 0u;
+                if (ok) {
+                    const int l2 = __ffs(m2) - 1;
+                    bin = (uint32_t)(seg * 32 + l2);
+                    r_bin = uk - __shfl_sync(0xFFFFFFFFu, fb, l2);
+                    n_bin = __shfl_sync(0xFFFFFFFFu, f, l2);
+                }
+            }
+            __syncwarp();
+            uint4* h4 = reinterpret_cast<uint4*>(hist);   // left clean for the next attempt
+#pragma unroll
+            for (int j = 0; j < kWinBins / 128; ++j) h4[j * 32 + lane] = make_uint4(0u, 0u, 0u, 0u);
+            coarse[lane] = 0u;
+            if (lane == 0) {
+                sel.ok = ok ? 1u : 0u;
+                sel.bin = bin;
+                sel.q = r_bin;       // rank inside the bin
+                sel.n_eq = n_bin;    // keys in the bin
+                sel.T = slot[bin];   // the key itself if it is alone in its bin
+                n_list = 0u;
+            }
+        }
+        __syncthreads();
+        if (sel.ok == 0u) return 1;
+        const uint32_t bin = sel.bin, r_bin = sel.q, n_bin = sel.n_eq;
+        uint32_t T = sel.T;
+        MOSAIC_STAT_ADD(7, n_bin);
+        if (n_bin > 1u) {
+            if (n_bin > (uint32_t)kBinListCap) return 2;
+            // collect the keys of that bin; warp 0 ranks them
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                uint32_t c = cand[v];
+                while (c) {
+                    const int b = __ffs(c) - 1;
+                    c &= c - 1u;
+                    const uint32_t key = cand_key(cur, v, flag_elem(b));
+                    if (((key - lo) >> shift) == bin) {
+                        const uint32_t pos = atomicAdd(&n_list, 1u);
+                        if (pos < (uint32_t)kBinListCap) list[pos] = key;
+                    }
+                }
+            }
+            __syncthreads();
+            if (wid == 0) {
+                uint32_t t = 0u, qq = 0u, ne = 0u;
+                const bool ok = warp_select(list, n_bin, lo + (bin << shift), shift, r_bin, whist, &t, &qq, &ne);
+                if (lane == 0) {
+                    sel.ok = (ok && qq == ne) ? 1u : 0u;   // a tie group that is only partly pruned goes the slow way
+                    sel.T = t;
+                }
+            }
+            __syncthreads();
+            if (sel.ok == 0u) return 2;
+            T = sel.T;
+        } else {
+            MOSAIC_STAT(6);
+        }
+
+        // prune: surely below lo, or a candidate whose exact key is <= T
+        const uint32_t thr = T + 1u;
+        uint16_t* out_row = W_out + row * ldw;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int vec = v * nt + tid;
+            uint32_t c = cand[v], gone = 0u;
+            uint16_t* mine = reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + tid]);
+            while (c) {
+                const int b = __ffs(c) - 1;
+                c &= c - 1u;
+                const int e = flag_elem(b);
+                if (cand_key(cur, v, e) < thr) {
+                    gone |= 1u << b;
+                    sts_u16_zero(mine + e);
+                }
+            }
+            if (vec < nvec) {
+                const uint4 r = rowbuf[(cur * V + v) * nt + tid];
+                uint4 o;
+                // byte 1 / byte 3 of a difference carry the "not below" flag in their top bit: spread it over the lane
+                o.x = r.x & __byte_perm((r.x | 0x80008000u) - Alo[v][0], 0u, 0xBB99u);
+                o.y = r.y & __byte_perm((r.y | 0x80008000u) - Alo[v][1], 0u, 0xBB99u);
+                o.z = r.z & __byte_perm((r.z | 0x80008000u) - Alo[v][2], 0u, 0xBB99u);
+                o.w = r.w & __byte_perm((r.w | 0x80008000u) - Alo[v][3], 0u, 0xBB99u);
+                st_stream16(out_row + (int64_t)vec * kVec, o);
+            }
+            if (mask_bytes != nullptr && vec < mask_row_bytes) {
+                uint32_t keep = 0u;
+                if (vec < nvec) {
+                    const uint32_t rr = __brev(keepf[v] & ~gone);   // odd elements on bits 0..3, even ones on bits 16..19
+                    keep = (uint32_t)spread[(rr >> 16) & 0xFu] | ((uint32_t)spread[rr & 0xFu] << 1);
+                }
+                mask_bytes[row * mask_row_bytes + vec] = (uint8_t)keep;
+            }
+        }
+        T_out = T;
+        return 0;
+    };
+
+    int cur = 0;
+    int64_t row = blockIdx.x;
+    if (row < rows) prefetch(0, row);
+    for (; row < rows; row += gridDim.x, cur ^= 1) {
+        if (row + gridDim.x < rows) prefetch(cur ^ 1, row + gridDim.x);
+        else cp_async_commit();
+        cp_async_wait_all_but_one();   // this row has landed; a thread only ever reads the vectors it copied itself
+
+        MOSAIC_STAT(0);
+        int status = 1;
+        uint32_t T_row = 0u;
+        if (all_finite) {
+            for (int tries = 0; tries < 2 && status == 1; ++tries) {
+                if (!win_valid || tries == 1) {
+                    MOSAIC_STAT(3);
+                    set_window(sample_center(cur), kSampleBits);
+                }
+                if (!win_valid) break;
+                status = fast_attempt(cur, row, T_row);
+                if (status == 0) MOSAIC_STAT(win_w == kTrackBits ? 2 : 4);
+            }
+        }
+        if (status != 0) {
+            MOSAIC_STAT(5);
+            for (int b = tid; b < kWinBins; b += nt) slot[b] = 0u;
+            __syncthreads();
+            T_row = generic_row_bf16<V>(&rowbuf[(cur * V) * nt + tid], nt, norms, cols, nvec, uk, buf, warp_tot, &sel3, W_out,
+                                        row * ldw, mask_bytes, row * mask_row_bytes, mask_row_bytes);
+        }
+        if (all_finite && (status != 0 || win_w != kTrackBits)) set_window(T_row, kTrackBits);
+    }
+}
+
+template <int MAXNT, int MINB>
+static int launch_prune_bf16(const void* W_in, void* W_out, int64_t rows, int cols, int64_t ldw, const float* norms, int k,
+                             uint32_t* mask, int nt, cudaStream_t st) {
+    static int blocks_per_sm[MAXNT / 32 + 1] = {0};
+    const size_t dyn = (size_t)2 * kFastV * nt * sizeof(uint4);
+    int& bps = blocks_per_sm[nt / 32];
+    if (bps == 0) {
+        if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)((size_t)2 * kFastV * MAXNT * sizeof(uint4))) != cudaSuccess)
+            return MOSAIC_ERR_CUDA;
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB>, nt, dyn) != cudaSuccess || n < 1) {
+            (void)cudaGetLastError();
+            n = 1;
+        }
+        bps = n > MOSAIC_FAST_MAX_CTAS ? MOSAIC_FAST_MAX_CTAS : n;
+    }
+    int64_t grid = (int64_t)sm_count() * bps;
+    if (grid > rows) grid = rows;
+    const int words = (cols + 31) / 32;
+    prune_rows_bf16_kernel<MAXNT, MINB><<<(unsigned)grid, nt, dyn, st>>>(
+        static_cast<const uint16_t*>(W_in), static_cast<uint16_t*>(W_out), rows, cols, ldw, norms, k,
+        reinterpret_cast<uint8_t*>(mask), words * 4);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
 template <int DT, int V, int NT, int MINB>
 static int launch_prune(const void* W_in, void* W_out, int64_t rows, int cols, int64_t ldw, const float* norms, int k,
                         uint32_t* mask, cudaStream_t st) {
@@ -358,6 +786,16 @@ extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t 
         if (a < b + span && b < a + span) return MOSAIC_ERR_ALIASING;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dtype == MOSAIC_BF16 && cols % kVec == 0 && k > 0 && k < cols) {
+        const int nvec = (int)(cols / kVec);
+        const int nt = ((nvec + kFastV - 1) / kFastV + 31) / 32 * 32;   // threads so that kFastV vectors each cover the row
+        if (nvec >= 256 && nt <= 128)
+            return launch_prune_bf16<128, 6>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
+        if (nvec >= 256 && nt <= 256)
+            return launch_prune_bf16<256, 3>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
+        if (nvec >= 256 && nt <= 512)
+            return launch_prune_bf16<512, 1>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
+    }
     if (dtype == MOSAIC_BF16)
         return dispatch_prune<MOSAIC_BF16>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, st);
     return dispatch_prune<MOSAIC_F32>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, st);
