@@ -307,6 +307,13 @@ __device__ __forceinline__ void sts_u16_zero(void* smem) {
 __device__ __forceinline__ uint32_t comb_flags(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3) {
     return (t0 & 0x80008000u) | ((t1 >> 1) & 0x40004000u) | ((t2 >> 2) & 0x20002000u) | ((t3 >> 3) & 0x10001000u);
 }
+// Bit 15 / bit 31 of t spread over their 16-bit lane: 0xFFFF where the flag is set.  (prmt's
+// generic mode replicates the top bit of the selected byte when bit 3 of the selector nibble is set.)
+__device__ __forceinline__ uint32_t lane_mask_from_flags(uint32_t t) {
+    uint32_t m;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(m) : "r"(t), "r"(0u), "r"(0xBB99u));
+    return m;
+}
 __device__ __forceinline__ int flag_elem(int b) {   // flag bit of comb_flags -> element 0..7 of the vector
     const int half = b >> 4;
     const int i = (15 | (half << 4)) - b;
@@ -626,10 +633,10 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
                 const uint4 r = rowbuf[(cur * V + v) * nt + tid];
                 uint4 o;
                 // byte 1 / byte 3 of a difference carry the "not below" flag in their top bit: spread it over the lane
-                o.x = r.x & __byte_perm((r.x | 0x80008000u) - Alo[v][0], 0u, 0xBB99u);
-                o.y = r.y & __byte_perm((r.y | 0x80008000u) - Alo[v][1], 0u, 0xBB99u);
-                o.z = r.z & __byte_perm((r.z | 0x80008000u) - Alo[v][2], 0u, 0xBB99u);
-                o.w = r.w & __byte_perm((r.w | 0x80008000u) - Alo[v][3], 0u, 0xBB99u);
+                o.x = r.x & lane_mask_from_flags((r.x | 0x80008000u) - Alo[v][0]);
+                o.y = r.y & lane_mask_from_flags((r.y | 0x80008000u) - Alo[v][1]);
+                o.z = r.z & lane_mask_from_flags((r.z | 0x80008000u) - Alo[v][2]);
+                o.w = r.w & lane_mask_from_flags((r.w | 0x80008000u) - Alo[v][3]);
                 st_stream16(out_row + (int64_t)vec * kVec, o);
             }
             if (mask_bytes != nullptr && vec < mask_row_bytes) {
