@@ -209,8 +209,8 @@ def run_native(args, cfg):
         counts = driver.exchange_counts(st.counts, total_cfg.n_layers, rank, world)
         _, k, _ = driver.plan_sparsity(total_cfg, counts)
         if record: ev[3].record()
-        for layer in mine:
-            launches += driver.prune_unstructured_layer(st, layer, k)
+        driver.prune_unstructured_all(st, k)
+        launches += 2 * len({cfg.shape(p)[1] for p in PROJECTIONS})      # planning + pruning launch per distinct row length
         if record: ev[4].record()
         return launches
 

@@ -192,6 +192,34 @@ int mosaic_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64
                               uint32_t *mask_out, void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * mosaic_prune_unstructured_batch - mosaic_prune_unstructured for a list of
+ * projections in as few launches as possible (a model has N*M projections,
+ * Section 3.1; each is a few tens of microseconds of work, so one launch per
+ * projection is dominated by launch and ramp-up time).  Results are bit for
+ * bit those of calling mosaic_prune_unstructured once per job.
+ *   jobs     HOST array of n_jobs descriptors (read during the call only);
+ *            every pointer inside a descriptor is a device pointer with the
+ *            meaning and alignment rules of mosaic_prune_unstructured
+ *   dtype    one dtype for the whole list
+ *   ws       device scratch, >= mosaic_prune_unstructured_batch_workspace_bytes
+ *            for the same list; it receives, per job, the key window and the
+ *            per-column thresholds a planning kernel derives from three rows
+ * Jobs must not overlap each other's outputs.  Not re-entrant: one call at a
+ * time per process.
+ * ------------------------------------------------------------------------- */
+typedef struct mosaic_prune_job {
+    const void *W_in;
+    void *W_out;
+    int64_t rows, cols, ldw;
+    const float *norms;
+    int64_t k;
+    uint32_t *mask_out;
+} mosaic_prune_job;
+size_t mosaic_prune_unstructured_batch_workspace_bytes(const mosaic_prune_job *jobs, int64_t n_jobs, int dtype);
+int mosaic_prune_unstructured_batch(const mosaic_prune_job *jobs, int64_t n_jobs, int dtype, void *ws,
+                                    size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
  * mosaic_prune_structured_compact - structured projection pruning (Section
  * 4.1.3: remove the lowest-magnitude heads and channels; Section 2.3:
  * structured pruning removes whole data structures and leaves smaller dense

@@ -32,6 +32,7 @@ SYMBOLS = (
     "mosaic_outlier_ratio_static_max_workspace_bytes", "mosaic_outlier_ratio_static",
     "mosaic_allocate_sparsity",
     "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
+    "mosaic_prune_unstructured_batch_workspace_bytes", "mosaic_prune_unstructured_batch",
     "mosaic_prune_structured_compact_workspace_bytes", "mosaic_prune_structured_compact",
     "mosaic_rank_units", "mosaic_sum_unit_scores",
 )
@@ -81,6 +82,10 @@ def lib() -> C.CDLL:
         L.mosaic_prune_unstructured_workspace_bytes.argtypes = [i64, i64]
         L.mosaic_prune_unstructured.restype = ci
         L.mosaic_prune_unstructured.argtypes = [vp, vp, i64, i64, i64, ci, vp, i64, vp, vp, sz, vp]
+        L.mosaic_prune_unstructured_batch_workspace_bytes.restype = sz
+        L.mosaic_prune_unstructured_batch_workspace_bytes.argtypes = [vp, i64, ci]
+        L.mosaic_prune_unstructured_batch.restype = ci
+        L.mosaic_prune_unstructured_batch.argtypes = [vp, i64, ci, vp, sz, vp]
         L.mosaic_prune_structured_compact_workspace_bytes.restype = sz
         L.mosaic_prune_structured_compact_workspace_bytes.argtypes = [i64, i64]
         L.mosaic_prune_structured_compact.restype = ci
@@ -264,6 +269,38 @@ def mosaic_prune_unstructured(W_in: torch.Tensor, W_out: torch.Tensor, norms: to
             raise ValueError("mask_out must be a contiguous int32 [rows, ceil(cols/32)]")
     _check(lib().mosaic_prune_unstructured(p, po, rows, cols, ldw, _dtype_code(W_in), norms.data_ptr(), int(k),
                                            _ptr(mask_out), None, 0, _stream(stream)), "mosaic_prune_unstructured")
+
+
+class PruneJob(C.Structure):
+    """mosaic_prune_job of include/mosaic.h."""
+    _fields_ = [("W_in", C.c_void_p), ("W_out", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64),
+                ("ldw", C.c_int64), ("norms", C.c_void_p), ("k", C.c_int64), ("mask_out", C.c_void_p)]
+
+
+def mosaic_prune_unstructured_batch(jobs, ws: Workspace | None = None, stream=None) -> None:
+    """mosaic_prune_unstructured over a list of (W_in, W_out, norms, k, mask_out or None) in few launches."""
+    if not jobs:
+        return
+    arr = (PruneJob * len(jobs))()
+    dtype = jobs[0][0].dtype
+    for i, (W_in, W_out, norms, k, mask_out) in enumerate(jobs):
+        p, rows, cols, ldw = _mat(W_in, "W_in")
+        po, r2, c2, ld2 = _mat(W_out, "W_out")
+        if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or W_in.dtype != dtype or (rows > 1 and ld2 != ldw):
+            raise ValueError("W_out must match W_in in shape, dtype and leading dimension; one dtype per batch")
+        _dev(norms, "norms", torch.float32)
+        if norms.numel() != cols:
+            raise ValueError("norms must be [cols]")
+        if mask_out is not None:
+            _dev(mask_out, "mask_out", torch.int32)
+            if tuple(mask_out.shape) != (rows, (cols + 31) // 32) or not mask_out.is_contiguous():
+                raise ValueError("mask_out must be a contiguous int32 [rows, ceil(cols/32)]")
+        arr[i] = PruneJob(p, po, rows, cols, ldw, norms.data_ptr(), int(k), _ptr(mask_out))
+    L = lib()
+    code = _dtype_code(jobs[0][0])
+    wp, wn = _ws(ws, jobs[0][0].device).get(L.mosaic_prune_unstructured_batch_workspace_bytes(C.addressof(arr), len(jobs), code))
+    _check(L.mosaic_prune_unstructured_batch(C.addressof(arr), len(jobs), code, wp, wn, _stream(stream)),
+           "mosaic_prune_unstructured_batch")
 
 
 def mosaic_prune_structured_compact(W_in: torch.Tensor, norms: torch.Tensor | None, row_group: int, col_group: int,

@@ -32,6 +32,8 @@
 //       between A_lo[j] and A_hi[j] - a few percent of the row - are the
 //       candidates, and only they get an exact fp32 score.
 //   prune_rows_kernel       any dtype, any shape; scores of all entries in fp32.
+#include <vector>
+
 #include "select.cuh"
 
 #ifndef MOSAIC_PRUNE_MINB_2X256
@@ -53,7 +55,10 @@ __device__ unsigned long long g_prune_stats[8];
 #endif
 
 constexpr int kListCap = kBins1;  // candidate list shares the histogram's storage
-constexpr int kTrackBits = 21;    // width (log2, in key units) of a window carried from row to row
+#ifndef MOSAIC_TRACK_BITS
+#define MOSAIC_TRACK_BITS 21
+#endif
+constexpr int kTrackBits = MOSAIC_TRACK_BITS;    // width (log2, in key units) of a window carried from row to row
 constexpr int kSampleBits = 23;   // width of the window around a sampled quantile
 
 struct RowSelect {   // hand-over between warp 0 and the CTA during a window attempt
@@ -320,6 +325,109 @@ __device__ __forceinline__ int flag_elem(int b) {   // flag bit of comb_flags ->
     return (i << 1) | half;
 }
 
+// One matrix to prune, as the kernels see it.  A launch works through a list of them, all with
+// the same number of columns; rows are numbered across the list (row0 = first global row).
+struct PruneJob {
+    const uint16_t* W_in;
+    uint16_t* W_out;
+    const float* norms;
+    uint8_t* mask;          // keep bitmask as bytes, or nullptr
+    uint32_t* plan;         // window and thresholds prepared by prune_plan_kernel, or nullptr
+    int64_t rows, ldw, row0;
+    int k, mask_row_bytes;
+};
+template <int NJ>
+struct PruneJobList {
+    int n;
+    PruneJob job[NJ];
+};
+constexpr int kBatchJobs = 256;   // jobs per launch of the batched kernels (the list travels as a kernel parameter)
+
+// Layout of a plan (32-bit words): [0] valid, [1] window lo, [2] window width log2, [3] unused, then
+// for every vector slot vec = v*nt + tid eight words: Alo[0..3], Ahi[0..3].
+constexpr int kPlanHeader = 4;
+inline size_t plan_words(int nt) { return (size_t)kPlanHeader + (size_t)kFastV * nt * 8; }
+
+// Thresholds of the window of width 2^w centred on `center`, for the columns of this thread
+// (vectors v*nt + tid).  For column j with norm n:
+//   magnitude bits a <  Alo  =>  score key < lo      (surely pruned once T >= lo)
+//   magnitude bits a >= Ahi  =>  score key >= hi     (surely kept once T < hi)
+// With x = l/n, the estimate x' = l * rcp(n) is within 2^-22 of x and g = top 16 bits of x' is
+// the bf16 pattern just below or at x'.  Patterns <= g-2 are more than one bf16 step (2^-8)
+// below x, so their product with n rounds below l; patterns >= g+2 are above x.  Alo = g-2 and
+// Ahi = g+2 keep an extra step in hand.  The window is refused (false) where products could be
+// subnormal (lo < 2^24) or overflow, and columns whose norm is outside [2^-100, 2^100] get
+// thresholds that make every weight a candidate (norm 0: every finite weight scores 0).
+template <int V>
+__device__ __forceinline__ bool window_thresholds(uint32_t center, int w, const float* __restrict__ norms, int cols, int nt,
+                                                  uint32_t (&Alo)[V][4], uint32_t (&Ahi)[V][4], uint32_t* lo_out) {
+    const int tid = threadIdx.x;
+    const uint32_t half = 1u << (w - 1);
+    if (center < (1u << 24) + half) return false;
+    const uint32_t lo = center - half;
+    if (lo > 0x7F7FFFFFu - (1u << w)) return false;
+    const float flo = __uint_as_float(lo), fhi = __uint_as_float(lo + (1u << w));
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t al[2], ah[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = (v * nt + tid) * kVec + 2 * i + h;
+                al[h] = 0u;   // past the end of the row: never below, never a candidate
+                ah[h] = 0u;
+                if (c < cols) {
+                    const float n = __ldg(norms + c);
+                    if (n == 0.0f) {
+                        al[h] = 0x7F80u;
+                        ah[h] = 0x7F82u;
+                    } else if (!(n >= 0x1p-100f && n <= 0x1p100f)) {
+                        al[h] = 0u;
+                        ah[h] = 0x8000u;
+                    } else {
+                        const float r = rcp_approx(n);
+                        const uint32_t gl = __float_as_uint(__fmul_rn(flo, r)) >> 16;
+                        const uint32_t gh = __float_as_uint(__fmul_rn(fhi, r)) >> 16;
+                        al[h] = gl > 2u ? gl - 2u : 0u;
+                        ah[h] = gh + 2u;
+                    }
+                }
+            }
+            Alo[v][i] = al[0] | (al[1] << 16);
+            Ahi[v][i] = ah[0] | (ah[1] << 16);
+        }
+    *lo_out = lo;
+    return true;
+}
+
+// True iff every norm of this thread's columns is finite and >= 0: the bf16-domain classification
+// needs scores that are monotone in |w| for every column.
+template <int V>
+__device__ __forceinline__ bool norms_usable(const float* __restrict__ norms, int cols, int nt) {
+    bool fin = true;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) {
+            const int c = (v * nt + (int)threadIdx.x) * kVec + e;
+            if (c < cols) {
+                const float n = __ldg(norms + c);
+                fin = fin && (n >= 0.0f) && (n <= 3.402823466e38f);
+            }
+        }
+    return fin;
+}
+
+// The candidate flags of the thread's four vectors share one word: vector v's flags move down by
+// 4v bits (its eight flags sit on bits 12..15 and 28..31), so one loop over the set bits visits
+// all candidates of the thread and lanes with few candidates in one vector do not wait for lanes
+// with many in another.
+__device__ __forceinline__ uint32_t pack_flags4(const uint32_t (&f)[4]) {
+    return f[0] | (f[1] >> 4) | (f[2] >> 8) | (f[3] >> 12);
+}
+__device__ __forceinline__ int packed_vec(int b) { return 3 - ((b & 15) >> 2); }   // bit of the packed word -> vector
+
 // The slow, always-exact treatment of one row held in shared memory: full radix select, ordered
 // ties, store.  Returns the row's threshold key.  hist[0..kBins1) must be zero; it is zero after.
 template <int V>
@@ -353,13 +461,11 @@ __device__ __noinline__ uint32_t generic_row_bf16(const uint4* my_vecs, int nt, 
     return T;
 }
 
-// cols % 8 == 0, 0 < k < cols, blockDim.x = nt a multiple of 32 with kFastV*nt*8 >= cols and nt <= cols/8;
-// dynamic shared memory: 2 * kFastV * nt * 16 bytes.
-template <int MAXNT, int MINB>
-__global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint16_t* W_in, uint16_t* W_out, int64_t rows,
-                                                                       int cols, int64_t ldw,
-                                                                       const float* __restrict__ norms, int k,
-                                                                       uint8_t* __restrict__ mask_bytes, int mask_row_bytes) {
+// Every job: cols % 8 == 0, 0 < k < cols.  blockDim.x = nt, a multiple of 32 with kFastV*nt*8 >= cols and
+// nt <= cols/8; dynamic shared memory: 2 * kFastV * nt * 16 bytes.  total_rows = sum of the jobs' rows.
+template <int MAXNT, int MINB, int NJ>
+__global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __grid_constant__ PruneJobList<NJ> jobs,
+                                                                       int64_t total_rows, int cols) {
     constexpr int V = kFastV;
     extern __shared__ __align__(16) uint4 rowbuf[];      // [2][V][nt]: the row being selected and the next one
     __shared__ __align__(16) uint32_t buf[kBins1];       // window histogram + one key per bin, or the full select's histogram
@@ -375,7 +481,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
 
     const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = nt >> 5;
     const int nvec = cols >> 3;
-    const uint32_t uk = (uint32_t)k;
     uint32_t* hist = buf;
     uint32_t* slot = buf + kWinBins;
 
@@ -383,29 +488,29 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
     if (tid < 32) coarse[tid] = 0u;
     if (tid < 16) spread[tid] = (uint8_t)((tid & 1) | ((tid & 2) << 1) | ((tid & 4) << 2) | ((tid & 8) << 3));
     if (tid == 0) n_list = 0u;
-    bool fin = true;
-#pragma unroll
-    for (int v = 0; v < V; ++v)
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) {
-            const int c = (v * nt + tid) * kVec + e;
-            if (c < cols) {
-                const float n = __ldg(norms + c);
-                fin = fin && (n >= 0.0f) && (n <= 3.402823466e38f);
-            }
-        }
-    // The bf16-domain classification needs scores that are monotone in |w| for every column:
-    // true for finite norms >= 0.  Otherwise every row takes the exact slow path.
-    const bool all_finite = __syncthreads_and(fin ? 1 : 0) != 0;
+    __syncthreads();
 
-    auto prefetch = [&](int slot_idx, int64_t row) {
-        const uint16_t* src = W_in + row * ldw;
+    // ---- the job the CTA is in (set when a row crosses into it)
+    uint16_t* W_out = nullptr;
+    const float* norms = nullptr;
+    uint8_t* mask_bytes = nullptr;
+    int64_t ldw = 0, row0 = 0, job_end = 0;
+    int mask_row_bytes = 0;
+    uint32_t uk = 0u;
+    bool all_finite = false;
+
+    auto prefetch = [&](int slot_idx, const uint16_t* src) {
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int vec = v * nt + tid;
             if (vec < nvec) cp_async16(&rowbuf[(slot_idx * V + v) * nt + tid], src + (int64_t)vec * kVec);
         }
         cp_async_commit();
+    };
+    // Address of global row r; jj is a cursor into the job list that only moves forward.
+    auto row_src = [&](int64_t r, int& jj) -> const uint16_t* {
+        while (r >= jobs.job[jj].row0 + jobs.job[jj].rows) ++jj;
+        return jobs.job[jj].W_in + (r - jobs.job[jj].row0) * jobs.job[jj].ldw;
     };
 
     // ---- window state: [win_lo, win_lo + 2^win_w) and the thread's per-column thresholds
@@ -414,55 +519,9 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
     int win_w = 0;
     bool win_valid = false;
 
-    // Thresholds of the window of width 2^w centred on `center`.  For column j with norm n:
-    //   magnitude bits a <  Alo  =>  score key < lo      (surely pruned once T >= lo)
-    //   magnitude bits a >= Ahi  =>  score key >= hi     (surely kept once T < hi)
-    // With x = l/n, the estimate x' = l * rcp(n) is within 2^-22 of x and g = top 16 bits of x' is
-    // the bf16 pattern just below or at x'.  Patterns <= g-2 are more than one bf16 step (2^-8)
-    // below x, so their product with n rounds below l; patterns >= g+2 are above x.  Alo = g-2 and
-    // Ahi = g+2 keep an extra step in hand.  The window is refused where products could be
-    // subnormal (lo < 2^24) or overflow, and columns whose norm is outside [2^-100, 2^100] get
-    // thresholds that make every weight a candidate (norm 0: every finite weight scores 0).
     auto set_window = [&](uint32_t center, int w) {
-        const uint32_t half = 1u << (w - 1);
-        win_valid = false;
-        if (center < (1u << 24) + half) return;
-        const uint32_t lo = center - half;
-        if (lo > 0x7F7FFFFFu - (1u << w)) return;
-        const float flo = __uint_as_float(lo), fhi = __uint_as_float(lo + (1u << w));
-#pragma unroll
-        for (int v = 0; v < V; ++v)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t al[2], ah[2];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int c = (v * nt + tid) * kVec + 2 * i + h;
-                    al[h] = 0u;   // past the end of the row: never below, never a candidate
-                    ah[h] = 0u;
-                    if (c < cols) {
-                        const float n = __ldg(norms + c);
-                        if (n == 0.0f) {
-                            al[h] = 0x7F80u;
-                            ah[h] = 0x7F82u;
-                        } else if (!(n >= 0x1p-100f && n <= 0x1p100f)) {
-                            al[h] = 0u;
-                            ah[h] = 0x8000u;
-                        } else {
-                            const float r = rcp_approx(n);
-                            const uint32_t gl = __float_as_uint(__fmul_rn(flo, r)) >> 16;
-                            const uint32_t gh = __float_as_uint(__fmul_rn(fhi, r)) >> 16;
-                            al[h] = gl > 2u ? gl - 2u : 0u;
-                            ah[h] = gh + 2u;
-                        }
-                    }
-                }
-                Alo[v][i] = al[0] | (al[1] << 16);
-                Ahi[v][i] = ah[0] | (ah[1] << 16);
-            }
-        win_lo = lo;
+        win_valid = window_thresholds<V>(center, w, norms, cols, nt, Alo, Ahi, &win_lo);
         win_w = w;
-        win_valid = true;
     };
 
     // Exact score key of element e of the thread's vector v of the row in buffer `cur`.
@@ -507,22 +566,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
             below += 8u - (uint32_t)__popc(keepf[v]);
         }
         // exact scores of the candidates: below lo, or into the window histogram
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            uint32_t c = cand[v];
-            while (c) {
-                const int b = __ffs(c) - 1;
-                c &= c - 1u;
-                const uint32_t key = cand_key(cur, v, flag_elem(b));
-                const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
-                if (d < width) {
-                    const uint32_t bin = d >> shift;
-                    atomicAdd(&hist[bin], 1u);
-                    atomicAdd(&coarse[bin >> 5], 1u);
-                    slot[bin] = key;
-                } else {
-                    below += d >> 31;
-                }
+        const uint32_t cand_all = pack_flags4(cand);
+        for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
+            const int b = __ffs(c) - 1;
+            const int v = packed_vec(b);
+            const uint32_t key = cand_key(cur, v, flag_elem(b + 4 * v));
+            const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
+            if (d < width) {
+                const uint32_t bin = d >> shift;
+                atomicAdd(&hist[bin], 1u);
+                atomicAdd(&coarse[bin >> 5], 1u);
+                slot[bin] = key;
+            } else {
+                below += d >> 31;
             }
         }
         below = __reduce_add_sync(0xFFFFFFFFu, below);
@@ -583,17 +639,13 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
         if (n_bin > 1u) {
             if (n_bin > (uint32_t)kBinListCap) return 2;
             // collect the keys of that bin; warp 0 ranks them
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                uint32_t c = cand[v];
-                while (c) {
-                    const int b = __ffs(c) - 1;
-                    c &= c - 1u;
-                    const uint32_t key = cand_key(cur, v, flag_elem(b));
-                    if (((key - lo) >> shift) == bin) {
-                        const uint32_t pos = atomicAdd(&n_list, 1u);
-                        if (pos < (uint32_t)kBinListCap) list[pos] = key;
-                    }
+            for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
+                const int b = __ffs(c) - 1;
+                const int v = packed_vec(b);
+                const uint32_t key = cand_key(cur, v, flag_elem(b + 4 * v));
+                if (((key - lo) >> shift) == bin) {
+                    const uint32_t pos = atomicAdd(&n_list, 1u);
+                    if (pos < (uint32_t)kBinListCap) list[pos] = key;
                 }
             }
             __syncthreads();
@@ -615,20 +667,20 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
         // prune: surely below lo, or a candidate whose exact key is <= T
         const uint32_t thr = T + 1u;
         uint16_t* out_row = W_out + row * ldw;
+        uint32_t gone_all = 0u;
+        for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
+            const int b = __ffs(c) - 1;
+            const int v = packed_vec(b);
+            const int e = flag_elem(b + 4 * v);
+            if (cand_key(cur, v, e) < thr) {
+                gone_all |= 1u << b;
+                sts_u16_zero(reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + tid]) + e);
+            }
+        }
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int vec = v * nt + tid;
-            uint32_t c = cand[v], gone = 0u;
-            uint16_t* mine = reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + tid]);
-            while (c) {
-                const int b = __ffs(c) - 1;
-                c &= c - 1u;
-                const int e = flag_elem(b);
-                if (cand_key(cur, v, e) < thr) {
-                    gone |= 1u << b;
-                    sts_u16_zero(mine + e);
-                }
-            }
+            const uint32_t gone = (gone_all << (4 * v)) & 0xF000F000u;
             if (vec < nvec) {
                 const uint4 r = rowbuf[(cur * V + v) * nt + tid];
                 uint4 o;
@@ -652,13 +704,42 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
         return 0;
     };
 
-    int cur = 0;
-    int64_t row = blockIdx.x;
-    if (row < rows) prefetch(0, row);
-    for (; row < rows; row += gridDim.x, cur ^= 1) {
-        if (row + gridDim.x < rows) prefetch(cur ^ 1, row + gridDim.x);
+    int cur = 0, j_next = 0, j_cur = 0;
+    int64_t r = blockIdx.x;
+    if (r < total_rows) prefetch(0, row_src(r, j_next));
+    for (; r < total_rows; r += gridDim.x, cur ^= 1) {
+        if (r + gridDim.x < total_rows) prefetch(cur ^ 1, row_src(r + gridDim.x, j_next));
         else cp_async_commit();
         cp_async_wait_all_but_one();   // this row has landed; a thread only ever reads the vectors it copied itself
+
+        if (r >= job_end) {   // the row belongs to the next job: pick up its parameters and its plan
+            while (r >= jobs.job[j_cur].row0 + jobs.job[j_cur].rows) ++j_cur;
+            const PruneJob& J = jobs.job[j_cur];
+            W_out = J.W_out;
+            norms = J.norms;
+            mask_bytes = J.mask;
+            ldw = J.ldw;
+            row0 = J.row0;
+            job_end = J.row0 + J.rows;
+            mask_row_bytes = J.mask_row_bytes;
+            uk = (uint32_t)J.k;
+            all_finite = __syncthreads_and(norms_usable<V>(norms, cols, nt) ? 1 : 0) != 0;
+            win_valid = false;
+            const uint32_t* plan = J.plan;
+            if (all_finite && plan != nullptr && plan[0] != 0u) {
+                win_lo = plan[1];
+                win_w = (int)plan[2];
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const uint4* p = reinterpret_cast<const uint4*>(plan + kPlanHeader + (size_t)(v * nt + tid) * 8);
+                    const uint4 a = p[0], b = p[1];
+                    Alo[v][0] = a.x; Alo[v][1] = a.y; Alo[v][2] = a.z; Alo[v][3] = a.w;
+                    Ahi[v][0] = b.x; Ahi[v][1] = b.y; Ahi[v][2] = b.z; Ahi[v][3] = b.w;
+                }
+                win_valid = true;
+            }
+        }
+        const int64_t row = r - row0;   // row inside the job
 
         MOSAIC_STAT(0);
         int status = 1;
@@ -685,31 +766,112 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const uint
     }
 }
 
-template <int MAXNT, int MINB>
-static int launch_prune_bf16(const void* W_in, void* W_out, int64_t rows, int cols, int64_t ldw, const float* norms, int k,
-                             uint32_t* mask, int nt, cudaStream_t st) {
+// One CTA per job: the exact thresholds of three rows (first, middle, last) by the full radix
+// select, a window of width 2^kTrackBits centred on their median, and the per-column thresholds
+// of that window in the layout the pruning kernel loads (same nt).
+template <int MAXNT, int NJ>
+__global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_constant__ PruneJobList<NJ> jobs, int cols) {
+    constexpr int V = kFastV;
+    __shared__ __align__(16) uint32_t hist[kBins1];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ SelectResult sel3;
+    const int nt = blockDim.x, tid = threadIdx.x;
+    const int nvec = cols >> 3;
+    const PruneJob& J = jobs.job[blockIdx.x];
+    uint32_t* plan = J.plan;
+    if (plan == nullptr) return;
+    for (int b = tid; b < kBins1; b += nt) hist[b] = 0u;
+    const bool usable = __syncthreads_and(norms_usable<V>(J.norms, cols, nt) ? 1 : 0) != 0;
+    bool valid = usable;
+    uint32_t Alo[V][4], Ahi[V][4], lo = 0u;
+    if (usable) {
+        float nrm[V][kVec];
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) {
+                const int c = (v * nt + tid) * kVec + e;
+                nrm[v][e] = (c < cols) ? __ldg(J.norms + c) : __int_as_float(0x7F800000);
+            }
+        uint32_t Ts[3];
+#pragma unroll 1
+        for (int s = 0; s < 3; ++s) {
+            const int64_t row = (s == 0) ? 0 : (s == 1 ? J.rows / 2 : J.rows - 1);
+            Raw8<MOSAIC_BF16> raw[V];
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int vec = v * nt + tid;
+                if (vec < nvec) raw[v].template load<true>(J.W_in + row * J.ldw + (int64_t)vec * kVec);
+                else raw[v].clear();
+            }
+            auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))); };
+            uint32_t q, n_eq;
+            radix_select_row<V>(key_of, (uint32_t)J.k, hist, warp_tot, &sel3, nt, &Ts[s], &q, &n_eq);
+        }
+        const uint32_t mx = max(max(Ts[0], Ts[1]), Ts[2]), mn = min(min(Ts[0], Ts[1]), Ts[2]);
+        const uint32_t median = (uint32_t)((uint64_t)Ts[0] + Ts[1] + Ts[2] - mx - mn);
+        valid = window_thresholds<V>(median, kTrackBits, J.norms, cols, nt, Alo, Ahi, &lo);
+    }
+    if (valid) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            uint4* p = reinterpret_cast<uint4*>(plan + kPlanHeader + (size_t)(v * nt + tid) * 8);
+            p[0] = make_uint4(Alo[v][0], Alo[v][1], Alo[v][2], Alo[v][3]);
+            p[1] = make_uint4(Ahi[v][0], Ahi[v][1], Ahi[v][2], Ahi[v][3]);
+        }
+    }
+    if (tid == 0) {
+        plan[0] = valid ? 1u : 0u;
+        plan[1] = lo;
+        plan[2] = (uint32_t)kTrackBits;
+        plan[3] = 0u;
+    }
+}
+
+// Launches the pruning kernel (and, with_plan, the planning kernel before it) over a list of jobs.
+template <int MAXNT, int MINB, int NJ>
+static int launch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int nt, bool with_plan,
+                             cudaStream_t st) {
     static int blocks_per_sm[MAXNT / 32 + 1] = {0};
     const size_t dyn = (size_t)2 * kFastV * nt * sizeof(uint4);
     int& bps = blocks_per_sm[nt / 32];
     if (bps == 0) {
-        if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB, NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)((size_t)2 * kFastV * MAXNT * sizeof(uint4))) != cudaSuccess)
             return MOSAIC_ERR_CUDA;
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB>, nt, dyn) != cudaSuccess || n < 1) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB, NJ>, nt, dyn) != cudaSuccess ||
+            n < 1) {
             (void)cudaGetLastError();
             n = 1;
         }
         bps = n > MOSAIC_FAST_MAX_CTAS ? MOSAIC_FAST_MAX_CTAS : n;
     }
+    if (with_plan) {
+        prune_plan_kernel<MAXNT, NJ><<<(unsigned)jobs.n, nt, 0, st>>>(jobs, cols);
+        MOSAIC_LAUNCH_CHECK();
+    }
     int64_t grid = (int64_t)sm_count() * bps;
-    if (grid > rows) grid = rows;
-    const int words = (cols + 31) / 32;
-    prune_rows_bf16_kernel<MAXNT, MINB><<<(unsigned)grid, nt, dyn, st>>>(
-        static_cast<const uint16_t*>(W_in), static_cast<uint16_t*>(W_out), rows, cols, ldw, norms, k,
-        reinterpret_cast<uint8_t*>(mask), words * 4);
+    if (grid > total_rows) grid = total_rows;
+    prune_rows_bf16_kernel<MAXNT, MINB, NJ><<<(unsigned)grid, nt, dyn, st>>>(jobs, total_rows, cols);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
+}
+
+template <int NJ>
+static int dispatch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int nt, bool with_plan,
+                               cudaStream_t st) {
+    if (nt <= 128) return launch_prune_bf16<128, 6, NJ>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 256) return launch_prune_bf16<256, 3, NJ>(jobs, total_rows, cols, nt, with_plan, st);
+    return launch_prune_bf16<512, 1, NJ>(jobs, total_rows, cols, nt, with_plan, st);
+}
+
+// Threads per CTA of the bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
+static int fast_threads(int dtype, int64_t cols, int64_t k) {
+    if (dtype != MOSAIC_BF16 || cols % kVec != 0 || k <= 0 || k >= cols) return 0;
+    const int64_t nvec = cols / kVec;
+    const int64_t nt = ((nvec + kFastV - 1) / kFastV + 31) / 32 * 32;
+    return (nvec >= 256 && nt <= 512) ? (int)nt : 0;
 }
 
 template <int DT, int V, int NT, int MINB>
@@ -774,11 +936,9 @@ extern "C" int mosaic_debug_prune_stats(unsigned long long* host_out, int reset)
 
 extern "C" size_t mosaic_prune_unstructured_workspace_bytes(int64_t, int64_t) { return 0; }
 
-extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t rows, int64_t cols, int64_t ldw, int dtype,
-                                         const float* norms, int64_t k, uint32_t* mask_out, void* ws, size_t ws_bytes,
-                                         void* stream) {
-    (void)ws;
-    (void)ws_bytes;
+// Argument checks of one pruning job (shared by the single and the batched entry point).
+static int validate_prune(const void* W_in, void* W_out, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                          const float* norms, int64_t k, uint32_t* mask_out) {
     int rc = check_matrix(W_in, rows, cols, ldw, dtype);
     if (rc != MOSAIC_OK) return rc;
     rc = check_matrix(W_out, rows, cols, ldw, dtype);
@@ -786,24 +946,111 @@ extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t 
     if (!norms) return MOSAIC_ERR_NULL_PTR;
     if ((reinterpret_cast<uintptr_t>(norms) & 3u) || (reinterpret_cast<uintptr_t>(mask_out) & 3u)) return MOSAIC_ERR_MISALIGNED;
     if (k < 0 || k > cols || cols > 65536) return MOSAIC_ERR_INVALID_ARG;
-    if (rows == 0) return MOSAIC_OK;
-    if (W_in != W_out) {
+    if (rows > 0 && W_in != W_out) {
         const size_t span = ((size_t)(rows - 1) * (size_t)ldw + (size_t)cols) * elem_size(dtype);
         const char *a = static_cast<const char*>(W_in), *b = static_cast<const char*>(W_out);
         if (a < b + span && b < a + span) return MOSAIC_ERR_ALIASING;
     }
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                                         const float* norms, int64_t k, uint32_t* mask_out, void* ws, size_t ws_bytes,
+                                         void* stream) {
+    (void)ws;
+    (void)ws_bytes;
+    const int rc = validate_prune(W_in, W_out, rows, cols, ldw, dtype, norms, k, mask_out);
+    if (rc != MOSAIC_OK) return rc;
+    if (rows == 0) return MOSAIC_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dtype == MOSAIC_BF16 && cols % kVec == 0 && k > 0 && k < cols) {
-        const int nvec = (int)(cols / kVec);
-        const int nt = ((nvec + kFastV - 1) / kFastV + 31) / 32 * 32;   // threads so that kFastV vectors each cover the row
-        if (nvec >= 256 && nt <= 128)
-            return launch_prune_bf16<128, 6>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
-        if (nvec >= 256 && nt <= 256)
-            return launch_prune_bf16<256, 3>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
-        if (nvec >= 256 && nt <= 512)
-            return launch_prune_bf16<512, 1>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, nt, st);
+    if (const int nt = fast_threads(dtype, cols, k)) {
+        PruneJobList<1> one;
+        one.n = 1;
+        one.job[0] = PruneJob{static_cast<const uint16_t*>(W_in), static_cast<uint16_t*>(W_out), norms,
+                              reinterpret_cast<uint8_t*>(mask_out), nullptr, rows, ldw, 0, (int)k,
+                              (int)((cols + 31) / 32) * 4};
+        return dispatch_prune_bf16<1>(one, rows, (int)cols, nt, false, st);
     }
     if (dtype == MOSAIC_BF16)
         return dispatch_prune<MOSAIC_BF16>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, st);
     return dispatch_prune<MOSAIC_F32>(W_in, W_out, rows, (int)cols, ldw, norms, (int)k, mask_out, st);
+}
+
+// Workspace of the batched call: one plan (window + per-column thresholds) per job that the bf16
+// kernel takes, 256-byte aligned, in job order.
+static size_t batch_plan_bytes(const mosaic_prune_job& j, int dtype) {
+    const int nt = (j.rows > 0) ? fast_threads(dtype, j.cols, j.k) : 0;
+    return nt ? align_up(plan_words(nt) * sizeof(uint32_t), 256) : 0;
+}
+
+extern "C" size_t mosaic_prune_unstructured_batch_workspace_bytes(const mosaic_prune_job* jobs, int64_t n_jobs, int dtype) {
+    size_t total = 256;
+    if (jobs == nullptr) return total;
+    for (int64_t i = 0; i < n_jobs; ++i) total += batch_plan_bytes(jobs[i], dtype);
+    return total;
+}
+
+extern "C" int mosaic_prune_unstructured_batch(const mosaic_prune_job* jobs, int64_t n_jobs, int dtype, void* ws,
+                                               size_t ws_bytes, void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_prune_job& j = jobs[i];
+        const int rc = validate_prune(j.W_in, j.W_out, j.rows, j.cols, j.ldw, dtype, j.norms, j.k, j.mask_out);
+        if (rc != MOSAIC_OK) return rc;
+    }
+    const size_t need = mosaic_prune_unstructured_batch_workspace_bytes(jobs, n_jobs, dtype);
+    if (need > 256) {
+        if (ws == nullptr) return MOSAIC_ERR_NULL_PTR;
+        if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
+        if (ws_bytes < need) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // jobs for the bf16 kernel are launched together, one launch (plus its planning launch) per
+    // distinct row length and per kBatchJobs jobs; everything else goes through the single call
+    std::vector<char> done((size_t)n_jobs, 0);
+    std::vector<size_t> plan_off((size_t)n_jobs, 0);
+    size_t off = 0;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        plan_off[(size_t)i] = off;
+        off += batch_plan_bytes(jobs[i], dtype);
+    }
+    static PruneJobList<kBatchJobs> list;   // host staging of the kernel parameter; calls are not re-entrant
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        if (done[(size_t)i]) continue;
+        const mosaic_prune_job& lead = jobs[i];
+        const int nt = (lead.rows > 0) ? fast_threads(dtype, lead.cols, lead.k) : 0;
+        if (nt == 0) {
+            done[(size_t)i] = 1;
+            const int rc = mosaic_prune_unstructured(lead.W_in, lead.W_out, lead.rows, lead.cols, lead.ldw, dtype, lead.norms,
+                                                     lead.k, lead.mask_out, nullptr, 0, stream);
+            if (rc != MOSAIC_OK) return rc;
+            continue;
+        }
+        list.n = 0;
+        int64_t total_rows = 0;
+        for (int64_t m = i; m < n_jobs; ++m) {
+            const mosaic_prune_job& j = jobs[m];
+            if (done[(size_t)m] || j.cols != lead.cols || j.rows <= 0 || fast_threads(dtype, j.cols, j.k) == 0) continue;
+            done[(size_t)m] = 1;
+            list.job[list.n] = PruneJob{static_cast<const uint16_t*>(j.W_in), static_cast<uint16_t*>(j.W_out), j.norms,
+                                        reinterpret_cast<uint8_t*>(j.mask_out),
+                                        reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + plan_off[(size_t)m]), j.rows,
+                                        j.ldw, total_rows, (int)j.k, (int)((j.cols + 31) / 32) * 4};
+            total_rows += j.rows;
+            if (++list.n == kBatchJobs || m == n_jobs - 1) {
+                const int rc = dispatch_prune_bf16<kBatchJobs>(list, total_rows, (int)lead.cols, nt, true, st);
+                if (rc != MOSAIC_OK) return rc;
+                list.n = 0;
+                total_rows = 0;
+            }
+        }
+        if (list.n > 0) {
+            const int rc = dispatch_prune_bf16<kBatchJobs>(list, total_rows, (int)lead.cols, nt, true, st);
+            if (rc != MOSAIC_OK) return rc;
+        }
+    }
+    return MOSAIC_OK;
 }

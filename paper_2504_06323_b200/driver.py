@@ -81,6 +81,7 @@ class ModelState:
     norms: dict = field(default_factory=dict)          # (layer, x_key) -> fp32 norms
     counts: torch.Tensor | None = None                 # int64 [len(layers)*M]
     ws: api.Workspace | None = None
+    ws_batch: api.Workspace | None = None             # holds the plans of the batched pruning call
 
     def q_local(self, layer: int, proj: str) -> int:
         return self.layers.index(layer) * len(PROJECTIONS) + PROJECTIONS.index(proj)
@@ -145,6 +146,24 @@ def prune_unstructured_layer(st: ModelState, layer: int, k_global: list[int], in
         api.mosaic_prune_unstructured(W, out, st.norms[layer, cfg.x_key(pr)], int(k_global[layer * M + m]),
                                       st.mask.get((layer, pr)), st.ws)
     return M
+
+
+def prune_unstructured_all(st: ModelState, k_global: list[int], in_place: bool = False) -> int:
+    """Phase B for every owned projection through the batched call: one planning launch and one
+    pruning launch per distinct row length instead of one launch per projection.  Returns the
+    number of jobs."""
+    cfg = st.cfg
+    M = len(PROJECTIONS)
+    jobs = []
+    for layer in st.layers:
+        for m, pr in enumerate(PROJECTIONS):
+            W = st.W[layer, pr]
+            jobs.append((W, W if in_place else st.W_out[layer, pr], st.norms[layer, cfg.x_key(pr)],
+                         int(k_global[layer * M + m]), st.mask.get((layer, pr))))
+    if getattr(st, "ws_batch", None) is None:
+        st.ws_batch = api.Workspace(st.device)
+    api.mosaic_prune_unstructured_batch(jobs, st.ws_batch)
+    return len(jobs)
 
 
 def _scores(W, norms, row_group, col_group, out, accumulate, ws):

@@ -77,6 +77,16 @@ def test_unstructured_model(name, kw):
                 if (layer, pr) in prev:
                     assert ((m & ~prev[layer, pr]) == 0).all()  # masks nested across the sweep
                 prev[layer, pr] = m
+        # the batched call over all projections must give the same bits
+        for key in st.W_out:
+            st.W_out[key].fill_(3.0)
+            st.mask[key].fill_(-1)
+        driver.prune_unstructured_all(st, k)
+        for layer in st.layers:
+            ref = op.unstructured(cfg, Wh, norms_ref, layer, k_ref)
+            for pr in PROJECTIONS:
+                assert bits_equal(wl.to_numpy(st.W_out[layer, pr]), ref[pr][0]), (layer, pr)
+                assert bits_equal(st.mask[layer, pr].cpu().numpy().view(np.uint32), ref[pr][1]), (layer, pr)
 
 
 @pytest.mark.parametrize("name,kw", [("tiny", None), ("llama3_8b", dict(hidden=640, n_heads=10, n_kv_heads=5, head_dim=64, intermediate=1728))])
@@ -139,3 +149,31 @@ def test_full_size_rows_sampled_against_oracle():
         ref = oracle.outlier_ratio(wl.to_numpy(W), nh, cfg.alpha, "bf16")     # whole matrix: a second or two
         assert ref["certified"] and cnt.item() == ref["count"]
         np.testing.assert_allclose(ssum.item(), ref["sum"], rtol=1e-12)
+
+
+def test_full_size_batched_model_pass_sampled_against_oracle():
+    # two full LLaMA-7B-shaped layers through the batched call, as the benchmark launches it:
+    # sampled rows of every projection against the oracle, exact per-row sparsity everywhere
+    cfg = wl.scaled(wl.CONFIGS["llama7b"], n_layers=2)
+    st = driver.alloc_model(cfg, DEV)
+    g = torch.Generator(device="cpu").manual_seed(5)
+    for layer in st.layers:
+        for xk in cfg.x_keys():
+            c = cfg.x_cols(xk)
+            n = (torch.rand(c, generator=g) * 500 + 100)
+            n[wl.outlier_columns(cfg, layer, xk, c, cfg.x_outlier_frac)] *= 100
+            st.norms[layer, xk].copy_(n)
+    M = len(PROJECTIONS)
+    k = [int(cfg.shape(pr)[1] * (0.42 + 0.02 * ((l * M + m) % 9))) for l in st.layers for m, pr in enumerate(PROJECTIONS)]
+    driver.prune_unstructured_all(st, k)
+    for layer in st.layers:
+        for m, pr in enumerate(PROJECTIONS):
+            rows, cols = cfg.shape(pr)
+            kk = k[layer * M + m]
+            sample = torch.randperm(rows, generator=g)[:24].sort().values.to(DEV)
+            nh = st.norms[layer, cfg.x_key(pr)].cpu().numpy()
+            ref_W, ref_mask = oracle.prune_unstructured(wl.to_numpy(st.W[layer, pr][sample]), nh, kk, "bf16")
+            assert bits_equal(wl.to_numpy(st.W_out[layer, pr][sample]), ref_W), (layer, pr)
+            assert bits_equal(st.mask[layer, pr][sample].cpu().numpy().view(np.uint32), ref_mask), (layer, pr)
+            kept = st.mask[layer, pr].cpu().numpy().view(np.uint8)
+            assert (np.unpackbits(kept, axis=1).sum(1) == cols - kk).all(), (layer, pr)

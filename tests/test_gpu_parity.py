@@ -268,6 +268,30 @@ def test_prune_already_pruned_matrix():
         _check_prune(half, norms, k, "bf16")
 
 
+@pytest.mark.parametrize("dtype", ["bf16", "f32"])
+def test_prune_batch_matches_oracle_job_by_job(dtype):
+    # several projections of different shapes in one call: rows long enough for the bf16-domain
+    # kernel (planned from three sample rows), short ones, k = 0 and k = cols, one job in place
+    shapes = [(700, 4096, 2048), (300, 4096, 400), (260, 11008, 5504), (50, 688, 300), (40, 4096, 0), (33, 4096, 4096),
+              (500, 4096, 3000), (128, 5120, 2560), (1, 4096, 2048)]
+    jobs, refs = [], []
+    for i, (rows, cols, k) in enumerate(shapes):
+        W = make(rows, cols, dtype, seed=500 + i, heavy=(i % 2 == 0))
+        if i == 6:
+            W = (W.float() * torch.exp2(torch.arange(rows, device=DEV).remainder(9).float() - 4.0)[:, None]).to(W.dtype)
+        norms = norms_for(cols, 40 + i)
+        ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, dtype)
+        out = W if i == 3 else torch.full_like(W, 7.0)
+        mask = None if i == 1 else torch.full((rows, (cols + 31) // 32), -1, dtype=torch.int32, device=DEV)
+        jobs.append((W, out, norms, k, mask))
+        refs.append((ref_W, ref_mask))
+    api.mosaic_prune_unstructured_batch(jobs)
+    for (W, out, norms, k, mask), (ref_W, ref_mask) in zip(jobs, refs):
+        assert_bits_equal(host(out), ref_W)
+        if mask is not None:
+            assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+
+
 # ------------------------------------------------------------------ structured
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("rows,cols,rg,cg,fr,fc", [(256, 688, 1, 1, 0.3, 0.3), (512, 1024, 64, 1, 0.25, 0.5),
