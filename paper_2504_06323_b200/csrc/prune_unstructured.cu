@@ -39,6 +39,12 @@
 #ifndef MOSAIC_PRUNE_MINB_2X256
 #define MOSAIC_PRUNE_MINB_2X256 3
 #endif
+#ifndef MOSAIC_RING_SMALL
+#define MOSAIC_RING_SMALL 3
+#endif
+#ifndef MOSAIC_MINB_SMALL
+#define MOSAIC_MINB_SMALL 4
+#endif
 #ifndef MOSAIC_FAST_MAX_CTAS
 #define MOSAIC_FAST_MAX_CTAS 8
 #endif
@@ -287,6 +293,7 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
 // ---------------------------------------------------------------------------------------------
 constexpr int kFastV = 4;          // vectors (of 8 columns) per thread
 constexpr int kWinBins = 1024;     // histogram over the top 10 bits of a window
+constexpr int kQueueCap = 448;     // candidates a warp can queue (of its 1024 weights)
 constexpr int kBinListCap = 512;   // keys of one histogram bin that warp 0 will rank; also the sample size limit
 
 __device__ __forceinline__ float rcp_approx(float x) {   // relative error <= 2^-23 for normal x
@@ -299,7 +306,8 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
                  : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all_but_one() { asm volatile("cp.async.wait_group 1;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 __device__ __forceinline__ void sts_u16_zero(void* smem) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "h"((unsigned short)0) : "memory");
 }
@@ -462,12 +470,13 @@ __device__ __noinline__ uint32_t generic_row_bf16(const uint4* my_vecs, int nt, 
 }
 
 // Every job: cols % 8 == 0, 0 < k < cols.  blockDim.x = nt, a multiple of 32 with kFastV*nt*8 >= cols and
-// nt <= cols/8; dynamic shared memory: 2 * kFastV * nt * 16 bytes.  total_rows = sum of the jobs' rows.
-template <int MAXNT, int MINB, int NJ>
+// nt <= cols/8; dynamic shared memory: fast_dyn_smem(nt, RING).  total_rows = sum of the jobs' rows.  RING rows of the
+// CTA are resident in shared memory: the one being selected and RING-1 in flight from HBM.
+template <int MAXNT, int MINB, int NJ, int RING>
 __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __grid_constant__ PruneJobList<NJ> jobs,
                                                                        int64_t total_rows, int cols) {
     constexpr int V = kFastV;
-    extern __shared__ __align__(16) uint4 rowbuf[];      // [2][V][nt]: the row being selected and the next one
+    extern __shared__ __align__(16) uint4 rowbuf[];      // [RING][V][nt] row ring; then the queues
     __shared__ __align__(16) uint32_t buf[kBins1];       // window histogram + one key per bin, or the full select's histogram
     __shared__ __align__(16) uint32_t whist[256];        // warp 0's digit histogram
     __shared__ uint32_t coarse[32];                      // window histogram summed over groups of 32 bins
@@ -483,7 +492,16 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
     const int nvec = cols >> 3;
     uint32_t* hist = buf;
     uint32_t* slot = buf + kWinBins;
+    // Per warp: a queue of its candidates (who holds the weight, and its exact key), so that the
+    // candidates of the warp are worked on 32 at a time whatever their spread over the lanes;
+    // and per thread a word that collects which of its candidates end up pruned.
+    uint32_t* qkey = reinterpret_cast<uint32_t*>(rowbuf + RING * V * nt) + wid * kQueueCap;
+    uint32_t* gone_w = reinterpret_cast<uint32_t*>(rowbuf + RING * V * nt) + nwarps * kQueueCap;
+    uint16_t* qid = reinterpret_cast<uint16_t*>(gone_w + nt) + wid * kQueueCap;
+    __shared__ uint32_t q_overflow;
 
+    gone_w[tid] = 0u;
+    if (tid == 0) q_overflow = 0u;
     for (int b = tid; b < kBins1; b += nt) buf[b] = 0u;
     if (tid < 32) coarse[tid] = 0u;
     if (tid < 16) spread[tid] = (uint8_t)((tid & 1) | ((tid & 2) << 1) | ((tid & 4) << 2) | ((tid & 8) << 3));
@@ -565,12 +583,36 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
             cand[v] = keepf[v] & ~above;
             below += 8u - (uint32_t)__popc(keepf[v]);
         }
-        // exact scores of the candidates: below lo, or into the window histogram
+        // queue the warp's candidates: entry = (lane that holds the weight) << 5 | packed flag bit
         const uint32_t cand_all = pack_flags4(cand);
-        for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
-            const int b = __ffs(c) - 1;
-            const int v = packed_vec(b);
-            const uint32_t key = cand_key(cur, v, flag_elem(b + 4 * v));
+        uint32_t q_n;
+        {
+            const uint32_t mine = (uint32_t)__popc(cand_all);
+            uint32_t incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                if (lane >= o) incl += n;
+            }
+            q_n = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (q_n > (uint32_t)kQueueCap) {
+                if (lane == 0) q_overflow = 1u;   // the whole CTA gives the row to the slow path (after the barrier)
+                q_n = 0u;
+            } else {
+                uint32_t off = incl - mine;
+                for (uint32_t c = cand_all; c != 0u; c &= c - 1u) qid[off++] = (uint16_t)((lane << 5) | (__ffs(c) - 1));
+            }
+            __syncwarp();
+        }
+        // exact scores of the candidates, 32 at a time: below lo, or into the window histogram
+        for (uint32_t i = lane; i < q_n; i += 32) {
+            const uint32_t id = qid[i];
+            const int b = id & 31, v = packed_vec(b), e = flag_elem(b + 4 * v);
+            const int owner = (wid << 5) | (int)(id >> 5);
+            const uint16_t* p = reinterpret_cast<const uint16_t*>(&rowbuf[(cur * V + v) * nt + owner]);
+            const uint32_t a = ((uint32_t)p[e] & 0x7FFFu) << 16;
+            const uint32_t key = __float_as_uint(__fmul_rn(__ldg(norms + (v * nt + owner) * kVec + e), __uint_as_float(a)));
+            qkey[i] = key;
             const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
             if (d < width) {
                 const uint32_t bin = d >> shift;
@@ -628,10 +670,13 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 sel.q = r_bin;       // rank inside the bin
                 sel.n_eq = n_bin;    // keys in the bin
                 sel.T = slot[bin];   // the key itself if it is alone in its bin
+                sel.lo = q_overflow;  // some warp had more candidates than its queue holds
+                q_overflow = 0u;
                 n_list = 0u;
             }
         }
         __syncthreads();
+        if (sel.lo != 0u) return 2;
         if (sel.ok == 0u) return 1;
         const uint32_t bin = sel.bin, r_bin = sel.q, n_bin = sel.n_eq;
         uint32_t T = sel.T;
@@ -639,10 +684,8 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         if (n_bin > 1u) {
             if (n_bin > (uint32_t)kBinListCap) return 2;
             // collect the keys of that bin; warp 0 ranks them
-            for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
-                const int b = __ffs(c) - 1;
-                const int v = packed_vec(b);
-                const uint32_t key = cand_key(cur, v, flag_elem(b + 4 * v));
+            for (uint32_t i = lane; i < q_n; i += 32) {
+                const uint32_t key = qkey[i];
                 if (((key - lo) >> shift) == bin) {
                     const uint32_t pos = atomicAdd(&n_list, 1u);
                     if (pos < (uint32_t)kBinListCap) list[pos] = key;
@@ -667,16 +710,18 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         // prune: surely below lo, or a candidate whose exact key is <= T
         const uint32_t thr = T + 1u;
         uint16_t* out_row = W_out + row * ldw;
-        uint32_t gone_all = 0u;
-        for (uint32_t c = cand_all; c != 0u; c &= c - 1u) {
-            const int b = __ffs(c) - 1;
-            const int v = packed_vec(b);
-            const int e = flag_elem(b + 4 * v);
-            if (cand_key(cur, v, e) < thr) {
-                gone_all |= 1u << b;
-                sts_u16_zero(reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + tid]) + e);
+        for (uint32_t i = lane; i < q_n; i += 32) {
+            if (qkey[i] < thr) {
+                const uint32_t id = qid[i];
+                const int b = id & 31, v = packed_vec(b), e = flag_elem(b + 4 * v);
+                const int owner = (wid << 5) | (int)(id >> 5);
+                sts_u16_zero(reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + owner]) + e);
+                atomicOr(&gone_w[owner], 1u << b);
             }
         }
+        __syncwarp();
+        const uint32_t gone_all = gone_w[tid];
+        gone_w[tid] = 0u;
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int vec = v * nt + tid;
@@ -704,13 +749,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         return 0;
     };
 
-    int cur = 0, j_next = 0, j_cur = 0;
+    int cur = 0, nxt = RING - 1, j_next = 0, j_cur = 0;
     int64_t r = blockIdx.x;
-    if (r < total_rows) prefetch(0, row_src(r, j_next));
-    for (; r < total_rows; r += gridDim.x, cur ^= 1) {
-        if (r + gridDim.x < total_rows) prefetch(cur ^ 1, row_src(r + gridDim.x, j_next));
+#pragma unroll
+    for (int d = 0; d < RING - 1; ++d) {   // fill the ring: rows r, r+grid, ... (one copy group each, possibly empty)
+        if (r + d * (int64_t)gridDim.x < total_rows) prefetch(d, row_src(r + d * (int64_t)gridDim.x, j_next));
         else cp_async_commit();
-        cp_async_wait_all_but_one();   // this row has landed; a thread only ever reads the vectors it copied itself
+    }
+    for (; r < total_rows; r += gridDim.x, cur = (cur + 1 == RING ? 0 : cur + 1), nxt = (nxt + 1 == RING ? 0 : nxt + 1)) {
+        const int64_t r_far = r + (RING - 1) * (int64_t)gridDim.x;
+        if (r_far < total_rows) prefetch(nxt, row_src(r_far, j_next));
+        else cp_async_commit();
+        cp_async_wait_all_but<RING - 1>();   // this row has landed (the RING-1 younger groups may still be in flight)
+        __syncwarp();                        // ... for every lane of the warp: lanes read each other's vectors
 
         if (r >= job_end) {   // the row belongs to the next job: pick up its parameters and its plan
             while (r >= jobs.job[j_cur].row0 + jobs.job[j_cur].rows) ++j_cur;
@@ -723,10 +774,11 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
             job_end = J.row0 + J.rows;
             mask_row_bytes = J.mask_row_bytes;
             uk = (uint32_t)J.k;
-            all_finite = __syncthreads_and(norms_usable<V>(norms, cols, nt) ? 1 : 0) != 0;
             win_valid = false;
             const uint32_t* plan = J.plan;
-            if (all_finite && plan != nullptr && plan[0] != 0u) {
+            const bool planned = plan != nullptr && plan[0] != 0u;   // a valid plan vouches for the norms
+            all_finite = planned || __syncthreads_and(norms_usable<V>(norms, cols, nt) ? 1 : 0) != 0;
+            if (planned) {
                 win_lo = plan[1];
                 win_w = (int)plan[2];
 #pragma unroll
@@ -828,19 +880,24 @@ __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_const
     }
 }
 
+// Row ring (`ring` rows of kFastV*nt vectors), per-warp queues (key + id per entry), one word per thread.
+static size_t fast_dyn_smem(int nt, int ring) {
+    return (size_t)ring * kFastV * nt * sizeof(uint4) + (size_t)(nt / 32) * kQueueCap * 6 + (size_t)nt * 4;
+}
+
 // Launches the pruning kernel (and, with_plan, the planning kernel before it) over a list of jobs.
-template <int MAXNT, int MINB, int NJ>
+template <int MAXNT, int MINB, int NJ, int RING>
 static int launch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int nt, bool with_plan,
                              cudaStream_t st) {
     static int blocks_per_sm[MAXNT / 32 + 1] = {0};
-    const size_t dyn = (size_t)2 * kFastV * nt * sizeof(uint4);
+    const size_t dyn = fast_dyn_smem(nt, RING);
     int& bps = blocks_per_sm[nt / 32];
     if (bps == 0) {
-        if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB, NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)((size_t)2 * kFastV * MAXNT * sizeof(uint4))) != cudaSuccess)
+        if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB, NJ, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)fast_dyn_smem(MAXNT, RING)) != cudaSuccess)
             return MOSAIC_ERR_CUDA;
         int n = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB, NJ>, nt, dyn) != cudaSuccess ||
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB, NJ, RING>, nt, dyn) != cudaSuccess ||
             n < 1) {
             (void)cudaGetLastError();
             n = 1;
@@ -853,7 +910,7 @@ static int launch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, i
     }
     int64_t grid = (int64_t)sm_count() * bps;
     if (grid > total_rows) grid = total_rows;
-    prune_rows_bf16_kernel<MAXNT, MINB, NJ><<<(unsigned)grid, nt, dyn, st>>>(jobs, total_rows, cols);
+    prune_rows_bf16_kernel<MAXNT, MINB, NJ, RING><<<(unsigned)grid, nt, dyn, st>>>(jobs, total_rows, cols);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
@@ -861,9 +918,10 @@ static int launch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, i
 template <int NJ>
 static int dispatch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int nt, bool with_plan,
                                cudaStream_t st) {
-    if (nt <= 128) return launch_prune_bf16<128, 6, NJ>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 256) return launch_prune_bf16<256, 3, NJ>(jobs, total_rows, cols, nt, with_plan, st);
-    return launch_prune_bf16<512, 1, NJ>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 128) return launch_prune_bf16<128, MOSAIC_MINB_SMALL, NJ, MOSAIC_RING_SMALL>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 256) return launch_prune_bf16<256, 3, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 384) return launch_prune_bf16<384, 2, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
+    return launch_prune_bf16<512, 1, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
 }
 
 // Threads per CTA of the bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
