@@ -203,8 +203,8 @@ def run_native(args, cfg):
         for layer in mine:
             launches += 2 * driver.accumulate_norms(st, layer, X)
         if record: ev[1].record()
-        for layer in mine:
-            launches += 2 * driver.count_outliers(st, layer)
+        driver.count_outliers_all(st)
+        launches += 2                                                   # the two sweeps, each over every projection
         if record: ev[2].record()
         counts = driver.exchange_counts(st.counts, total_cfg.n_layers, rank, world)
         _, k, _ = driver.plan_sparsity(total_cfg, counts)

@@ -121,6 +121,28 @@ int mosaic_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw,
 double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
 
 /* ---------------------------------------------------------------------------
+ * mosaic_outlier_ratio_batch - mosaic_outlier_ratio for a list of projections
+ * (Algorithm 1 loops over all N*M of them) in two launches instead of two per
+ * projection.  Results are bit for bit those of the single call.
+ *   jobs   HOST array of n_jobs descriptors (read during the call only); the
+ *          pointers inside are device pointers with the meaning of the
+ *          single call's arguments (score_sum_out may be NULL)
+ *   ws     device scratch, >= mosaic_outlier_ratio_batch_workspace_bytes for
+ *          the same list
+ * Not re-entrant: one call at a time per process.
+ * ------------------------------------------------------------------------- */
+typedef struct mosaic_outlier_job {
+    const void *W;
+    int64_t rows, cols, ldw;
+    const float *norms;
+    int64_t *outlier_count_out;
+    double *score_sum_out;
+} mosaic_outlier_job;
+size_t mosaic_outlier_ratio_batch_workspace_bytes(const mosaic_outlier_job *jobs, int64_t n_jobs);
+int mosaic_outlier_ratio_batch(const mosaic_outlier_job *jobs, int64_t n_jobs, int dtype, float alpha,
+                               void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
  * mosaic_outlier_ratio_static - mosaic_outlier_ratio without a workspace
  * argument.  (The paper has no counterpart: this is a packaging variant of the
  * call above, not another operation.)
@@ -142,9 +164,9 @@ double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
  *   - The first call on each device looks up the array's device address (a
  *     host-side runtime query, with that device current).  Make that first
  *     call during start-up, outside any stream capture.
- *   - All calls on one device share the one array.  The part that has to
- *     start from zero is cleared on the stream at the start of every call, so
- *     back-to-back calls on one stream are fine; two calls that can overlap
+ *   - All calls on one device share the one array.  Every call overwrites
+ *     what it reads from it, so whatever an earlier call left there does no
+ *     harm and back-to-back calls on one stream are fine; two calls that can overlap
  *     on the GPU (different streams, different host threads) race on it and
  *     give wrong counts.  Serialise them, or give the overlapping ones their
  *     own workspace through mosaic_outlier_ratio.

@@ -30,6 +30,7 @@ SYMBOLS = (
     "mosaic_score",
     "mosaic_outlier_ratio_workspace_bytes", "mosaic_outlier_ratio", "mosaic_ratio_from_count",
     "mosaic_outlier_ratio_static_max_workspace_bytes", "mosaic_outlier_ratio_static",
+    "mosaic_outlier_ratio_batch_workspace_bytes", "mosaic_outlier_ratio_batch",
     "mosaic_allocate_sparsity",
     "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
     "mosaic_prune_unstructured_batch_workspace_bytes", "mosaic_prune_unstructured_batch",
@@ -74,6 +75,10 @@ def lib() -> C.CDLL:
         L.mosaic_outlier_ratio_static_max_workspace_bytes.argtypes = []
         L.mosaic_outlier_ratio_static.restype = ci
         L.mosaic_outlier_ratio_static.argtypes = [vp, i64, i64, i64, ci, vp, flt, vp, vp, vp]
+        L.mosaic_outlier_ratio_batch_workspace_bytes.restype = sz
+        L.mosaic_outlier_ratio_batch_workspace_bytes.argtypes = [vp, i64]
+        L.mosaic_outlier_ratio_batch.restype = ci
+        L.mosaic_outlier_ratio_batch.argtypes = [vp, i64, ci, flt, vp, sz, vp]
         L.mosaic_ratio_from_count.restype = dbl
         L.mosaic_ratio_from_count.argtypes = [i64, i64]
         L.mosaic_allocate_sparsity.restype = ci
@@ -234,6 +239,36 @@ def mosaic_outlier_ratio_static(W: torch.Tensor, norms: torch.Tensor, alpha: flo
     _check(lib().mosaic_outlier_ratio_static(p, rows, cols, ldw, _dtype_code(W), norms.data_ptr(), float(alpha),
                                              outlier_count_out.data_ptr(), _ptr(score_sum_out), _stream(stream)),
            "mosaic_outlier_ratio_static")
+
+
+class OutlierJob(C.Structure):
+    """mosaic_outlier_job of include/mosaic.h."""
+    _fields_ = [("W", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ldw", C.c_int64),
+                ("norms", C.c_void_p), ("outlier_count_out", C.c_void_p), ("score_sum_out", C.c_void_p)]
+
+
+def mosaic_outlier_ratio_batch(jobs, alpha: float, ws: Workspace | None = None, stream=None) -> None:
+    """mosaic_outlier_ratio over a list of (W, norms, outlier_count_out[1], score_sum_out[1] or None)
+    in two launches; the count tensors may be one-element views of a larger int64 tensor."""
+    if not jobs:
+        return
+    arr = (OutlierJob * len(jobs))()
+    dtype = jobs[0][0].dtype
+    for i, (W, norms, cnt, ssum) in enumerate(jobs):
+        p, rows, cols, ldw = _mat(W, "W")
+        if W.dtype != dtype:
+            raise TypeError("one dtype per batch")
+        _dev(norms, "norms", torch.float32)
+        _dev(cnt, "outlier_count_out", torch.int64)
+        if ssum is not None:
+            _dev(ssum, "score_sum_out", torch.float64)
+        if norms.numel() != cols:
+            raise ValueError("norms must be [cols]")
+        arr[i] = OutlierJob(p, rows, cols, ldw, norms.data_ptr(), cnt.data_ptr(), _ptr(ssum))
+    L = lib()
+    wp, wn = _ws(ws, jobs[0][0].device).get(L.mosaic_outlier_ratio_batch_workspace_bytes(C.addressof(arr), len(jobs)))
+    _check(L.mosaic_outlier_ratio_batch(C.addressof(arr), len(jobs), _dtype_code(jobs[0][0]), float(alpha), wp, wn,
+                                        _stream(stream)), "mosaic_outlier_ratio_batch")
 
 
 def mosaic_ratio_from_count(outlier_count: int, numel: int) -> float:

@@ -2,15 +2,17 @@
 // the outlier-count step of Algorithm 1): fp64 sum of the weight metric over a projection,
 // threshold tau = alpha * mean, strict outlier count.
 //
-// Decomposition of both sweeps: a CTA of 128 threads owns a chunk of 1024
-// columns (a thread owns 8 adjacent columns, whose norms stay in registers)
-// and a contiguous range of rows; 8 row loads are in flight per thread.
-// Sweep 1 writes one fp64 partial per CTA; the last CTA to finish adds the
-// partials in index order (so the sum does not depend on scheduling) and
-// publishes tau.  Sweep 2 walks the CTAs in reverse order, so that it starts on
-// the part of W that sweep 1 touched last and finds it in L2, and compares in
-// fp32 against tau rounded toward -inf: for an fp32 score s,
-// (double)s > tau  <=>  s > fl32_down(tau), so no fp64 work is needed.
+// Every matrix is cut into tiles of 1024 columns (a thread owns 8 adjacent
+// columns, whose norms stay in registers) by 64 rows; 8 row loads are in flight
+// per thread.  A launch works through the tiles of a whole list of matrices
+// with resident CTAs, each taking a contiguous range of tiles, so a model's
+// worth of projections costs two launches, not two per projection.
+//   sweep 1  writes one fp64 partial per tile.
+//   sweep 2  on entering a matrix adds that matrix's partials in tile order (so
+//            the sum depends neither on scheduling nor on the grid), forms tau,
+//            and counts in fp32 against tau rounded toward -inf: for an fp32
+//            score s, (double)s > tau  <=>  s > fl32_down(tau).  It walks the
+//            tiles in reverse, starting on what sweep 1 touched last.
 #include "common.cuh"
 
 namespace mosaic {
@@ -18,146 +20,159 @@ namespace mosaic {
 constexpr int kOutThreads = 128;
 constexpr int kOutChunk = kOutThreads * kVec;  // 1024 columns
 constexpr int kOutUnroll = 8;
+constexpr int kOutTileRows = 64;
+constexpr int kOutBatch = 256;                 // matrices per launch (the list travels as a kernel parameter)
 
-struct OutlierWs {           // layout of the workspace head
-    unsigned int done;       // CTAs of sweep 1 that have published their partial
-    unsigned int pad;
-    float tau_down;          // alpha*mean rounded toward -inf to fp32
-    float pad2;
-    double sum;              // S
-    double tau;              // alpha*mean in fp64
-    double partial[1];       // [grid]
+struct OutlierJob {
+    const void* W;
+    const float* norms;
+    unsigned long long* count_out;
+    double* sum_out;       // or nullptr
+    double* partial;       // [tiles of this matrix], in the workspace
+    int64_t rows, cols, ldw;
+    int tile0;             // first global tile
+    int chunks;            // tiles per row band
+};
+template <int NJ>
+struct OutlierJobList {
+    int n;
+    float alpha;
+    OutlierJob job[NJ];
 };
 
-struct OutlierPlan {
-    int chunks, splits, rows_per_split;
-};
-
-static OutlierPlan outlier_plan(int64_t rows, int64_t cols) {
-    OutlierPlan p;
-    p.chunks = (int)((cols + kOutChunk - 1) / kOutChunk);
-    int64_t target = (int64_t)sm_count() * 16;
-    int64_t splits = target / p.chunks;
-    if (splits < 1) splits = 1;
-    int64_t max_splits = (rows + kOutUnroll - 1) / kOutUnroll;
-    if (splits > max_splits) splits = max_splits;
-    if (splits < 1) splits = 1;
-    int64_t rps = (rows + splits - 1) / splits;
-    rps = (rps + kOutUnroll - 1) / kOutUnroll * kOutUnroll;
-    p.rows_per_split = (int)rps;
-    p.splits = (int)((rows + rps - 1) / rps);
-    if (p.splits < 1) p.splits = 1;
-    return p;
+__host__ __device__ inline int64_t outlier_tiles(int64_t rows, int64_t cols) {
+    return ((cols + kOutChunk - 1) / kOutChunk) * ((rows + kOutTileRows - 1) / kOutTileRows);
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kOutThreads) score_sum_kernel(const void* __restrict__ W, int64_t rows, int64_t cols,
-                                                                 int64_t ldw, const float* __restrict__ norms, int chunks,
-                                                                 int rows_per_split, float alpha, OutlierWs* ws,
-                                                                 double* score_sum_out) {
+// Tiles [t_begin, t_end) of this CTA: an equal share of the n_tiles, contiguous.
+__device__ __forceinline__ void tile_share(int n_tiles, int* t_begin, int* t_end) {
+    const int64_t g = gridDim.x, b = blockIdx.x;
+    *t_begin = (int)((int64_t)n_tiles * b / g);
+    *t_end = (int)((int64_t)n_tiles * (b + 1) / g);
+}
+
+template <int DT, int NJ>
+__global__ void __launch_bounds__(kOutThreads) score_sum_kernel(const __grid_constant__ OutlierJobList<NJ> jobs, int n_tiles) {
     __shared__ double red[32];
-    __shared__ bool is_last;
-    const int chunk = blockIdx.x % chunks, split = blockIdx.x / chunks;
-    const int64_t c0 = (int64_t)chunk * kOutChunk + threadIdx.x * kVec;
-    const int64_t r0 = (int64_t)split * rows_per_split;
-    const int64_t r1 = (r0 + rows_per_split < rows) ? r0 + rows_per_split : rows;
-
-    double acc[4] = {0.0, 0.0, 0.0, 0.0};
-    if (c0 < cols) {
-        float nrm[kVec];
+    int t_begin, t_end;
+    tile_share(n_tiles, &t_begin, &t_end);
+    int j = 0;
+    for (int tile = t_begin; tile < t_end; ++tile) {
+        while (j + 1 < jobs.n && tile >= jobs.job[j + 1].tile0) ++j;
+        const OutlierJob& J = jobs.job[j];
+        const int local = tile - J.tile0;
+        if (local == 0 && threadIdx.x == 0) *J.count_out = 0ull;   // sweep 2 is a later launch
+        const int chunk = local % J.chunks, band = local / J.chunks;
+        const int64_t rows = J.rows, cols = J.cols, ldw = J.ldw;
+        const int64_t c0 = (int64_t)chunk * kOutChunk + threadIdx.x * kVec;
+        const int64_t r0 = (int64_t)band * kOutTileRows;
+        const int64_t r1 = (r0 + kOutTileRows < rows) ? r0 + kOutTileRows : rows;
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+        if (c0 < cols) {
+            float nrm[kVec];
 #pragma unroll
-        for (int e = 0; e < kVec; ++e) nrm[e] = (c0 + e < cols) ? norms[c0 + e] : 0.0f;
-        int64_t r = r0;
-        for (; r + kOutUnroll <= r1; r += kOutUnroll) {
-            Raw8<DT> v[kOutUnroll];
+            for (int e = 0; e < kVec; ++e) nrm[e] = (c0 + e < cols) ? J.norms[c0 + e] : 0.0f;
+            int64_t r = r0;
+            for (; r + kOutUnroll <= r1; r += kOutUnroll) {
+                Raw8<DT> v[kOutUnroll];
 #pragma unroll
-            for (int u = 0; u < kOutUnroll; ++u) load_vec<DT, true>(v[u], W, (r + u) * ldw, c0, cols);
+                for (int u = 0; u < kOutUnroll; ++u) load_vec<DT, true>(v[u], J.W, (r + u) * ldw, c0, cols);
 #pragma unroll
-            for (int u = 0; u < kOutUnroll; ++u)
+                for (int u = 0; u < kOutUnroll; ++u)
 #pragma unroll
-                for (int e = 0; e < kVec; ++e) acc[u & 3] += (double)__fmul_rn(nrm[e], v[u].abs_f32(e));
+                    for (int e = 0; e < kVec; ++e) acc[u & 3] += (double)__fmul_rn(nrm[e], v[u].abs_f32(e));
+            }
+            for (; r < r1; ++r) {
+                Raw8<DT> v;
+                load_vec<DT, true>(v, J.W, r * ldw, c0, cols);
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) acc[0] += (double)__fmul_rn(nrm[e], v.abs_f32(e));
+            }
         }
-        for (; r < r1; ++r) {
-            Raw8<DT> v;
-            load_vec<DT, true>(v, W, r * ldw, c0, cols);
-#pragma unroll
-            for (int e = 0; e < kVec; ++e) acc[0] += (double)__fmul_rn(nrm[e], v.abs_f32(e));
-        }
-    }
-    const double mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
-    const double blk = block_sum(mine, red);
-    if (threadIdx.x == 0) {
-        ws->partial[blockIdx.x] = blk;
-        __threadfence();
-        const unsigned prev = atomicAdd(&ws->done, 1u);
-        is_last = (prev == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    // last CTA: add all partials in index order (thread-strided, then a fixed tree)
-    double s = 0.0;
-    for (unsigned i = threadIdx.x; i < gridDim.x; i += kOutThreads) s += __ldcg(&ws->partial[i]);
-    const double total = block_sum(s, red);
-    if (threadIdx.x == 0) {
-        const double mean = total / (double)(rows * cols);
-        const double tau = (double)alpha * mean;
-        ws->sum = total;
-        ws->tau = tau;
-        ws->tau_down = __double2float_rd(tau);
-        ws->done = 0u;
-        if (score_sum_out) *score_sum_out = total;
+        const double mine = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+        const double blk = block_sum(mine, red);
+        if (threadIdx.x == 0) J.partial[local] = blk;
     }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kOutThreads) outlier_count_kernel(const void* __restrict__ W, int64_t rows, int64_t cols,
-                                                                     int64_t ldw, const float* __restrict__ norms,
-                                                                     int chunks, int rows_per_split, const OutlierWs* ws,
-                                                                     unsigned long long* count_out) {
-    __shared__ unsigned int red[32];
-    const unsigned b = gridDim.x - 1 - blockIdx.x;  // reverse order of sweep 1
-    const int chunk = b % chunks, split = b / chunks;
-    const int64_t c0 = (int64_t)chunk * kOutChunk + threadIdx.x * kVec;
-    const int64_t r0 = (int64_t)split * rows_per_split;
-    const int64_t r1 = (r0 + rows_per_split < rows) ? r0 + rows_per_split : rows;
-    const float tau = ws->tau_down;
-
+template <int DT, int NJ>
+__global__ void __launch_bounds__(kOutThreads) outlier_count_kernel(const __grid_constant__ OutlierJobList<NJ> jobs, int n_tiles) {
+    __shared__ double red[32];
+    __shared__ unsigned int cred[32];
+    __shared__ float tau_sh;
+    int t_begin, t_end;
+    tile_share(n_tiles, &t_begin, &t_end);
+    int j = jobs.n - 1, j_tau = -1;
+    float tau = 0.0f;
     unsigned int cnt = 0;
-    if (c0 < cols) {
-        float nrm[kVec];
-        bool valid[kVec];
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) {
-            valid[e] = (c0 + e < cols);
-            nrm[e] = valid[e] ? norms[c0 + e] : 0.0f;
+    auto flush = [&](int job) {   // add this CTA's count for `job` (block-uniform call)
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+        __syncthreads();
+        if (lane == 0) cred[wid] = cnt;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long tot = 0;
+            for (int i = 0; i < kOutThreads / 32; ++i) tot += cred[i];
+            if (tot) atomicAdd(jobs.job[job].count_out, tot);   // integer: exact in any order
         }
-        int64_t r = r1;
-        for (; r - kOutUnroll >= r0; r -= kOutUnroll) {
-            Raw8<DT> v[kOutUnroll];
-#pragma unroll
-            for (int u = 0; u < kOutUnroll; ++u) load_vec<DT, true>(v[u], W, (r - 1 - u) * ldw, c0, cols);
-#pragma unroll
-            for (int u = 0; u < kOutUnroll; ++u)
-#pragma unroll
-                for (int e = 0; e < kVec; ++e) cnt += (valid[e] && __fmul_rn(nrm[e], v[u].abs_f32(e)) > tau) ? 1u : 0u;
+        cnt = 0;
+    };
+    for (int t2 = t_begin; t2 < t_end; ++t2) {
+        const int tile = n_tiles - 1 - t2;   // reverse order of sweep 1
+        while (tile < jobs.job[j].tile0) --j;
+        const OutlierJob& J = jobs.job[j];
+        const int64_t rows = J.rows, cols = J.cols, ldw = J.ldw;
+        if (j != j_tau) {
+            if (j_tau >= 0) flush(j_tau);
+            // this matrix's partials in tile order: thread-strided, then a fixed tree
+            const int nt_j = (int)outlier_tiles(rows, cols);
+            double s = 0.0;
+            for (int i = threadIdx.x; i < nt_j; i += kOutThreads) s += __ldcg(&J.partial[i]);
+            const double total = block_sum(s, red);
+            if (threadIdx.x == 0) {
+                const double mean = total / (double)(rows * cols);
+                const double tau_d = (double)jobs.alpha * mean;
+                tau_sh = __double2float_rd(tau_d);
+                if (tile == J.tile0 + nt_j - 1 && J.sum_out) *J.sum_out = total;   // once: by the CTA that owns the last tile
+            }
+            __syncthreads();
+            tau = tau_sh;
+            j_tau = j;
         }
-        for (; r > r0; --r) {
-            Raw8<DT> v;
-            load_vec<DT, true>(v, W, (r - 1) * ldw, c0, cols);
+        const int local = tile - J.tile0;
+        const int chunk = local % J.chunks, band = local / J.chunks;
+        const int64_t c0 = (int64_t)chunk * kOutChunk + threadIdx.x * kVec;
+        const int64_t r0 = (int64_t)band * kOutTileRows;
+        const int64_t r1 = (r0 + kOutTileRows < rows) ? r0 + kOutTileRows : rows;
+        if (c0 < cols) {
+            float nrm[kVec];
+            bool valid[kVec];
 #pragma unroll
-            for (int e = 0; e < kVec; ++e) cnt += (valid[e] && __fmul_rn(nrm[e], v.abs_f32(e)) > tau) ? 1u : 0u;
+            for (int e = 0; e < kVec; ++e) {
+                valid[e] = (c0 + e < cols);
+                nrm[e] = valid[e] ? J.norms[c0 + e] : 0.0f;
+            }
+            int64_t r = r1;
+            for (; r - kOutUnroll >= r0; r -= kOutUnroll) {
+                Raw8<DT> v[kOutUnroll];
+#pragma unroll
+                for (int u = 0; u < kOutUnroll; ++u) load_vec<DT, true>(v[u], J.W, (r - 1 - u) * ldw, c0, cols);
+#pragma unroll
+                for (int u = 0; u < kOutUnroll; ++u)
+#pragma unroll
+                    for (int e = 0; e < kVec; ++e)
+                        cnt += (valid[e] && __fmul_rn(nrm[e], v[u].abs_f32(e)) > tau) ? 1u : 0u;
+            }
+            for (; r > r0; --r) {
+                Raw8<DT> v;
+                load_vec<DT, true>(v, J.W, (r - 1) * ldw, c0, cols);
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) cnt += (valid[e] && __fmul_rn(nrm[e], v.abs_f32(e)) > tau) ? 1u : 0u;
+            }
         }
     }
-    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    if (lane == 0) red[wid] = cnt;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        unsigned long long t = 0;
-        for (int i = 0; i < kOutThreads / 32; ++i) t += red[i];
-        if (t) atomicAdd(count_out, t);   // integer: exact in any order
-    }
+    if (j_tau >= 0) flush(j_tau);
 }
 
 template <int DT>
@@ -200,43 +215,117 @@ extern "C" int mosaic_score(const void* W, int64_t rows, int64_t cols, int64_t l
     return MOSAIC_OK;
 }
 
+static int validate_outlier(const void* W, int64_t rows, int64_t cols, int64_t ldw, int dtype, const float* norms,
+                            const int64_t* outlier_count_out, const double* score_sum_out) {
+    int rc = check_matrix(W, rows, cols, ldw, dtype);
+    if (rc != MOSAIC_OK) return rc;
+    if (rows == 0) return MOSAIC_ERR_INVALID_ARG;
+    if (!norms || !outlier_count_out) return MOSAIC_ERR_NULL_PTR;
+    if ((reinterpret_cast<uintptr_t>(outlier_count_out) & 7u) || (reinterpret_cast<uintptr_t>(score_sum_out) & 7u) ||
+        (reinterpret_cast<uintptr_t>(norms) & 3u))
+        return MOSAIC_ERR_MISALIGNED;
+    if (outlier_tiles(rows, cols) > 0x3FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    return MOSAIC_OK;
+}
+
+template <int NJ>
+static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int dtype, cudaStream_t st) {
+    static int blocks_per_sm[2] = {0, 0};
+    int& bps = blocks_per_sm[dtype == MOSAIC_BF16 ? 1 : 0];
+    if (bps == 0) {
+        int n1 = 0, n2 = 0;
+        cudaError_t e1, e2;
+        if (dtype == MOSAIC_BF16) {
+            e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n1, score_sum_kernel<MOSAIC_BF16, NJ>, kOutThreads, 0);
+            e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, outlier_count_kernel<MOSAIC_BF16, NJ>, kOutThreads, 0);
+        } else {
+            e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n1, score_sum_kernel<MOSAIC_F32, NJ>, kOutThreads, 0);
+            e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, outlier_count_kernel<MOSAIC_F32, NJ>, kOutThreads, 0);
+        }
+        if (e1 != cudaSuccess || e2 != cudaSuccess) {
+            (void)cudaGetLastError();
+            n1 = n2 = 4;
+        }
+        bps = n1 < n2 ? n1 : n2;
+        if (bps < 1) bps = 1;
+    }
+    int64_t grid = (int64_t)sm_count() * bps;
+    if (grid > n_tiles) grid = n_tiles;
+    if (dtype == MOSAIC_BF16) {
+        score_sum_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        MOSAIC_LAUNCH_CHECK();
+        outlier_count_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+    } else {
+        score_sum_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        MOSAIC_LAUNCH_CHECK();
+        outlier_count_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+    }
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
 extern "C" size_t mosaic_outlier_ratio_workspace_bytes(int64_t rows, int64_t cols) {
     if (rows <= 0 || cols <= 0) return 256;
-    const OutlierPlan p = outlier_plan(rows, cols);
-    return align_up(sizeof(OutlierWs) + sizeof(double) * (size_t)p.chunks * (size_t)p.splits, 256);
+    return align_up(sizeof(double) * (size_t)outlier_tiles(rows, cols), 256);
 }
 
 extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
                                     const float* norms, float alpha, int64_t* outlier_count_out, double* score_sum_out,
                                     void* ws, size_t ws_bytes, void* stream) {
-    int rc = check_matrix(W, rows, cols, ldw, dtype);
+    const int rc = validate_outlier(W, rows, cols, ldw, dtype, norms, outlier_count_out, score_sum_out);
     if (rc != MOSAIC_OK) return rc;
-    if (rows == 0) return MOSAIC_ERR_INVALID_ARG;
-    if (!norms || !outlier_count_out || !ws) return MOSAIC_ERR_NULL_PTR;
-    if ((reinterpret_cast<uintptr_t>(ws) & 255u) || (reinterpret_cast<uintptr_t>(outlier_count_out) & 7u) ||
-        (reinterpret_cast<uintptr_t>(score_sum_out) & 7u) || (reinterpret_cast<uintptr_t>(norms) & 3u))
-        return MOSAIC_ERR_MISALIGNED;
+    if (!ws) return MOSAIC_ERR_NULL_PTR;
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
     if (ws_bytes < mosaic_outlier_ratio_workspace_bytes(rows, cols)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const OutlierPlan p = outlier_plan(rows, cols);
-    const unsigned grid = (unsigned)(p.chunks * p.splits);
-    OutlierWs* w = static_cast<OutlierWs*>(ws);
-    MOSAIC_CUDA_TRY(cudaMemsetAsync(w, 0, 16, st));
-    MOSAIC_CUDA_TRY(cudaMemsetAsync(outlier_count_out, 0, sizeof(int64_t), st));
-    if (dtype == MOSAIC_BF16) {
-        score_sum_kernel<MOSAIC_BF16><<<grid, kOutThreads, 0, st>>>(W, rows, cols, ldw, norms, p.chunks, p.rows_per_split,
-                                                                  alpha, w, score_sum_out);
-        MOSAIC_LAUNCH_CHECK();
-        outlier_count_kernel<MOSAIC_BF16><<<grid, kOutThreads, 0, st>>>(
-            W, rows, cols, ldw, norms, p.chunks, p.rows_per_split, w, reinterpret_cast<unsigned long long*>(outlier_count_out));
-    } else {
-        score_sum_kernel<MOSAIC_F32><<<grid, kOutThreads, 0, st>>>(W, rows, cols, ldw, norms, p.chunks, p.rows_per_split,
-                                                                 alpha, w, score_sum_out);
-        MOSAIC_LAUNCH_CHECK();
-        outlier_count_kernel<MOSAIC_F32><<<grid, kOutThreads, 0, st>>>(
-            W, rows, cols, ldw, norms, p.chunks, p.rows_per_split, w, reinterpret_cast<unsigned long long*>(outlier_count_out));
+    OutlierJobList<1> one;
+    one.n = 1;
+    one.alpha = alpha;
+    one.job[0] = OutlierJob{W, norms, reinterpret_cast<unsigned long long*>(outlier_count_out), score_sum_out,
+                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk)};
+    return launch_outlier<1>(one, outlier_tiles(rows, cols), dtype, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" size_t mosaic_outlier_ratio_batch_workspace_bytes(const mosaic_outlier_job* jobs, int64_t n_jobs) {
+    size_t total = 256;
+    if (jobs == nullptr) return total;
+    for (int64_t i = 0; i < n_jobs; ++i) total += mosaic_outlier_ratio_workspace_bytes(jobs[i].rows, jobs[i].cols);
+    return total;
+}
+
+extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_t n_jobs, int dtype, float alpha, void* ws,
+                                          size_t ws_bytes, void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr || ws == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_outlier_job& j = jobs[i];
+        const int rc = validate_outlier(j.W, j.rows, j.cols, j.ldw, dtype, j.norms, j.outlier_count_out, j.score_sum_out);
+        if (rc != MOSAIC_OK) return rc;
     }
-    MOSAIC_LAUNCH_CHECK();
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
+    if (ws_bytes < mosaic_outlier_ratio_batch_workspace_bytes(jobs, n_jobs)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    static OutlierJobList<kOutBatch> list;   // host staging of the kernel parameter; calls are not re-entrant
+    char* wsp = static_cast<char*>(ws);
+    int64_t i = 0;
+    while (i < n_jobs) {
+        list.n = 0;
+        list.alpha = alpha;
+        int64_t tiles = 0;
+        while (i < n_jobs && list.n < kOutBatch) {
+            const mosaic_outlier_job& j = jobs[i];
+            const int64_t nt = outlier_tiles(j.rows, j.cols);
+            if (tiles + nt > 0x3FFFFFFF) break;
+            list.job[list.n++] = OutlierJob{j.W, j.norms, reinterpret_cast<unsigned long long*>(j.outlier_count_out),
+                                            j.score_sum_out, reinterpret_cast<double*>(wsp), j.rows, j.cols, j.ldw,
+                                            (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk)};
+            wsp += mosaic_outlier_ratio_workspace_bytes(j.rows, j.cols);
+            tiles += nt;
+            ++i;
+        }
+        const int rc = launch_outlier<kOutBatch>(list, tiles, dtype, st);
+        if (rc != MOSAIC_OK) return rc;
+    }
     return MOSAIC_OK;
 }
 
@@ -247,8 +336,8 @@ extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, i
 namespace mosaic {
 
 // Scratch of mosaic_outlier_ratio_static.  Every device that loads the library carries these
-// 64 KiB until the process exits.  It holds the sweep counter, the threshold and one fp64
-// partial sum per CTA of the first sweep (a few thousand at most on current parts).
+// 64 KiB until the process exits.  It holds one fp64 partial sum per tile (1024 columns by 64
+// rows) of the first sweep: room for matrices of up to 8192 tiles, i.e. half a billion weights.
 constexpr size_t kStaticScratchBytes = MOSAIC_OUTLIER_STATIC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_outlier_scratch[kStaticScratchBytes];
 
@@ -288,8 +377,8 @@ extern "C" int mosaic_outlier_ratio_static(const void* W, int64_t rows, int64_t 
     void* scratch = nullptr;
     rc = static_scratch_address(&scratch);
     if (rc != MOSAIC_OK) return rc;
-    // The regular entry point clears the part of the scratch that must start at zero (the sweep
-    // counter) on the stream before the first kernel, so what an earlier call left behind is harmless.
+    // Nothing in the scratch has to start at zero: every partial sum is written by the first sweep
+    // before the second reads it, so what an earlier call left behind is harmless.
     return mosaic_outlier_ratio(W, rows, cols, ldw, dtype, norms, alpha, outlier_count_out, score_sum_out, scratch,
                                 kStaticScratchBytes, stream);
 }

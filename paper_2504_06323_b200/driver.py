@@ -136,6 +136,21 @@ def count_outliers(st: ModelState, layer: int, alpha: float | None = None) -> in
     return len(PROJECTIONS)
 
 
+def count_outliers_all(st: ModelState, alpha: float | None = None) -> int:
+    """Outlier counts of every owned projection through the batched call (two launches)."""
+    cfg = st.cfg
+    a = cfg.alpha if alpha is None else alpha
+    jobs = []
+    for layer in st.layers:
+        for pr in PROJECTIONS:
+            q = st.q_local(layer, pr)
+            jobs.append((st.W[layer, pr], st.norms[layer, cfg.x_key(pr)], st.counts[q:q + 1], None))
+    if getattr(st, "ws_batch", None) is None:
+        st.ws_batch = api.Workspace(st.device)
+    api.mosaic_outlier_ratio_batch(jobs, a, st.ws_batch)
+    return len(jobs)
+
+
 # ------------------------------------------------------------------ phase B
 def prune_unstructured_layer(st: ModelState, layer: int, k_global: list[int], in_place: bool = False) -> int:
     cfg = st.cfg

@@ -50,6 +50,9 @@ def run_phase_a(cfg):
         assert ok.all(), "re-seed: a column sits on an fp32 rounding boundary"
         assert bits_equal(got, norms_ref[key])
     assert counts == counts_ref
+    st.counts.fill_(-3)                     # and the batched call over every projection gives the same counts
+    driver.count_outliers_all(st)
+    assert driver.exchange_counts(st.counts, cfg.n_layers, 0, 1) == counts_ref
     return st, Wh, Xh, norms_ref, counts
 
 

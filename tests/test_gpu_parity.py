@@ -129,6 +129,35 @@ def test_outlier_ratio(dtype, rows, cols, ld, alpha):
     assert cnt2.item() == cnt.item()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_outlier_ratio_batch_matches_oracle_job_by_job(dtype):
+    shapes = [(256, 256), (688, 256), (300, 1000), (7, 13), (1100, 4096), (64, 11008), (65, 1024), (1, 8)]
+    jobs, refs = [], []
+    counts = torch.full((len(shapes),), -5, dtype=torch.int64, device=DEV)
+    sums = torch.full((len(shapes),), -1.0, dtype=torch.float64, device=DEV)
+    for i, (rows, cols) in enumerate(shapes):
+        ld = cols if cols % 8 == 0 else (cols + 7) // 8 * 8
+        W = make(rows, cols, dtype, seed=900 + i, ld=ld, heavy=(i % 2 == 1))
+        norms = norms_for(cols, 60 + i)
+        refs.append(oracle.outlier_ratio(host(W), norms.cpu().numpy(), 4.0, dtype))
+        jobs.append((W, norms, counts[i:i + 1], sums[i:i + 1] if i != 2 else None))
+    api.mosaic_outlier_ratio_batch(jobs, 4.0)
+    for i, ref in enumerate(refs):
+        assert ref["certified"]
+        assert counts[i].item() == ref["count"], shapes[i]
+        if i != 2:
+            np.testing.assert_allclose(sums[i].item(), ref["sum"], rtol=1e-12)
+    assert sums[2].item() == -1.0
+    # the single call gives the same bits as the batch
+    for i, (W, norms, _, _) in enumerate(jobs):
+        c1 = torch.zeros(1, dtype=torch.int64, device=DEV)
+        s1 = torch.zeros(1, dtype=torch.float64, device=DEV)
+        api.mosaic_outlier_ratio(W, norms, 4.0, c1, s1)
+        assert c1.item() == counts[i].item()
+        if i != 2:
+            assert s1.cpu().numpy().tobytes() == sums[i:i + 1].cpu().numpy().tobytes()
+
+
 def test_outlier_planted_and_constant():
     rows, cols = 64, 1024
     W = torch.ones(rows, cols, dtype=torch.bfloat16, device=DEV)
