@@ -40,9 +40,10 @@ from paper_2504_06323_b200.workloads import PROJECTIONS  # noqa: E402
 METRIC = "weight_GBps_scored_and_pruned"
 UNIT = "GB/s"
 
-# DRAM traffic per launch of the dominant kernel from an ncu capture (bytes read + written
-# divided by the bytes of X the launch reduces); see profiles/.  None until captured.
-NCU_TRAFFIC_RATIO = {"col_partial_kernel": None}
+# DRAM traffic of the dominant kernel from an ncu capture of a smaller launch (profiles/
+# col_partial_kernel_act_norms_small.md): reads = 1.00006 x the bytes of X (they scale with the
+# token count), writes = the split partials, 1172 B per column whatever the token count.
+NCU_TRAFFIC = {"col_partial_kernel": {"read_ratio": 1.00006, "write_bytes_per_col": 1172.0}}
 
 
 def measured_peaks():
@@ -195,23 +196,22 @@ def run_native(args, cfg):
     w_bytes = sum(st.W[l, p].numel() * cfg.itemsize for l in mine for p in PROJECTIONS)
     x_bytes_layer = sum(x.numel() * cfg.itemsize for x in X.values())
 
-    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-
-    def step(record=False):
+    def step(ev=None):
+        """One pass of the whole path.  `ev`: five CUDA events recorded at the phase boundaries."""
         launches = 0
-        if record: ev[0].record()
+        if ev: ev[0].record()
         for layer in mine:
             launches += 2 * driver.accumulate_norms(st, layer, X)
-        if record: ev[1].record()
+        if ev: ev[1].record()
         driver.count_outliers_all(st)
         launches += 2                                                   # the two sweeps, each over every projection
-        if record: ev[2].record()
+        if ev: ev[2].record()
         counts = driver.exchange_counts(st.counts, total_cfg.n_layers, rank, world)
         _, k, _ = driver.plan_sparsity(total_cfg, counts)
-        if record: ev[3].record()
+        if ev: ev[3].record()
         driver.prune_unstructured_all(st, k)
         launches += 2 * len({cfg.shape(p)[1] for p in PROJECTIONS})      # planning + pruning launch per distinct row length
-        if record: ev[4].record()
+        if ev: ev[4].record()
         return launches
 
     for _ in range(max(args.warmup, 3)):
@@ -220,23 +220,18 @@ def run_native(args, cfg):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    phase_ms = [0.0, 0.0, 0.0, 0.0]
+    # phase boundaries are marked inside the timed region (an event record costs nothing on the device)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     start.record()
     launches = 0
-    phase_events = []
-    for _ in range(args.steps):
-        launches += step(record=False)
+    for s in range(args.steps):
+        launches += step(events[s])
     end.record()
     barrier()
     total_ms = start.elapsed_time(end)
-    # phase breakdown on separate (untimed) steps so that event bookkeeping does not sit in the timed region
-    for _ in range(3):
-        step(record=True)
-        torch.cuda.synchronize()
-        for i in range(4):
-            phase_ms[i] += ev[i].elapsed_time(ev[i + 1]) / 3.0
+    phase_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) / args.steps for i in range(4)]
     clocks = sampler.stop() if rank == 0 else None
 
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -273,11 +268,14 @@ def run_native(args, cfg):
     n_act_launch = len(mine) * len(X)
     act_bytes = x_bytes_layer * len(mine)
     act_gbs = act_bytes / (phase_ms[0] * 1e-3) / 1e9
-    ratio = NCU_TRAFFIC_RATIO["col_partial_kernel"]
+    tr = NCU_TRAFFIC["col_partial_kernel"]
+    avg_cols = sum(x.shape[1] for x in X.values()) / len(X)
     roofline = {
         "kernel": "col_partial_kernel<bf16, square> (activation norms)", "bound": "hbm", "achieved": act_gbs,
         "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": act_gbs / peak,
-        "traffic": None if ratio is None else ratio * act_bytes / n_act_launch,
+        "traffic": tr["read_ratio"] * act_bytes / n_act_launch + tr["write_bytes_per_col"] * avg_cols,
+        "traffic_note": "bytes per launch, scaled from an ncu capture of a 32768-token launch (reads scale with tokens, "
+                        "partial-sum writes do not)",
         "algorithmic_bytes_per_launch": act_bytes / n_act_launch, "launches_per_step": n_act_launch,
         "avg_launch_ms": phase_ms[0] / n_act_launch,
     }
@@ -302,10 +300,12 @@ def run_native(args, cfg):
                         "frac_of_peak": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / peak,
                         "frac_of_8TBps": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / 8000.0},
         "roofline_other": [
-            {"kernel": "score_sum_kernel + outlier_count_kernel", "bound": "hbm", "achieved": outl_gbs, "peak": peak,
-             "unit": "GB/s", "frac": outl_gbs / peak, "algorithmic_bytes": "2 B/weight"},
-            {"kernel": "prune_rows_kernel", "bound": "hbm", "achieved": prune_gbs, "peak": peak, "unit": "GB/s",
-             "frac": prune_gbs / peak, "algorithmic_bytes": "4.125 B/weight"}],
+            {"kernel": "score_sum_kernel + outlier_count_kernel (two launches over all projections)", "bound": "hbm",
+             "achieved": outl_gbs, "peak": peak, "unit": "GB/s", "frac": outl_gbs / peak,
+             "algorithmic_bytes": "2 B/weight (the count sweep is a second read: 4 B/weight executed)"},
+            {"kernel": "prune_plan_kernel + prune_rows_bf16_kernel (one pair of launches per row length)", "bound": "hbm",
+             "achieved": prune_gbs, "peak": peak, "unit": "GB/s", "frac": prune_gbs / peak,
+             "algorithmic_bytes": "4.125 B/weight"}],
     }
     print(json.dumps(line), flush=True)
     if world > 1:
