@@ -45,6 +45,12 @@
 #ifndef MOSAIC_MINB_SMALL
 #define MOSAIC_MINB_SMALL 4
 #endif
+#ifndef MOSAIC_ROUND_UNROLL
+#define MOSAIC_ROUND_UNROLL 1
+#endif
+#ifndef MOSAIC_NORM_EVICT_LAST
+#define MOSAIC_NORM_EVICT_LAST 1
+#endif
 #ifndef MOSAIC_FAST_MAX_CTAS
 #define MOSAIC_FAST_MAX_CTAS 8
 #endif
@@ -293,6 +299,7 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
 // ---------------------------------------------------------------------------------------------
 constexpr int kFastV = 4;          // vectors (of 8 columns) per thread
 constexpr int kWinBins = 1024;     // histogram over the top 10 bits of a window
+constexpr int kRoundUnroll = MOSAIC_ROUND_UNROLL;
 constexpr int kQueueCap = 448;     // candidates a warp can queue (of its 1024 weights)
 constexpr int kBinListCap = 512;   // keys of one histogram bin that warp 0 will rank; also the sample size limit
 
@@ -308,6 +315,16 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+// A norm, kept in L1 with priority: the row data streams past it.
+__device__ __forceinline__ float ld_norm(const float* p) {
+#if MOSAIC_NORM_EVICT_LAST
+    float v;
+    asm volatile("ld.global.nc.L1::evict_last.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+#else
+    return __ldg(p);
+#endif
+}
 __device__ __forceinline__ void sts_u16_zero(void* smem) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "h"((unsigned short)0) : "memory");
 }
@@ -487,6 +504,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
     __shared__ SelectResult sel3;
     __shared__ RowSelect sel;
     __shared__ uint8_t spread[16];                       // bits abcd -> 0a0b0c0d
+    __shared__ uint16_t col_of_flag[32];                 // packed flag bit -> column of that weight relative to the lane's first column
 
     const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = nt >> 5;
     const int nvec = cols >> 3;
@@ -505,6 +523,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
     for (int b = tid; b < kBins1; b += nt) buf[b] = 0u;
     if (tid < 32) coarse[tid] = 0u;
     if (tid < 16) spread[tid] = (uint8_t)((tid & 1) | ((tid & 2) << 1) | ((tid & 4) << 2) | ((tid & 8) << 3));
+    if (tid < 32) col_of_flag[tid] = (uint16_t)(packed_vec(tid) * nt * kVec + flag_elem(tid + 4 * packed_vec(tid)));
     if (tid == 0) n_list = 0u;
     __syncthreads();
 
@@ -605,13 +624,14 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
             __syncwarp();
         }
         // exact scores of the candidates, 32 at a time: below lo, or into the window histogram
+        const uint16_t* row_elems = reinterpret_cast<const uint16_t*>(rowbuf + cur * V * nt);   // column c of the row is element c
+        const int warp_col0 = (wid << 5) * kVec;
+#pragma unroll kRoundUnroll
         for (uint32_t i = lane; i < q_n; i += 32) {
             const uint32_t id = qid[i];
-            const int b = id & 31, v = packed_vec(b), e = flag_elem(b + 4 * v);
-            const int owner = (wid << 5) | (int)(id >> 5);
-            const uint16_t* p = reinterpret_cast<const uint16_t*>(&rowbuf[(cur * V + v) * nt + owner]);
-            const uint32_t a = ((uint32_t)p[e] & 0x7FFFu) << 16;
-            const uint32_t key = __float_as_uint(__fmul_rn(__ldg(norms + (v * nt + owner) * kVec + e), __uint_as_float(a)));
+            const int col = warp_col0 + (int)(id >> 5) * kVec + col_of_flag[id & 31];
+            const uint32_t a = ((uint32_t)row_elems[col] & 0x7FFFu) << 16;
+            const uint32_t key = __float_as_uint(__fmul_rn(ld_norm(norms + col), __uint_as_float(a)));
             qkey[i] = key;
             const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
             if (d < width) {
@@ -713,10 +733,9 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         for (uint32_t i = lane; i < q_n; i += 32) {
             if (qkey[i] < thr) {
                 const uint32_t id = qid[i];
-                const int b = id & 31, v = packed_vec(b), e = flag_elem(b + 4 * v);
-                const int owner = (wid << 5) | (int)(id >> 5);
-                sts_u16_zero(reinterpret_cast<uint16_t*>(&rowbuf[(cur * V + v) * nt + owner]) + e);
-                atomicOr(&gone_w[owner], 1u << b);
+                const int col = warp_col0 + (int)(id >> 5) * kVec + col_of_flag[id & 31];
+                sts_u16_zero(reinterpret_cast<uint16_t*>(rowbuf + cur * V * nt) + col);
+                atomicOr(&gone_w[(wid << 5) | (int)(id >> 5)], 1u << (id & 31));
             }
         }
         __syncwarp();
