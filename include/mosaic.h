@@ -129,7 +129,6 @@ double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
  *          single call's arguments (score_sum_out may be NULL)
  *   ws     device scratch, >= mosaic_outlier_ratio_batch_workspace_bytes for
  *          the same list
- * Not re-entrant: one call at a time per process.
  * ------------------------------------------------------------------------- */
 typedef struct mosaic_outlier_job {
     const void *W;
@@ -226,8 +225,7 @@ int mosaic_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64
  *   ws       device scratch, >= mosaic_prune_unstructured_batch_workspace_bytes
  *            for the same list; it receives, per job, the key window and the
  *            per-column thresholds a planning kernel derives from three rows
- * Jobs must not overlap each other's outputs.  Not re-entrant: one call at a
- * time per process.
+ * Jobs must not overlap each other's outputs.
  * ------------------------------------------------------------------------- */
 typedef struct mosaic_prune_job {
     const void *W_in;

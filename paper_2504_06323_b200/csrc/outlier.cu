@@ -13,6 +13,8 @@
 //            and counts in fp32 against tau rounded toward -inf: for an fp32
 //            score s, (double)s > tau  <=>  s > fl32_down(tau).  It walks the
 //            tiles in reverse, starting on what sweep 1 touched last.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace mosaic {
@@ -305,7 +307,9 @@ extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_
     if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
     if (ws_bytes < mosaic_outlier_ratio_batch_workspace_bytes(jobs, n_jobs)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    static OutlierJobList<kOutBatch> list;   // host staging of the kernel parameter; calls are not re-entrant
+    static OutlierJobList<kOutBatch> list;   // host staging of the kernel parameter (kept off the stack)
+    static std::mutex list_mutex;
+    std::lock_guard<std::mutex> lock(list_mutex);
     char* wsp = static_cast<char*>(ws);
     int64_t i = 0;
     while (i < n_jobs) {

@@ -32,6 +32,7 @@
 //       between A_lo[j] and A_hi[j] - a few percent of the row - are the
 //       candidates, and only they get an exact fp32 score.
 //   prune_rows_kernel       any dtype, any shape; scores of all entries in fp32.
+#include <mutex>
 #include <vector>
 
 #include "select.cuh"
@@ -1094,7 +1095,9 @@ extern "C" int mosaic_prune_unstructured_batch(const mosaic_prune_job* jobs, int
         plan_off[(size_t)i] = off;
         off += batch_plan_bytes(jobs[i], dtype);
     }
-    static PruneJobList<kBatchJobs> list;   // host staging of the kernel parameter; calls are not re-entrant
+    static PruneJobList<kBatchJobs> list;   // host staging of the kernel parameter (18 KB: kept off the stack)
+    static std::mutex list_mutex;
+    std::lock_guard<std::mutex> lock(list_mutex);
     for (int64_t i = 0; i < n_jobs; ++i) {
         if (done[(size_t)i]) continue;
         const mosaic_prune_job& lead = jobs[i];
