@@ -158,6 +158,30 @@ def test_outlier_ratio_batch_matches_oracle_job_by_job(dtype):
             assert s1.cpu().numpy().tobytes() == sums[i:i + 1].cpu().numpy().tobytes()
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_outlier_ratio_uneven_rows_and_dense_threshold(dtype):
+    # rows of very different scale (a sample of rows would misjudge the mean), and a matrix whose
+    # scores all sit within 3 % of the threshold
+    rows, cols = 1100, 2048
+    W = make(rows, cols, dtype, seed=321).clone()
+    W[::3] *= 40.0                      # every third row is large; the sample sees a different mix
+    W[5::7, ::5] *= 300.0
+    norms = norms_for(cols, 70)
+    for alpha in (2.0, 5.0, 9.0):
+        ref = oracle.outlier_ratio(host(W), norms.cpu().numpy(), alpha, dtype)
+        cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+        api.mosaic_outlier_ratio(W, norms, alpha, cnt)
+        assert ref["certified"] and cnt.item() == ref["count"], alpha
+    # all weights equal up to 3 %, alpha = 1: the threshold cuts through the bulk of the scores
+    g = torch.Generator(device="cpu").manual_seed(5)
+    W2 = ((1.0 + 0.03 * torch.rand(600, 2048, generator=g)) * 0.5).to(W.dtype).to(DEV)
+    ones = torch.ones(2048, dtype=torch.float32, device=DEV)
+    ref = oracle.outlier_ratio(host(W2), ones.cpu().numpy(), 1.0, dtype)
+    cnt = torch.zeros(1, dtype=torch.int64, device=DEV)
+    api.mosaic_outlier_ratio(W2, ones, 1.0, cnt)
+    assert ref["certified"] and cnt.item() == ref["count"] and 0 < ref["count"] < 600 * 2048
+
+
 def test_outlier_planted_and_constant():
     rows, cols = 64, 1024
     W = torch.ones(rows, cols, dtype=torch.bfloat16, device=DEV)
