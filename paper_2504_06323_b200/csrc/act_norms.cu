@@ -12,7 +12,8 @@ __global__ void act_finish_kernel(const double* __restrict__ partial, int splits
     const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (c >= cols) return;
     double s = reset ? 0.0 : sumsq[c];
-    for (int p = 0; p < splits; ++p) s += partial[(int64_t)p * cols + c];
+#pragma unroll 16
+    for (int p = 0; p < splits; ++p) s += partial[(int64_t)p * cols + c];   // loads batched, adds in split order
     sumsq[c] = s;
     if (norms_out) norms_out[c] = (float)sqrt(s);
 }

@@ -2,26 +2,35 @@
 // pruning (Section 4.1.3; Section 2.3) - unit scores, exact ranking of units,
 // dense compaction.
 //
-//   scores : row sums (one warp per row, fp64, fixed butterfly) and column sums
-//            (the two-stage column reduction shared with the activation norms),
-//            then one fp64 sum per unit over its rows / columns in index order,
-//            rounded once to fp32.
+//   scores : one sweep over W in tiles of 256 columns x 256 rows.  A lane owns 8
+//            adjacent columns: it adds every score to its column accumulators
+//            and to the row's partial sum (fp64); a row's partial over a chunk
+//            is combined by a fixed butterfly, the chunks of a row in chunk
+//            order, the warps' and the bands' column partials in index order.  One fp64 sum per unit over its rows / columns in
+//            index order follows, rounded once to fp32.
 //   rank   : one CTA per dimension; 4 x 8-bit radix select on the fp32 score
 //            bits finds the threshold key and tie quota; an ordered block scan
 //            then emits the ascending keep list (ties: lowest index removed
 //            first).
-//   compact: one CTA per output row; each thread gathers 8 output elements
-//            through the kept-column map and stores 16 bytes.
+//   compact: one CTA per output row: the source row is staged in shared memory
+//            with coalesced 16-byte loads, every thread then gathers 8 output
+//            elements from it through the kept-column list and stores 16 bytes.
 #include "colreduce.cuh"
 
 namespace mosaic {
 
 constexpr int kRankThreads = 1024;
 
+constexpr int kSTileCols = 256;    // columns per tile: one warp row of 32 lanes x 8 columns
+constexpr int kSTileRows = 256;    // rows per tile, dealt round-robin to the CTA's warps
+constexpr int kSThreads = 128;
+constexpr int kSWarps = kSThreads / 32;
+
 struct StructWs {  // carve-up of the caller's workspace
-    double* row_sum;      // [rows]
-    double* col_partial;  // [splits, cols]
+    double* row_partial;  // [chunks, rows]
+    double* col_partial;  // [bands, cols]
     float* scores;        // [n_ru + n_cu]
+    int chunks, bands;
     size_t bytes;
 };
 
@@ -29,56 +38,97 @@ static StructWs struct_ws(void* base, int64_t rows, int64_t cols) {
     StructWs w;
     char* p = static_cast<char*>(base);
     size_t off = 0;
-    w.row_sum = reinterpret_cast<double*>(p + off);
-    off += align_up(sizeof(double) * (size_t)rows, 256);
-    const ColSplit cs = col_split_plan(rows, cols);
+    w.chunks = (int)((cols + kSTileCols - 1) / kSTileCols);
+    w.bands = (int)((rows + kSTileRows - 1) / kSTileRows);
+    w.row_partial = reinterpret_cast<double*>(p + off);
+    off += align_up(sizeof(double) * (size_t)w.chunks * (size_t)rows, 256);
     w.col_partial = reinterpret_cast<double*>(p + off);
-    off += align_up(sizeof(double) * (size_t)cs.splits * (size_t)cols, 256);
+    off += align_up(sizeof(double) * (size_t)w.bands * (size_t)cols, 256);
     w.scores = reinterpret_cast<float*>(p + off);
     off += align_up(sizeof(float) * (size_t)(rows + cols), 256);
     w.bytes = off;
     return w;
 }
 
-// One warp per row: fp64 sum of the weight metric along the row.
+// One tile per CTA (blockIdx.x = column chunk of 256, blockIdx.y = row band of 256).  Every warp
+// covers the chunk's 256 columns (a lane owns 8 adjacent ones) and takes every fourth row of the
+// band: the row's partial sum over the chunk is one butterfly away, and the lane's column
+// accumulators are combined over the four warps in warp order at the end.  All sums in fp64.
 template <int DT>
-__global__ void __launch_bounds__(256) row_sum_kernel(const void* __restrict__ W, int64_t rows, int64_t cols, int64_t ldw,
-                                                       const float* __restrict__ norms, double* __restrict__ row_sum) {
-    const int lane = threadIdx.x & 31;
-    const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-    const int64_t nvec = (cols + kVec - 1) / kVec;
-    for (int64_t row = warp; row < rows; row += nwarps) {
-        double acc = 0.0;
-        for (int64_t v = lane; v < nvec; v += 32) {
-            Raw8<DT> r;
-            const int64_t c0 = v * kVec;
-            load_vec<DT, true>(r, W, row * ldw, c0, cols);
+__global__ void __launch_bounds__(kSThreads) unit_partial_kernel(const void* __restrict__ W, int64_t rows, int64_t cols,
+                                                                  int64_t ldw, const float* __restrict__ norms,
+                                                                  double* __restrict__ row_partial,
+                                                                  double* __restrict__ col_partial) {
+    __shared__ double cp[kSWarps][kSTileCols + 2];
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const int64_t c0 = (int64_t)blockIdx.x * kSTileCols + lane * kVec;
+    const int64_t r0 = (int64_t)blockIdx.y * kSTileRows;
+    const int64_t r1 = (r0 + kSTileRows < rows) ? r0 + kSTileRows : rows;
+    float nrm[kVec];
+    double acc[kVec];
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) {
+        acc[e] = 0.0;
+        nrm[e] = (c0 + e < cols) ? (norms ? norms[c0 + e] : 1.0f) : 0.0f;
+    }
+    constexpr int U = 4;   // rows in flight per warp
+    for (int64_t r = r0 + wid; r < r1; r += U * kSWarps) {
+        Raw8<DT> v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t rr = r + u * kSWarps;
+            if (rr < r1 && c0 < cols) load_vec<DT, true>(v[u], W, rr * ldw, c0, cols);
+            else v[u].clear();
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t rr = r + u * kSWarps;
+            double p = 0.0;
 #pragma unroll
             for (int e = 0; e < kVec; ++e) {
-                const float n = (c0 + e < cols) ? (norms ? norms[c0 + e] : 1.0f) : 0.0f;
-                acc += (double)__fmul_rn(n, r.abs_f32(e));
+                const double s = (double)__fmul_rn(nrm[e], v[u].abs_f32(e));
+                acc[e] += s;
+                p += s;
             }
+            p = warp_sum(p);
+            if (lane == 0 && rr < r1) row_partial[(int64_t)blockIdx.x * rows + rr] = p;
         }
-        acc = warp_sum(acc);
-        if (lane == 0) row_sum[row] = acc;
+    }
+#pragma unroll
+    for (int e = 0; e < kVec; ++e) cp[wid][lane * kVec + e] = acc[e];
+    __syncthreads();
+    for (int i = threadIdx.x; i < kSTileCols; i += kSThreads) {
+        const int64_t c = (int64_t)blockIdx.x * kSTileCols + i;
+        if (c < cols) {
+            double s = 0.0;
+#pragma unroll
+            for (int w = 0; w < kSWarps; ++w) s += cp[w][i];
+            col_partial[(int64_t)blockIdx.y * cols + c] = s;
+        }
     }
 }
 
-// Unit score = fp64 sum of the unit's row sums (or of its columns' split partials), -> fp32.
-__global__ void unit_score_kernel(const double* __restrict__ row_sum, int64_t n_ru, int64_t row_group,
-                                  const double* __restrict__ col_partial, int splits, int64_t cols, int64_t n_cu,
-                                  int64_t col_group, float* __restrict__ out, int accumulate) {
+// Unit score = fp64 sum over the unit's rows (chunk partials in chunk order) or columns (band
+// partials in band order), in index order, rounded once to fp32.
+__global__ void unit_score_kernel(const double* __restrict__ row_partial, int chunks, int64_t rows, int64_t n_ru,
+                                  int64_t row_group, const double* __restrict__ col_partial, int bands, int64_t cols,
+                                  int64_t n_cu, int64_t col_group, float* __restrict__ out, int accumulate) {
     const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (u >= n_ru + n_cu) return;
     double s = 0.0;
     if (u < n_ru) {
-        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i) s += row_sum[i];
+        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i) {
+            double rs = 0.0;
+#pragma unroll 8
+            for (int p = 0; p < chunks; ++p) rs += row_partial[(int64_t)p * rows + i];
+            s += rs;
+        }
     } else {
         const int64_t v = u - n_ru;
         for (int64_t c = v * col_group; c < (v + 1) * col_group; ++c) {
             double cs = 0.0;
-            for (int p = 0; p < splits; ++p) cs += col_partial[(int64_t)p * cols + c];
+#pragma unroll 16
+            for (int p = 0; p < bands; ++p) cs += col_partial[(int64_t)p * cols + c];   // loads batched, adds in order
             s += cs;
         }
     }
@@ -113,16 +163,30 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
                 if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFFu], 1u);
             }
             __syncthreads();
-            if (tid == 0) {
-                int64_t cum = 0;
-                for (int b = 0; b < 256; ++b) {
-                    if (rank <= cum + (int64_t)hist[b]) {
-                        sel_bin = (uint32_t)b;
-                        sel_rank = (uint32_t)(rank - cum);
-                        sel_cnt = hist[b];
-                        break;
+            if (wid == 0) {   // warp 0: 8 bins per lane, prefix over the lanes, then inside the lane that holds the rank
+                uint32_t c[8], sum = 0u;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    c[i] = hist[lane * 8 + i];
+                    sum += c[i];
+                }
+                uint32_t incl = sum;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += n;
+                }
+                int64_t cum = (int64_t)(incl - sum);
+                if (cum < rank && rank <= cum + (int64_t)sum) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        if (cum < rank && rank <= cum + (int64_t)c[i]) {
+                            sel_bin = (uint32_t)(lane * 8 + i);
+                            sel_rank = (uint32_t)(rank - cum);
+                            sel_cnt = c[i];
+                        }
+                        cum += c[i];
                     }
-                    cum += hist[b];
                 }
             }
             __syncthreads();
@@ -201,16 +265,29 @@ __global__ void __launch_bounds__(kRankThreads) rank_kernel(const float* row_sco
     }
 }
 
-// Dense gather.  grid.x = output rows; threads walk output vectors of 8 elements.
+// Dense gather.  grid.x = output rows.  The source row is staged in shared memory (dynamic,
+// cols elements) with 16-byte loads; threads then walk output vectors of 8 elements.
 template <int DT>
-__global__ void __launch_bounds__(256) compact_kernel(const void* __restrict__ W, int64_t ldw, const int32_t* __restrict__ row_keep,
-                                                       int64_t n_ru, int64_t row_group, const int32_t* __restrict__ col_keep,
-                                                       int64_t n_cu, int64_t col_group, int64_t out_cols, void* __restrict__ out) {
+__global__ void __launch_bounds__(256) compact_kernel(const void* __restrict__ W, int64_t cols, int64_t ldw,
+                                                       const int32_t* __restrict__ row_keep, int64_t n_ru, int64_t row_group,
+                                                       const int32_t* __restrict__ col_keep, int64_t n_cu, int64_t col_group,
+                                                       int64_t out_cols, void* __restrict__ out) {
+    extern __shared__ __align__(16) unsigned char srow[];
     constexpr int esz = (DT == MOSAIC_F32) ? 4 : 2;
     const int64_t a = blockIdx.x;
     int64_t ru = row_keep[a / row_group];
     ru = ru < 0 ? 0 : (ru >= n_ru ? n_ru - 1 : ru);
     const int64_t src_row = ru * row_group + a % row_group;
+    const int64_t in_vec = (cols + kVec - 1) / kVec;
+    for (int64_t v = threadIdx.x; v < in_vec; v += blockDim.x) {
+        Raw8<DT> r;
+        load_vec<DT, true>(r, W, src_row * ldw, v * kVec, cols);
+        uint4* dst = reinterpret_cast<uint4*>(srow + v * kVec * esz);
+        dst[0] = make_uint4(r.w[0], r.w[1], r.w[2], r.w[3]);
+        if (DT == MOSAIC_F32) dst[1] = make_uint4(r.w[4 % (Raw8<DT>::kBytes / 4)], r.w[5 % (Raw8<DT>::kBytes / 4)],
+                                                  r.w[6 % (Raw8<DT>::kBytes / 4)], r.w[7 % (Raw8<DT>::kBytes / 4)]);
+    }
+    __syncthreads();
     const int64_t nvec = (out_cols + kVec - 1) / kVec;
     const bool vec_ok = (out_cols % kVec) == 0;   // every output row then starts 16-byte aligned
     for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
@@ -224,7 +301,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const void* __restrict__ W
                 int64_t cu = (col_group == 1) ? (int64_t)col_keep[b] : (int64_t)col_keep[b / col_group];
                 cu = cu < 0 ? 0 : (cu >= n_cu ? n_cu - 1 : cu);
                 const int64_t j = (col_group == 1) ? cu : cu * col_group + b % col_group;
-                r.set_scalar(e, W, src_row * ldw + j);
+                r.set_scalar(e, srow, j);
             }
         }
         if (vec_ok) {
@@ -311,28 +388,17 @@ extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, i
         if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
         if (ws_bytes < mosaic_prune_structured_compact_workspace_bytes(rows, cols)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
         w = struct_ws(ws, rows, cols);
-        const ColSplit cs = col_split_plan(rows, cols);
-        int64_t rblocks = (rows + 7) / 8;
-        const int64_t cap = (int64_t)sm_count() * 8;
-        if (rblocks > cap) rblocks = cap;
-        dim3 cgrid((unsigned)((cols + kColTile - 1) / kColTile), (unsigned)cs.splits);
-        if (dtype == MOSAIC_BF16) {
-            row_sum_kernel<MOSAIC_BF16><<<(unsigned)rblocks, 256, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_sum);
-            MOSAIC_LAUNCH_CHECK();
-            col_partial_kernel<MOSAIC_BF16, COL_SCORE><<<cgrid, kColTile, 0, st>>>(W_in, rows, cols, ldw, norms,
-                                                                                   cs.rows_per_split, w.col_partial);
-        } else {
-            row_sum_kernel<MOSAIC_F32><<<(unsigned)rblocks, 256, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_sum);
-            MOSAIC_LAUNCH_CHECK();
-            col_partial_kernel<MOSAIC_F32, COL_SCORE><<<cgrid, kColTile, 0, st>>>(W_in, rows, cols, ldw, norms,
-                                                                                  cs.rows_per_split, w.col_partial);
-        }
+        dim3 grid((unsigned)w.chunks, (unsigned)w.bands);
+        if (dtype == MOSAIC_BF16)
+            unit_partial_kernel<MOSAIC_BF16><<<grid, kSThreads, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_partial, w.col_partial);
+        else
+            unit_partial_kernel<MOSAIC_F32><<<grid, kSThreads, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_partial, w.col_partial);
         MOSAIC_LAUNCH_CHECK();
         // with SCORES_ACCUM the running totals live in the caller's array; ranking then uses those
         float* dst = (flags & MOSAIC_SCORES_ACCUM) ? unit_scores_out : w.scores;
         const int64_t nu = n_ru + n_cu;
-        unit_score_kernel<<<(unsigned)((nu + 127) / 128), 128, 0, st>>>(w.row_sum, n_ru, row_group, w.col_partial, cs.splits,
-                                                                       cols, n_cu, col_group, dst,
+        unit_score_kernel<<<(unsigned)((nu + 127) / 128), 128, 0, st>>>(w.row_partial, w.chunks, rows, n_ru, row_group,
+                                                                       w.col_partial, w.bands, cols, n_cu, col_group, dst,
                                                                        (flags & MOSAIC_SCORES_ACCUM) ? 1 : 0);
         MOSAIC_LAUNCH_CHECK();
         if (unit_scores_out && dst != unit_scores_out)
@@ -348,12 +414,22 @@ extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, i
     }
     if (rank_only) return MOSAIC_OK;
 
+    const size_t row_smem = align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
+    if (row_smem > 200 * 1024) return MOSAIC_ERR_INVALID_ARG;   // a source row must fit in shared memory (cols <= 51200 fp32)
+    static bool attr_set[2] = {false, false};
+    if (!attr_set[dtype == MOSAIC_BF16]) {
+        const cudaError_t e = (dtype == MOSAIC_BF16)
+            ? cudaFuncSetAttribute(compact_kernel<MOSAIC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+            : cudaFuncSetAttribute(compact_kernel<MOSAIC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) return MOSAIC_ERR_CUDA;
+        attr_set[dtype == MOSAIC_BF16] = true;
+    }
     if (dtype == MOSAIC_BF16)
-        compact_kernel<MOSAIC_BF16><<<(unsigned)out_rows, 256, 0, st>>>(W_in, ldw, row_keep_units, n_ru, row_group,
-                                                                       col_keep_units, n_cu, col_group, out_cols, W_out);
+        compact_kernel<MOSAIC_BF16><<<(unsigned)out_rows, 256, row_smem, st>>>(W_in, cols, ldw, row_keep_units, n_ru, row_group,
+                                                                              col_keep_units, n_cu, col_group, out_cols, W_out);
     else
-        compact_kernel<MOSAIC_F32><<<(unsigned)out_rows, 256, 0, st>>>(W_in, ldw, row_keep_units, n_ru, row_group,
-                                                                      col_keep_units, n_cu, col_group, out_cols, W_out);
+        compact_kernel<MOSAIC_F32><<<(unsigned)out_rows, 256, row_smem, st>>>(W_in, cols, ldw, row_keep_units, n_ru, row_group,
+                                                                             col_keep_units, n_cu, col_group, out_cols, W_out);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
