@@ -517,6 +517,11 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
     uint32_t* qkey = reinterpret_cast<uint32_t*>(rowbuf + RING * V * nt) + wid * kQueueCap;
     uint32_t* gone_w = reinterpret_cast<uint32_t*>(rowbuf + RING * V * nt) + nwarps * kQueueCap;
     uint16_t* qid = reinterpret_cast<uint16_t*>(gone_w + nt) + wid * kQueueCap;
+    // Keep-bitmask bytes of a finished row wait here (two rows' worth, alternating) and leave as
+    // 4-byte stores after the next block barrier: single-byte global stores cost a third of the row time.
+    uint8_t* mask_stage = reinterpret_cast<uint8_t*>(reinterpret_cast<uint16_t*>(gone_w + nt) + nwarps * kQueueCap);
+    uint32_t* pending_mask = nullptr;   // where the staged bytes go (block-uniform), or nullptr
+    int pending_slot = 0, stage_slot = 0;
     __shared__ uint32_t q_overflow;
 
     gone_w[tid] = 0u;
@@ -569,10 +574,20 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         return __float_as_uint(__fmul_rn(__ldg(norms + (v * nt + tid) * kVec + e), __uint_as_float(a)));
     };
 
+    // Stores the staged mask row.  Call only after a block barrier that follows the staging.
+    auto flush_mask = [&]() {
+        if (pending_mask != nullptr) {
+            if (tid * 4 < mask_row_bytes)
+                pending_mask[tid] = reinterpret_cast<const uint32_t*>(mask_stage + pending_slot * V * nt)[tid];
+            pending_mask = nullptr;
+        }
+    };
+
     // Key of the matching quantile of one key per thread (element 0 of vector 0), or 0.
     auto sample_center = [&](int cur) -> uint32_t {
         list[tid] = cand_key(cur, 0, 0);
         __syncthreads();
+        flush_mask();
         if (wid == 0) {
             uint32_t r_s = (uint32_t)(((uint64_t)uk * (uint32_t)nt + (uint32_t)cols / 2u) / (uint32_t)cols);
             r_s = r_s < 1u ? 1u : (r_s > (uint32_t)nt ? (uint32_t)nt : r_s);
@@ -647,6 +662,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         below = __reduce_add_sync(0xFFFFFFFFu, below);
         if (lane == 0) red[wid] = below;
         __syncthreads();
+        flush_mask();
         if (wid == 0) {
             const uint32_t n_below = __reduce_add_sync(0xFFFFFFFFu, (lane < nwarps) ? red[lane] : 0u);
             const uint32_t cc = coarse[lane];
@@ -756,14 +772,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 o.w = r.w & lane_mask_from_flags((r.w | 0x80008000u) - Alo[v][3]);
                 st_stream16(out_row + (int64_t)vec * kVec, o);
             }
-            if (mask_bytes != nullptr && vec < mask_row_bytes) {
+            if (mask_bytes != nullptr) {
                 uint32_t keep = 0u;
                 if (vec < nvec) {
                     const uint32_t rr = __brev(keepf[v] & ~gone);   // odd elements on bits 0..3, even ones on bits 16..19
                     keep = (uint32_t)spread[(rr >> 16) & 0xFu] | ((uint32_t)spread[rr & 0xFu] << 1);
                 }
-                mask_bytes[row * mask_row_bytes + vec] = (uint8_t)keep;
+                mask_stage[stage_slot * V * nt + vec] = (uint8_t)keep;   // slots past the row's end hold the padding zeros
             }
+        }
+        if (mask_bytes != nullptr) {
+            pending_mask = reinterpret_cast<uint32_t*>(mask_bytes + row * mask_row_bytes);
+            pending_slot = stage_slot;
+            stage_slot ^= 1;
         }
         T_out = T;
         return 0;
@@ -831,11 +852,14 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
             MOSAIC_STAT(5);
             for (int b = tid; b < kWinBins; b += nt) slot[b] = 0u;
             __syncthreads();
+            flush_mask();
             T_row = generic_row_bf16<V>(&rowbuf[(cur * V) * nt + tid], nt, norms, cols, nvec, uk, buf, warp_tot, &sel3, W_out,
                                         row * ldw, mask_bytes, row * mask_row_bytes, mask_row_bytes);
         }
         if (all_finite && (status != 0 || win_w != kTrackBits)) set_window(T_row, kTrackBits);
     }
+    __syncthreads();
+    flush_mask();
 }
 
 // One CTA per job: the exact thresholds of three rows (first, middle, last) by the full radix
@@ -900,9 +924,11 @@ __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_const
     }
 }
 
-// Row ring (`ring` rows of kFastV*nt vectors), per-warp queues (key + id per entry), one word per thread.
+// Row ring (`ring` rows of kFastV*nt vectors), per-warp queues (key + id per entry), one word per thread,
+// two staged mask rows.
 static size_t fast_dyn_smem(int nt, int ring) {
-    return (size_t)ring * kFastV * nt * sizeof(uint4) + (size_t)(nt / 32) * kQueueCap * 6 + (size_t)nt * 4;
+    return (size_t)ring * kFastV * nt * sizeof(uint4) + (size_t)(nt / 32) * kQueueCap * 6 + (size_t)nt * 4 +
+           (size_t)2 * kFastV * nt;
 }
 
 // Launches the pruning kernel (and, with_plan, the planning kernel before it) over a list of jobs.
