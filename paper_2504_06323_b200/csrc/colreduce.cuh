@@ -6,8 +6,8 @@
 //            The 8 row lanes are combined in shared memory in lane order and
 //            one fp64 partial per (split, column) is written.
 //   stage 2: the caller adds the partials of a column in split order.
-// The value reduced is either x^2 (activation norms, Eq. 5's ||A||_2 term) or
-// the weight metric norm_j*|w_ij| (column unit scores of structured pruning).
+// The value reduced is x^2 (activation norms, Eq. 5's ||A||_2 term); the COL_SCORE variant
+// (norm_j*|w_ij|) is kept for callers that want column sums of the weight metric alone.
 #pragma once
 #include "common.cuh"
 

@@ -15,7 +15,7 @@
 //   compact: one CTA per output row: the source row is staged in shared memory
 //            with coalesced 16-byte loads, every thread then gathers 8 output
 //            elements from it through the kept-column list and stores 16 bytes.
-#include "colreduce.cuh"
+#include "common.cuh"
 
 namespace mosaic {
 
