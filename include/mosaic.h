@@ -62,6 +62,9 @@ typedef enum mosaic_dtype { MOSAIC_F32 = 0, MOSAIC_BF16 = 1 } mosaic_dtype;
 /* mode of mosaic_allocate_sparsity */
 #define MOSAIC_GLOBAL_NORM 0       /* normalise ranks over all N*M projections            */
 #define MOSAIC_PER_CATEGORY_NORM 1 /* normalise separately over the N entries of each m   */
+#define MOSAIC_WEIGHTED_MEAN 2     /* flag, or-ed in: the targets average to p weighted by
+                                      each projection's parameter count, so the pruned share
+                                      of all parameters is p (Eq. 1-2 use the plain mean)   */
 
 /* flags of mosaic_prune_structured_compact */
 #define MOSAIC_ROWS_GIVEN 1    /* row_keep_units is an input (ascending unit indices)      */
@@ -183,7 +186,8 @@ int mosaic_outlier_ratio_static(const void *W, int64_t rows, int64_t cols, int64
  * The paper states only the properties (targets average to p; more outliers
  * => pruned less).  Definition used, fp64, loops in q order:
  *     R_q = 100*O_q/C_q;  lo = min R, hi = max R;  hi == lo -> s_q = p
- *     r_q = (R_q-lo)/(hi-lo);  d_q = 2*lambda*r_q;  dbar = (sum_q d_q)/count
+ *     r_q = (R_q-lo)/(hi-lo);  d_q = 2*lambda*r_q;  dbar = (sum_q w_q d_q)/(sum_q w_q)
+ *     (w_q = 1, or C_q with MOSAIC_WEIGHTED_MEAN)
  *     s_q = (p + dbar) - d_q, clamped to [0, 1 - 1/cols_q]
  *     k_q = floor(s_q * cols_q)       (weights removed from every row)
  * MOSAIC_PER_CATEGORY_NORM applies the same over the n_layers entries of each

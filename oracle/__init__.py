@@ -22,6 +22,7 @@ _SO = os.path.join(_HERE, "libmosaic_oracle.so")
 
 F32, BF16 = 0, 1
 MODE_GLOBAL_NORM, MODE_PER_CATEGORY_NORM = 0, 1
+MODE_WEIGHTED_MEAN = 2      # flag, or-ed into the mode
 
 
 def build(force: bool = False) -> str:

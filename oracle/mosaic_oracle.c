@@ -203,8 +203,12 @@ void oracle_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw
  * (Section 3.1).  Reading taken: min-max normalise the ranks R_q = 100*O_q/C_q
  * to r_q in [0,1]; give each projection the deviation d_q = 2*lambda*r_q;
  * s_q = p + mean(d) - d_q.  Then mean(s) = p, s decreases in R, and
- * max(s)-min(s) = 2*lambda.  mode 0 normalises over all N*M entries, mode 1
- * separately over the N entries of each projection category m.
+ * max(s)-min(s) = 2*lambda.  mode bit 0: 0 normalises over all N*M entries, 1
+ * separately over the N entries of each projection category m.  mode bit 1:
+ * the mean in "targets average to p" weighs every projection by its number of
+ * parameters C_q (mean(d) = sum C_q d_q / sum C_q), so that the pruned share
+ * of all parameters of the group is p; without it the mean is the plain one of
+ * Eq. 1-2.
  * s is clamped to [0, 1 - 1/cols_q]; k_q = floor(s_q * cols_q) weights are
  * removed from every row.  Returns 0, or 1 if any clamp was applied.
  */
@@ -218,12 +222,13 @@ int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numel
     for (int q = 0; q < total; ++q)
         R[q] = 100.0 * (double)outlier_counts[q] / (double)numels[q];
 
-    int n_groups = (mode == 1) ? n_proj : 1;
+    int per_category = mode & 1, weighted = (mode >> 1) & 1;
+    int n_groups = per_category ? n_proj : 1;
     for (int g = 0; g < n_groups; ++g) {
         /* members of this normalisation group, in q order */
-        int first = (mode == 1) ? g : 0;
-        int step = (mode == 1) ? n_proj : 1;
-        int count = (mode == 1) ? n_layers : total;
+        int first = per_category ? g : 0;
+        int step = per_category ? n_proj : 1;
+        int count = per_category ? n_layers : total;
 
         double lo = R[first], hi = R[first];
         for (int c = 0, q = first; c < count; ++c, q += step) {
@@ -235,13 +240,15 @@ int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numel
                 sparsity[q] = p;
             continue;
         }
-        double dsum = 0.0;
+        double dsum = 0.0, wsum = 0.0;
         for (int c = 0, q = first; c < count; ++c, q += step) {
             double r = (R[q] - lo) / (hi - lo);
             double d = 2.0 * lambda * r;
-            dsum = dsum + d;
+            double w = weighted ? (double)numels[q] : 1.0;
+            dsum = dsum + w * d;
+            wsum = wsum + w;
         }
-        double dbar = dsum / (double)count;
+        double dbar = dsum / wsum;
         for (int c = 0, q = first; c < count; ++c, q += step) {
             double r = (R[q] - lo) / (hi - lo);
             double d = 2.0 * lambda * r;

@@ -20,6 +20,7 @@ LIB_PATH = os.path.join(_HERE, "libmosaic.so")
 F32, BF16 = 0, 1
 RESET_ACCUM = 1
 GLOBAL_NORM, PER_CATEGORY_NORM = 0, 1
+WEIGHTED_MEAN = 2        # flag, or-ed into the mode
 ROWS_GIVEN, COLS_GIVEN, RANK_ONLY, SCORES_ONLY, SCORES_ACCUM = 1, 2, 4, 8, 16
 OK, ERR_INFEASIBLE = 0, -9
 

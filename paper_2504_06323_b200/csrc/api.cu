@@ -66,15 +66,16 @@ int mosaic_allocate_sparsity(const int64_t* outlier_counts, const int64_t* numel
                              double* sparsity_out, int64_t* k_out) {
     if (!outlier_counts || !numels || !cols || !sparsity_out || !k_out) return MOSAIC_ERR_NULL_PTR;
     if (n_layers <= 0 || n_proj <= 0 || !(p >= 0.0 && p < 1.0) || !(lambda >= 0.0)) return MOSAIC_ERR_INVALID_ARG;
-    if (mode != MOSAIC_GLOBAL_NORM && mode != MOSAIC_PER_CATEGORY_NORM) return MOSAIC_ERR_INVALID_ARG;
+    if (mode & ~(MOSAIC_PER_CATEGORY_NORM | MOSAIC_WEIGHTED_MEAN)) return MOSAIC_ERR_INVALID_ARG;
+    const bool per_category = (mode & MOSAIC_PER_CATEGORY_NORM) != 0, weighted = (mode & MOSAIC_WEIGHTED_MEAN) != 0;
     const int total = n_layers * n_proj;
     for (int q = 0; q < total; ++q)
         if (numels[q] <= 0 || cols[q] <= 0 || outlier_counts[q] < 0 || outlier_counts[q] > numels[q])
             return MOSAIC_ERR_INVALID_ARG;
 
-    const int n_groups = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_proj : 1;
-    const int stride = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_proj : 1;
-    const int members = (mode == MOSAIC_PER_CATEGORY_NORM) ? n_layers : total;
+    const int n_groups = per_category ? n_proj : 1;
+    const int stride = per_category ? n_proj : 1;
+    const int members = per_category ? n_layers : total;
     for (int g = 0; g < n_groups; ++g) {
         double lo = 0.0, hi = 0.0;
         for (int c = 0; c < members; ++c) {
@@ -88,14 +89,16 @@ int mosaic_allocate_sparsity(const int64_t* outlier_counts, const int64_t* numel
             continue;
         }
         const double range = hi - lo;
-        double dsum = 0.0;
+        double dsum = 0.0, wsum = 0.0;
         for (int c = 0; c < members; ++c) {
             const int q = g + c * stride;
             const double r = (mosaic_ratio_from_count(outlier_counts[q], numels[q]) - lo) / range;
             const double d = 2.0 * lambda * r;
-            dsum = dsum + d;
+            const double w = weighted ? (double)numels[q] : 1.0;
+            dsum = dsum + w * d;
+            wsum = wsum + w;
         }
-        const double dbar = dsum / (double)members;
+        const double dbar = dsum / wsum;
         for (int c = 0; c < members; ++c) {
             const int q = g + c * stride;
             const double r = (mosaic_ratio_from_count(outlier_counts[q], numels[q]) - lo) / range;

@@ -62,7 +62,8 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.mosaic_act_norms_workspace_bytes(262144, 4096) % 256 == 0
 
 
-@pytest.mark.parametrize("mode", [api.GLOBAL_NORM, api.PER_CATEGORY_NORM])
+@pytest.mark.parametrize("mode", [api.GLOBAL_NORM, api.PER_CATEGORY_NORM, api.GLOBAL_NORM | api.WEIGHTED_MEAN,
+                                  api.PER_CATEGORY_NORM | api.WEIGHTED_MEAN])
 @pytest.mark.parametrize("p,lam", [(0.5, 0.08), (0.8, 0.15), (0.1, 0.0), (0.7, 0.3)])
 def test_allocate_sparsity_bit_exact_vs_oracle(lib, mode, p, lam):
     rng = np.random.default_rng(42)

@@ -416,3 +416,31 @@ def test_tiny_config_outliers_sit_in_planted_columns():
         inside = (S[:, cols] > tau).sum()
         assert (S > tau).sum() == r["count"]
         assert inside >= 0.99 * r["count"] > 0
+
+
+@pytest.mark.parametrize("base", [oracle.MODE_GLOBAL_NORM, oracle.MODE_PER_CATEGORY_NORM])
+def test_allocation_weighted_mean_prunes_exactly_p_of_the_parameters(base):
+    # with the parameter-weighted mean the pruned share of all parameters (of each normalisation
+    # group) is p; the spread, the order and the equal-size special case are unchanged
+    rng = np.random.default_rng(7)
+    N, M, p, lam = 6, 7, 0.6, 0.1
+    numel = np.tile(np.array([16, 16, 16, 16, 43, 43, 43]) * 1_000_000, N).astype(np.int64)
+    cols = np.tile(np.array([4096] * 6 + [11008]), N).astype(np.int64)
+    O = (numel * rng.uniform(0.001, 0.03, N * M)).astype(np.int64)
+    s, k, clamped = oracle.allocate_sparsity(O, numel, cols, N, M, p, lam, base | oracle.MODE_WEIGHTED_MEAN)
+    assert not clamped
+    groups = [np.arange(N * M)] if base == 0 else [np.arange(N) * M + m for m in range(M)]
+    R = 100.0 * O / numel
+    for g in groups:
+        assert abs(np.sum(s[g] * numel[g]) / np.sum(numel[g]) - p) < 1e-12
+        assert abs((s[g].max() - s[g].min()) - 2 * lam) < 1e-12
+        order = np.argsort(R[g])
+        assert (np.diff(s[g][order]) <= 1e-15).all()
+    s_plain, _, _ = oracle.allocate_sparsity(O, numel, cols, N, M, p, lam, base)
+    if base == 0:
+        assert abs(np.mean(s_plain) - p) < 1e-12 and abs(np.sum(s_plain * numel) / np.sum(numel) - p) > 1e-6
+    # equal sizes: the weighted and the plain mean coincide
+    same = np.full(N * M, 1 << 20, np.int64)
+    a, _, _ = oracle.allocate_sparsity(O % (1 << 20), same, cols, N, M, p, lam, base | oracle.MODE_WEIGHTED_MEAN)
+    b, _, _ = oracle.allocate_sparsity(O % (1 << 20), same, cols, N, M, p, lam, base)
+    np.testing.assert_allclose(a, b, rtol=0, atol=1e-15)
