@@ -13,7 +13,7 @@ from paper_2504_06323_b200 import api, workloads as wl
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
-REL = 1e-5   # tolerance the benchmark spec states for norms and scores in fp32
+REL = 1e-5   # relative tolerance required of norms and scores in fp32
 
 
 def make(rows, cols, dtype, seed, ld=None, scale=0.02, heavy=False):
