@@ -248,28 +248,45 @@ class OutlierJob(C.Structure):
                 ("norms", C.c_void_p), ("outlier_count_out", C.c_void_p), ("score_sum_out", C.c_void_p)]
 
 
+class OutlierBatch:
+    """The marshalled job list of mosaic_outlier_ratio_batch for a list of
+    (W, norms, outlier_count_out[1], score_sum_out[1] or None); the count tensors may be
+    one-element views of a larger int64 tensor.  Checked and laid out once; run() only makes
+    the call, so a caller that repeats the sweep over matrices that stay where they are pays
+    the per-job Python work once.  The tensors are kept alive by the object."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (OutlierJob * len(self.jobs))()
+        dtype = self.jobs[0][0].dtype
+        for i, (W, norms, cnt, ssum) in enumerate(self.jobs):
+            p, rows, cols, ldw = _mat(W, "W")
+            if W.dtype != dtype:
+                raise TypeError("one dtype per batch")
+            _dev(norms, "norms", torch.float32)
+            _dev(cnt, "outlier_count_out", torch.int64)
+            if ssum is not None:
+                _dev(ssum, "score_sum_out", torch.float64)
+            if norms.numel() != cols:
+                raise ValueError("norms must be [cols]")
+            self.arr[i] = OutlierJob(p, rows, cols, ldw, norms.data_ptr(), cnt.data_ptr(), _ptr(ssum))
+        self.code = _dtype_code(self.jobs[0][0])
+        self.device = self.jobs[0][0].device
+        self.ws_bytes = lib().mosaic_outlier_ratio_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs))
+
+    def run(self, alpha: float, ws: Workspace | None = None, stream=None) -> None:
+        wp, wn = _ws(ws, self.device).get(self.ws_bytes)
+        _check(lib().mosaic_outlier_ratio_batch(C.addressof(self.arr), len(self.jobs), self.code, float(alpha), wp, wn,
+                                                _stream(stream)), "mosaic_outlier_ratio_batch")
+
+
 def mosaic_outlier_ratio_batch(jobs, alpha: float, ws: Workspace | None = None, stream=None) -> None:
     """mosaic_outlier_ratio over a list of (W, norms, outlier_count_out[1], score_sum_out[1] or None)
     in two launches; the count tensors may be one-element views of a larger int64 tensor."""
-    if not jobs:
-        return
-    arr = (OutlierJob * len(jobs))()
-    dtype = jobs[0][0].dtype
-    for i, (W, norms, cnt, ssum) in enumerate(jobs):
-        p, rows, cols, ldw = _mat(W, "W")
-        if W.dtype != dtype:
-            raise TypeError("one dtype per batch")
-        _dev(norms, "norms", torch.float32)
-        _dev(cnt, "outlier_count_out", torch.int64)
-        if ssum is not None:
-            _dev(ssum, "score_sum_out", torch.float64)
-        if norms.numel() != cols:
-            raise ValueError("norms must be [cols]")
-        arr[i] = OutlierJob(p, rows, cols, ldw, norms.data_ptr(), cnt.data_ptr(), _ptr(ssum))
-    L = lib()
-    wp, wn = _ws(ws, jobs[0][0].device).get(L.mosaic_outlier_ratio_batch_workspace_bytes(C.addressof(arr), len(jobs)))
-    _check(L.mosaic_outlier_ratio_batch(C.addressof(arr), len(jobs), _dtype_code(jobs[0][0]), float(alpha), wp, wn,
-                                        _stream(stream)), "mosaic_outlier_ratio_batch")
+    if jobs:
+        OutlierBatch(jobs).run(alpha, ws, stream)
 
 
 def mosaic_ratio_from_count(outlier_count: int, numel: int) -> float:
@@ -313,30 +330,51 @@ class PruneJob(C.Structure):
                 ("ldw", C.c_int64), ("norms", C.c_void_p), ("k", C.c_int64), ("mask_out", C.c_void_p)]
 
 
+class PruneBatch:
+    """The marshalled job list of mosaic_prune_unstructured_batch for a list of
+    (W_in, W_out, norms, k, mask_out or None).  Checked and laid out once; run() may replace
+    the per-row prune counts and then only makes the call.  The tensors are kept alive by the object."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (PruneJob * len(self.jobs))()
+        dtype = self.jobs[0][0].dtype
+        for i, (W_in, W_out, norms, k, mask_out) in enumerate(self.jobs):
+            p, rows, cols, ldw = _mat(W_in, "W_in")
+            po, r2, c2, ld2 = _mat(W_out, "W_out")
+            if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or W_in.dtype != dtype or (rows > 1 and ld2 != ldw):
+                raise ValueError("W_out must match W_in in shape, dtype and leading dimension; one dtype per batch")
+            _dev(norms, "norms", torch.float32)
+            if norms.numel() != cols:
+                raise ValueError("norms must be [cols]")
+            if mask_out is not None:
+                _dev(mask_out, "mask_out", torch.int32)
+                if tuple(mask_out.shape) != (rows, (cols + 31) // 32) or not mask_out.is_contiguous():
+                    raise ValueError("mask_out must be a contiguous int32 [rows, ceil(cols/32)]")
+            self.arr[i] = PruneJob(p, po, rows, cols, ldw, norms.data_ptr(), int(k), _ptr(mask_out))
+        self.code = _dtype_code(self.jobs[0][0])
+        self.device = self.jobs[0][0].device
+        self.ws_bytes = lib().mosaic_prune_unstructured_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs), self.code)
+
+    def run(self, k=None, ws: Workspace | None = None, stream=None) -> None:
+        """k: None (the counts given at construction) or one prune count per job."""
+        if k is not None:
+            if len(k) != len(self.jobs):
+                raise ValueError("one k per job")
+            for i, kk in enumerate(k):
+                self.arr[i].k = int(kk)
+            self.ws_bytes = lib().mosaic_prune_unstructured_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs), self.code)
+        wp, wn = _ws(ws, self.device).get(self.ws_bytes)
+        _check(lib().mosaic_prune_unstructured_batch(C.addressof(self.arr), len(self.jobs), self.code, wp, wn, _stream(stream)),
+               "mosaic_prune_unstructured_batch")
+
+
 def mosaic_prune_unstructured_batch(jobs, ws: Workspace | None = None, stream=None) -> None:
     """mosaic_prune_unstructured over a list of (W_in, W_out, norms, k, mask_out or None) in few launches."""
-    if not jobs:
-        return
-    arr = (PruneJob * len(jobs))()
-    dtype = jobs[0][0].dtype
-    for i, (W_in, W_out, norms, k, mask_out) in enumerate(jobs):
-        p, rows, cols, ldw = _mat(W_in, "W_in")
-        po, r2, c2, ld2 = _mat(W_out, "W_out")
-        if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or W_in.dtype != dtype or (rows > 1 and ld2 != ldw):
-            raise ValueError("W_out must match W_in in shape, dtype and leading dimension; one dtype per batch")
-        _dev(norms, "norms", torch.float32)
-        if norms.numel() != cols:
-            raise ValueError("norms must be [cols]")
-        if mask_out is not None:
-            _dev(mask_out, "mask_out", torch.int32)
-            if tuple(mask_out.shape) != (rows, (cols + 31) // 32) or not mask_out.is_contiguous():
-                raise ValueError("mask_out must be a contiguous int32 [rows, ceil(cols/32)]")
-        arr[i] = PruneJob(p, po, rows, cols, ldw, norms.data_ptr(), int(k), _ptr(mask_out))
-    L = lib()
-    code = _dtype_code(jobs[0][0])
-    wp, wn = _ws(ws, jobs[0][0].device).get(L.mosaic_prune_unstructured_batch_workspace_bytes(C.addressof(arr), len(jobs), code))
-    _check(L.mosaic_prune_unstructured_batch(C.addressof(arr), len(jobs), code, wp, wn, _stream(stream)),
-           "mosaic_prune_unstructured_batch")
+    if jobs:
+        PruneBatch(jobs).run(None, ws, stream)
 
 
 def mosaic_prune_structured_compact(W_in: torch.Tensor, norms: torch.Tensor | None, row_group: int, col_group: int,

@@ -82,6 +82,7 @@ class ModelState:
     counts: torch.Tensor | None = None                 # int64 [len(layers)*M]
     ws: api.Workspace | None = None
     ws_batch: api.Workspace | None = None             # holds the plans of the batched pruning call
+    batches: dict = field(default_factory=dict)        # name -> (identity of the tensors, marshalled batch)
 
     def q_local(self, layer: int, proj: str) -> int:
         return self.layers.index(layer) * len(PROJECTIONS) + PROJECTIONS.index(proj)
@@ -136,18 +137,29 @@ def count_outliers(st: ModelState, layer: int, alpha: float | None = None) -> in
     return len(PROJECTIONS)
 
 
+def _cached_batch(st: ModelState, name: str, jobs: list, make):
+    """The marshalled batch for `jobs`, rebuilt only when one of the tensors has been replaced."""
+    ident = tuple(id(t) for job in jobs for t in job if isinstance(t, torch.Tensor))
+    hit = st.batches.get(name)
+    if hit is None or hit[0] != ident:
+        hit = (ident, make(jobs))
+        st.batches[name] = hit
+    return hit[1]
+
+
 def count_outliers_all(st: ModelState, alpha: float | None = None) -> int:
-    """Outlier counts of every owned projection through the batched call (two launches)."""
+    """Outlier counts of every owned projection through the batched call (two launches).  The job
+    list is marshalled once and reused while the tensors of the ModelState stay the same objects."""
     cfg = st.cfg
     a = cfg.alpha if alpha is None else alpha
-    jobs = []
-    for layer in st.layers:
-        for pr in PROJECTIONS:
-            q = st.q_local(layer, pr)
-            jobs.append((st.W[layer, pr], st.norms[layer, cfg.x_key(pr)], st.counts[q:q + 1], None))
-    if getattr(st, "ws_batch", None) is None:
+    if "count_views" not in st.batches or st.batches["count_views"][0] is not st.counts:
+        st.batches["count_views"] = (st.counts, [st.counts[q:q + 1] for q in range(st.counts.numel())])
+    views = st.batches["count_views"][1]
+    jobs = [(st.W[layer, pr], st.norms[layer, cfg.x_key(pr)], views[st.q_local(layer, pr)], None)
+            for layer in st.layers for pr in PROJECTIONS]
+    if st.ws_batch is None:
         st.ws_batch = api.Workspace(st.device)
-    api.mosaic_outlier_ratio_batch(jobs, a, st.ws_batch)
+    _cached_batch(st, "outlier", jobs, api.OutlierBatch).run(a, st.ws_batch)
     return len(jobs)
 
 
@@ -165,20 +177,18 @@ def prune_unstructured_layer(st: ModelState, layer: int, k_global: list[int], in
 
 def prune_unstructured_all(st: ModelState, k_global: list[int], in_place: bool = False) -> int:
     """Phase B for every owned projection through the batched call: one planning launch and one
-    pruning launch per distinct row length instead of one launch per projection.  Returns the
-    number of jobs."""
+    pruning launch per distinct row length instead of one launch per projection.  The job list is
+    marshalled once and reused, with the new prune counts, while the tensors of the ModelState stay
+    the same objects.  Returns the number of jobs."""
     cfg = st.cfg
     M = len(PROJECTIONS)
-    jobs = []
-    for layer in st.layers:
-        for m, pr in enumerate(PROJECTIONS):
-            W = st.W[layer, pr]
-            jobs.append((W, W if in_place else st.W_out[layer, pr], st.norms[layer, cfg.x_key(pr)],
-                         int(k_global[layer * M + m]), st.mask.get((layer, pr))))
-    if getattr(st, "ws_batch", None) is None:
+    jobs = [(st.W[layer, pr], st.W[layer, pr] if in_place else st.W_out[layer, pr], st.norms[layer, cfg.x_key(pr)], 0,
+             st.mask.get((layer, pr))) for layer in st.layers for pr in PROJECTIONS]
+    if st.ws_batch is None:
         st.ws_batch = api.Workspace(st.device)
-    api.mosaic_prune_unstructured_batch(jobs, st.ws_batch)
-    return len(jobs)
+    ks = [int(k_global[layer * M + m]) for layer in st.layers for m in range(M)]
+    _cached_batch(st, "prune_in_place" if in_place else "prune", jobs, api.PruneBatch).run(ks, st.ws_batch)
+    return len(ks)
 
 
 def _scores(W, norms, row_group, col_group, out, accumulate, ws):
