@@ -46,11 +46,8 @@
 #ifndef MOSAIC_MINB_SMALL
 #define MOSAIC_MINB_SMALL 4
 #endif
-#ifndef MOSAIC_ROUND_UNROLL
-#define MOSAIC_ROUND_UNROLL 1
-#endif
-#ifndef MOSAIC_NORM_EVICT_LAST
-#define MOSAIC_NORM_EVICT_LAST 1
+#ifndef MOSAIC_ROUND_GROUP
+#define MOSAIC_ROUND_GROUP 4
 #endif
 #ifndef MOSAIC_FAST_MAX_CTAS
 #define MOSAIC_FAST_MAX_CTAS 8
@@ -300,7 +297,7 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
 // ---------------------------------------------------------------------------------------------
 constexpr int kFastV = 4;          // vectors (of 8 columns) per thread
 constexpr int kWinBins = 1024;     // histogram over the top 10 bits of a window
-constexpr int kRoundUnroll = MOSAIC_ROUND_UNROLL;
+constexpr int kRoundGroup = MOSAIC_ROUND_GROUP;   // candidate rounds of a warp whose loads are issued together
 constexpr int kQueueCap = 448;     // candidates a warp can queue (of its 1024 weights)
 constexpr int kBinListCap = 512;   // keys of one histogram bin that warp 0 will rank; also the sample size limit
 
@@ -316,15 +313,14 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait_all_but() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-// A norm, kept in L1 with priority: the row data streams past it.
+// A norm of a candidate's column, read from L2 past L1.  The candidates of a row hit columns at
+// random, so almost every 32-lane request has a lane that misses L1 whatever it holds, and a miss
+// there costs more than the L2 access it leads to; with several norm vectors in turn (a batch)
+// the L1 path was 15 % slower end to end.
 __device__ __forceinline__ float ld_norm(const float* p) {
-#if MOSAIC_NORM_EVICT_LAST
     float v;
-    asm volatile("ld.global.nc.L1::evict_last.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    asm("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
     return v;
-#else
-    return __ldg(p);
-#endif
 }
 __device__ __forceinline__ void sts_u16_zero(void* smem) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "h"((unsigned short)0) : "memory");
@@ -585,6 +581,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
 
     // Key of the matching quantile of one key per thread (element 0 of vector 0), or 0.
     auto sample_center = [&](int cur) -> uint32_t {
+        __syncthreads();   // a slower warp may still be ranking the previous row's bin out of `list`
         list[tid] = cand_key(cur, 0, 0);
         __syncthreads();
         flush_mask();
@@ -642,21 +639,39 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         // exact scores of the candidates, 32 at a time: below lo, or into the window histogram
         const uint16_t* row_elems = reinterpret_cast<const uint16_t*>(rowbuf + cur * V * nt);   // column c of the row is element c
         const int warp_col0 = (wid << 5) * kVec;
-#pragma unroll kRoundUnroll
-        for (uint32_t i = lane; i < q_n; i += 32) {
-            const uint32_t id = qid[i];
-            const int col = warp_col0 + (int)(id >> 5) * kVec + col_of_flag[id & 31];
-            const uint32_t a = ((uint32_t)row_elems[col] & 0x7FFFu) << 16;
-            const uint32_t key = __float_as_uint(__fmul_rn(ld_norm(norms + col), __uint_as_float(a)));
-            qkey[i] = key;
-            const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
-            if (d < width) {
-                const uint32_t bin = d >> shift;
-                atomicAdd(&hist[bin], 1u);
-                atomicAdd(&coarse[bin >> 5], 1u);
-                slot[bin] = key;
-            } else {
-                below += d >> 31;
+        // kRoundGroup rounds at a time, their dependent loads (entry, column, weight, norm) issued side by side
+        for (uint32_t base = lane; base < q_n; base += 32u * kRoundGroup) {
+            uint32_t id[kRoundGroup], a[kRoundGroup];
+            int col[kRoundGroup];
+            float nm[kRoundGroup];
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g) {
+                const uint32_t i = base + 32u * g;
+                id[g] = i < q_n ? (uint32_t)qid[i] : 0u;   // entry 0 of a spare slot: an in-range column, result unused
+            }
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g) col[g] = warp_col0 + (int)(id[g] >> 5) * kVec + col_of_flag[id[g] & 31];
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g) {
+                a[g] = ((uint32_t)row_elems[col[g]] & 0x7FFFu) << 16;
+                nm[g] = ld_norm(norms + col[g]);
+            }
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g) {
+                const uint32_t i = base + 32u * g;
+                if (i < q_n) {
+                    const uint32_t key = __float_as_uint(__fmul_rn(nm[g], __uint_as_float(a[g])));
+                    qkey[i] = key;
+                    const uint32_t d = key - lo;   // key < lo wraps to >= 2^31
+                    if (d < width) {
+                        const uint32_t bin = d >> shift;
+                        atomicAdd(&hist[bin], 1u);
+                        atomicAdd(&coarse[bin >> 5], 1u);
+                        slot[bin] = key;
+                    } else {
+                        below += d >> 31;
+                    }
+                }
             }
         }
         below = __reduce_add_sync(0xFFFFFFFFu, below);
@@ -729,17 +744,34 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 }
             }
             __syncthreads();
-            if (wid == 0) {
-                uint32_t t = 0u, qq = 0u, ne = 0u;
-                const bool ok = warp_select(list, n_bin, lo + (bin << shift), shift, r_bin, whist, &t, &qq, &ne);
-                if (lane == 0) {
-                    sel.ok = (ok && qq == ne) ? 1u : 0u;   // a tie group that is only partly pruned goes the slow way
-                    sel.T = t;
+            if (n_bin <= 32u) {
+                // a handful of keys: every warp ranks them for itself (same list, same answer), which
+                // spares the hand-over through warp 0 and its barrier
+                const uint32_t mine = lane < (int)n_bin ? list[lane] : 0xFFFFFFFFu;
+                uint32_t less = 0u, eq = 0u;
+                for (uint32_t j = 0; j < n_bin; ++j) {
+                    const uint32_t o = __shfl_sync(0xFFFFFFFFu, mine, (int)j);
+                    less += (o < mine) ? 1u : 0u;
+                    eq += (o == mine) ? 1u : 0u;
                 }
+                const unsigned hit = __ballot_sync(0xFFFFFFFFu, lane < (int)n_bin && less < r_bin && r_bin <= less + eq);
+                const int src = __ffs(hit) - 1;   // some key holds rank r_bin (1 <= r_bin <= n_bin)
+                T = __shfl_sync(0xFFFFFFFFu, mine, src);
+                // a tie group that is only partly pruned goes the slow way
+                if (hit == 0u || r_bin - __shfl_sync(0xFFFFFFFFu, less, src) != __shfl_sync(0xFFFFFFFFu, eq, src)) return 2;
+            } else {
+                if (wid == 0) {
+                    uint32_t t = 0u, qq = 0u, ne = 0u;
+                    const bool ok = warp_select(list, n_bin, lo + (bin << shift), shift, r_bin, whist, &t, &qq, &ne);
+                    if (lane == 0) {
+                        sel.ok = (ok && qq == ne) ? 1u : 0u;   // a tie group that is only partly pruned goes the slow way
+                        sel.T = t;
+                    }
+                }
+                __syncthreads();
+                if (sel.ok == 0u) return 2;
+                T = sel.T;
             }
-            __syncthreads();
-            if (sel.ok == 0u) return 2;
-            T = sel.T;
         } else {
             MOSAIC_STAT(6);
         }
