@@ -736,12 +736,19 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         if (n_bin > 1u) {
             if (n_bin > (uint32_t)kBinListCap) return 2;
             // collect the keys of that bin; warp 0 ranks them
-            for (uint32_t i = lane; i < q_n; i += 32) {
-                const uint32_t key = qkey[i];
-                if (((key - lo) >> shift) == bin) {
-                    const uint32_t pos = atomicAdd(&n_list, 1u);
-                    if (pos < (uint32_t)kBinListCap) list[pos] = key;
+            for (uint32_t base = lane; base < q_n; base += 32u * kRoundGroup) {
+                uint32_t key[kRoundGroup];
+#pragma unroll
+                for (int g = 0; g < kRoundGroup; ++g) {
+                    const uint32_t i = base + 32u * g;
+                    key[g] = i < q_n ? qkey[i] : lo - 1u;   // a key below the window is in no bin
                 }
+#pragma unroll
+                for (int g = 0; g < kRoundGroup; ++g)
+                    if (((key[g] - lo) >> shift) == bin) {
+                        const uint32_t pos = atomicAdd(&n_list, 1u);
+                        if (pos < (uint32_t)kBinListCap) list[pos] = key[g];
+                    }
             }
             __syncthreads();
             if (n_bin <= 32u) {
@@ -779,13 +786,21 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         // prune: surely below lo, or a candidate whose exact key is <= T
         const uint32_t thr = T + 1u;
         uint16_t* out_row = W_out + row * ldw;
-        for (uint32_t i = lane; i < q_n; i += 32) {
-            if (qkey[i] < thr) {
-                const uint32_t id = qid[i];
-                const int col = warp_col0 + (int)(id >> 5) * kVec + col_of_flag[id & 31];
-                sts_u16_zero(reinterpret_cast<uint16_t*>(rowbuf + cur * V * nt) + col);
-                atomicOr(&gone_w[(wid << 5) | (int)(id >> 5)], 1u << (id & 31));
+        for (uint32_t base = lane; base < q_n; base += 32u * kRoundGroup) {
+            uint32_t key[kRoundGroup], id[kRoundGroup];
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g) {
+                const uint32_t i = base + 32u * g;
+                key[g] = i < q_n ? qkey[i] : 0xFFFFFFFFu;   // never below thr <= 2^31
+                id[g] = i < q_n ? (uint32_t)qid[i] : 0u;
             }
+#pragma unroll
+            for (int g = 0; g < kRoundGroup; ++g)
+                if (key[g] < thr) {
+                    const int col = warp_col0 + (int)(id[g] >> 5) * kVec + col_of_flag[id[g] & 31];
+                    sts_u16_zero(reinterpret_cast<uint16_t*>(rowbuf + cur * V * nt) + col);
+                    atomicOr(&gone_w[(wid << 5) | (int)(id[g] >> 5)], 1u << (id[g] & 31));
+                }
         }
         __syncwarp();
         const uint32_t gone_all = gone_w[tid];
