@@ -69,6 +69,9 @@ constexpr int kListCap = kBins1;  // candidate list shares the histogram's stora
 #define MOSAIC_TRACK_BITS 21
 #endif
 constexpr int kTrackBits = MOSAIC_TRACK_BITS;    // width (log2, in key units) of a window carried from row to row
+// The k-th score of a row scatters from row to row like 1/sqrt(cols): long rows get by with half the window
+// (half the candidates).
+__host__ __device__ constexpr int track_bits_for(int cols) { return cols >= 8192 ? kTrackBits - 1 : kTrackBits; }
 constexpr int kSampleBits = 23;   // width of the window around a sampled quantile
 
 struct RowSelect {   // hand-over between warp 0 and the CTA during a window attempt
@@ -505,6 +508,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
 
     const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = nt >> 5;
     const int nvec = cols >> 3;
+    const int track_bits = track_bits_for(cols);
     uint32_t* hist = buf;
     uint32_t* slot = buf + kWinBins;
     // Per warp: a queue of its candidates (who holds the weight, and its exact key), so that the
@@ -892,7 +896,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 }
                 if (!win_valid) break;
                 status = fast_attempt(cur, row, T_row);
-                if (status == 0) MOSAIC_STAT(win_w == kTrackBits ? 2 : 4);
+                if (status == 0) MOSAIC_STAT(win_w == track_bits ? 2 : 4);
             }
         }
         if (status != 0) {
@@ -903,14 +907,14 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
             T_row = generic_row_bf16<V>(&rowbuf[(cur * V) * nt + tid], nt, norms, cols, nvec, uk, buf, warp_tot, &sel3, W_out,
                                         row * ldw, mask_bytes, row * mask_row_bytes, mask_row_bytes);
         }
-        if (all_finite && (status != 0 || win_w != kTrackBits)) set_window(T_row, kTrackBits);
+        if (all_finite && (status != 0 || win_w != track_bits)) set_window(T_row, track_bits);
     }
     __syncthreads();
     flush_mask();
 }
 
 // One CTA per job: the exact thresholds of three rows (first, middle, last) by the full radix
-// select, a window of width 2^kTrackBits centred on their median, and the per-column thresholds
+// select, a window of width 2^track_bits_for(cols) centred on their median, and the per-column thresholds
 // of that window in the layout the pruning kernel loads (same nt).
 template <int MAXNT, int NJ>
 __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_constant__ PruneJobList<NJ> jobs, int cols) {
@@ -953,7 +957,7 @@ __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_const
         }
         const uint32_t mx = max(max(Ts[0], Ts[1]), Ts[2]), mn = min(min(Ts[0], Ts[1]), Ts[2]);
         const uint32_t median = (uint32_t)((uint64_t)Ts[0] + Ts[1] + Ts[2] - mx - mn);
-        valid = window_thresholds<V>(median, kTrackBits, J.norms, cols, nt, Alo, Ahi, &lo);
+        valid = window_thresholds<V>(median, track_bits_for(cols), J.norms, cols, nt, Alo, Ahi, &lo);
     }
     if (valid) {
 #pragma unroll
@@ -966,7 +970,7 @@ __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_const
     if (tid == 0) {
         plan[0] = valid ? 1u : 0u;
         plan[1] = lo;
-        plan[2] = (uint32_t)kTrackBits;
+        plan[2] = (uint32_t)track_bits_for(cols);
         plan[3] = 0u;
     }
 }
