@@ -5,17 +5,32 @@
 
 namespace mosaic {
 
-// Stage 2: add the split partials of each column in split order to the caller's
-// accumulator, and optionally finalise norm = (float) sqrt(sumsq).
-__global__ void act_finish_kernel(const double* __restrict__ partial, int splits, int64_t cols,
-                                  double* __restrict__ sumsq, float* __restrict__ norms_out, int reset) {
-    const int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= cols) return;
-    double s = reset ? 0.0 : sumsq[c];
-#pragma unroll 16
-    for (int p = 0; p < splits; ++p) s += partial[(int64_t)p * cols + c];   // loads batched, adds in split order
-    sumsq[c] = s;
-    if (norms_out) norms_out[c] = (float)sqrt(s);
+// Stage 2: add the split partials of each column to the caller's accumulator, and optionally
+// finalise norm = (float) sqrt(sumsq).  A CTA covers 32 columns with 8 lanes of threads per
+// column: lane g adds the partials g, g+8, ... in that order (all its loads in flight at once),
+// then the 8 lane sums are added in lane order.  The order is fixed, so the result does not
+// depend on the launch.
+constexpr int kFinCols = 32, kFinLanes = 8;
+__global__ void __launch_bounds__(kFinCols * kFinLanes) act_finish_kernel(const double* __restrict__ partial, int splits,
+                                                                            int64_t cols, double* __restrict__ sumsq,
+                                                                            float* __restrict__ norms_out, int reset) {
+    __shared__ double sm[kFinLanes][kFinCols + 1];
+    const int cl = threadIdx.x % kFinCols, g = threadIdx.x / kFinCols;
+    const int64_t c = (int64_t)blockIdx.x * kFinCols + cl;
+    double s = 0.0;
+    if (c < cols) {
+#pragma unroll 8
+        for (int p = g; p < splits; p += kFinLanes) s += partial[(int64_t)p * cols + c];
+    }
+    sm[g][cl] = s;
+    __syncthreads();
+    if (g == 0 && c < cols) {
+        double t = reset ? 0.0 : sumsq[c];
+#pragma unroll
+        for (int r = 0; r < kFinLanes; ++r) t += sm[r][cl];
+        sumsq[c] = t;
+        if (norms_out) norms_out[c] = (float)sqrt(t);
+    }
 }
 
 }  // namespace mosaic
@@ -55,8 +70,7 @@ extern "C" int mosaic_act_norms(const void* X, int64_t tokens, int64_t cols, int
                 X, tokens, cols, ldx, nullptr, p.rows_per_split, static_cast<double*>(ws));
         MOSAIC_LAUNCH_CHECK();
     }
-    const int threads = 128;
-    act_finish_kernel<<<(unsigned)((cols + threads - 1) / threads), threads, 0, st>>>(
+    act_finish_kernel<<<(unsigned)((cols + kFinCols - 1) / kFinCols), kFinCols * kFinLanes, 0, st>>>(
         static_cast<const double*>(ws), splits, cols, sumsq_accum, norms_out, (flags & MOSAIC_RESET_ACCUM) ? 1 : 0);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
