@@ -40,8 +40,10 @@
 #ifndef MOSAIC_PRUNE_MINB_2X256
 #define MOSAIC_PRUNE_MINB_2X256 3
 #endif
-#ifndef MOSAIC_RING_SMALL
-#define MOSAIC_RING_SMALL 3
+// Rows of a CTA resident in shared memory: the one being selected and the next one on its way from HBM.
+// A third (two in flight) was 2-4 % slower on every row length once the selection itself got faster.
+#ifndef MOSAIC_RING
+#define MOSAIC_RING 2
 #endif
 #ifndef MOSAIC_MINB_SMALL
 #define MOSAIC_MINB_SMALL 4
@@ -1017,12 +1019,12 @@ static int dispatch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows,
                                cudaStream_t st) {
     // CTAs per SM are chosen so that a thread keeps about 128 registers where shared memory allows it: with the
     // thresholds in registers, a smaller budget spills them (rows of 5120 / 8192 columns ran 25 % slower at 80).
-    if (nt <= 128) return launch_prune_bf16<128, MOSAIC_MINB_SMALL, NJ, MOSAIC_RING_SMALL>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 160) return launch_prune_bf16<160, 3, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 256) return launch_prune_bf16<256, 2, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 352) return launch_prune_bf16<352, 2, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 384) return launch_prune_bf16<384, 2, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
-    return launch_prune_bf16<512, 1, NJ, 3>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 128) return launch_prune_bf16<128, MOSAIC_MINB_SMALL, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 160) return launch_prune_bf16<160, 3, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 256) return launch_prune_bf16<256, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 352) return launch_prune_bf16<352, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 384) return launch_prune_bf16<384, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    return launch_prune_bf16<512, 1, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
 }
 
 // Threads per CTA of the bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
