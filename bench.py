@@ -201,7 +201,7 @@ def run_native(args, cfg):
         launches = 0
         if ev: ev[0].record()
         for layer in mine:
-            launches += 2 * driver.accumulate_norms(st, layer, X)
+            launches += 2 * driver.accumulate_norms(st, layer, X, join=(layer == mine[-1]))
         if ev: ev[1].record()
         driver.count_outliers_all(st)
         launches += 2                                                   # the two sweeps, each over every projection

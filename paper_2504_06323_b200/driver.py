@@ -83,6 +83,7 @@ class ModelState:
     ws: api.Workspace | None = None
     ws_batch: api.Workspace | None = None             # holds the plans of the batched pruning call
     batches: dict = field(default_factory=dict)        # name -> (identity of the tensors, marshalled batch)
+    side: list | None = None                           # two (stream, workspace) pairs for independent calls
 
     def q_local(self, layer: int, proj: str) -> int:
         return self.layers.index(layer) * len(PROJECTIONS) + PROJECTIONS.index(proj)
@@ -117,15 +118,50 @@ def make_activations(cfg: ModelConfig, layer: int, device="cuda", tokens: int | 
 
 
 # ------------------------------------------------------------------ phase A
-def accumulate_norms(st: ModelState, layer: int, X: dict, first: bool = True, last: bool = True) -> int:
+def accumulate_norms(st: ModelState, layer: int, X: dict, first: bool = True, last: bool = True,
+                     overlap: bool = True, join: bool = True) -> int:
     """Add one chunk of calibration tokens per input; `last` also finalises the fp32 norms.
-    Returns the number of library calls made."""
-    n = 0
-    for xk, x in X.items():
+    Returns the number of library calls made.
+
+    The inputs of a layer are independent, so with `overlap` their calls alternate between two side
+    streams (each with a workspace of its own): the start-up and the finishing kernel of one input
+    then run under the streaming of the next.  With `join` the current stream waits for both before
+    returning; a caller that runs several layers in a row joins on the last one only (join_side())
+    so that the layers overlap as well."""
+    if not overlap or st.device.type != "cuda" or len(X) < 2:
+        for xk, x in X.items():
+            api.mosaic_act_norms(x, st.sumsq[layer, xk], st.norms[layer, xk] if last else None,
+                                 api.RESET_ACCUM if first else 0, st.ws)
+        return len(X)
+    if st.side is None:
+        st.side = [(torch.cuda.Stream(st.device), api.Workspace(st.device)) for _ in range(2)]
+    need = max(api.lib().mosaic_act_norms_workspace_bytes(x.shape[0], x.shape[1]) for x in X.values())
+    cur = torch.cuda.current_stream(st.device)
+    fork = torch.cuda.Event()
+    fork.record(cur)
+    for s, ws in st.side:
+        if ws.buf is None or ws.buf.numel() < need:   # grown before anything is in flight on the side stream
+            s.synchronize()
+            ws.get(need)
+        s.wait_event(fork)
+    for i, (xk, x) in enumerate(X.items()):
+        s, ws = st.side[i % 2]
         api.mosaic_act_norms(x, st.sumsq[layer, xk], st.norms[layer, xk] if last else None,
-                             api.RESET_ACCUM if first else 0, st.ws)
-        n += 1
-    return n
+                             api.RESET_ACCUM if first else 0, ws, stream=s)
+    if join:
+        join_side(st)
+    return len(X)
+
+
+def join_side(st: ModelState) -> None:
+    """Make the current stream wait for everything issued on the side streams so far."""
+    if st.side is None:
+        return
+    cur = torch.cuda.current_stream(st.device)
+    for s, _ in st.side:
+        done = torch.cuda.Event()
+        done.record(s)
+        cur.wait_event(done)
 
 
 def count_outliers(st: ModelState, layer: int, alpha: float | None = None) -> int:
