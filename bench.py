@@ -278,6 +278,9 @@ def run_native(args, cfg):
                         "partial-sum writes do not)",
         "algorithmic_bytes_per_launch": act_bytes / n_act_launch, "launches_per_step": n_act_launch,
         "avg_launch_ms": phase_ms[0] / n_act_launch,
+        "note": "duration = the phase's CUDA-event time / launches (a layer's launches alternate between two streams, so "
+                "the finishing kernel of one runs under the next); the peak is a copy (read + write): a read-only "
+                "stream like this one can exceed it by a few per cent",
     }
     outl_gbs = w_bytes / (phase_ms[1] * 1e-3) / 1e9
     prune_gbs = w_bytes * 4.125 / 2 / (phase_ms[3] * 1e-3) / 1e9
