@@ -180,3 +180,26 @@ def test_full_size_batched_model_pass_sampled_against_oracle():
             assert bits_equal(st.mask[layer, pr][sample].cpu().numpy().view(np.uint32), ref_mask), (layer, pr)
             kept = st.mask[layer, pr].cpu().numpy().view(np.uint8)
             assert (np.unpackbits(kept, axis=1).sum(1) == cols - kk).all(), (layer, pr)
+
+
+def test_norm_calls_on_side_streams_match_the_serial_order():
+    # the same layers three ways: one stream, two side streams joined after every layer, joined once at the end
+    cfg = small("llama7b", n_layers=3, tokens=2500)
+    X = {layer: driver.make_activations(cfg, layer, DEV) for layer in range(cfg.n_layers)}
+    results = []
+    for mode in ("serial", "join_each", "join_last"):
+        st = driver.alloc_model(cfg, DEV, outputs=False, masks=False)
+        for n in st.norms.values():
+            n.fill_(-1.0)
+        for layer in st.layers:
+            if mode == "serial":
+                driver.accumulate_norms(st, layer, X[layer], overlap=False)
+            else:
+                driver.accumulate_norms(st, layer, X[layer], join=(mode == "join_each"))
+        if mode == "join_last":
+            driver.join_side(st)
+        torch.cuda.current_stream().synchronize()      # the current stream alone: it must already cover the side streams
+        results.append({k: v.cpu().numpy() for k, v in st.norms.items()})
+    for key, ref in results[0].items():
+        assert (ref > 0).all()
+        assert bits_equal(results[1][key], ref) and bits_equal(results[2][key], ref), key

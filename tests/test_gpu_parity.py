@@ -345,6 +345,42 @@ def test_prune_batch_matches_oracle_job_by_job(dtype):
             assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
 
 
+def test_prune_batch_reused_with_new_counts():
+    # one marshalled job list run three times with different per-row prune counts (k = 0 <-> k > 0 changes
+    # which kernel a job takes and how much workspace the call needs)
+    shapes = [(300, 4096), (120, 11008), (64, 688), (200, 8192)]
+    Ws = [make(r, c, "bf16", seed=900 + i, heavy=(i == 1)) for i, (r, c) in enumerate(shapes)]
+    norms = [norms_for(c, 70 + i) for i, (r, c) in enumerate(shapes)]
+    outs = [torch.empty_like(W) for W in Ws]
+    masks = [torch.empty(r, (c + 31) // 32, dtype=torch.int32, device=DEV) for r, c in shapes]
+    batch = api.PruneBatch([(W, o, n, 0, m) for W, o, n, m in zip(Ws, outs, norms, masks)])
+    ws = api.Workspace(DEV)
+    for ks in ([0, 0, 0, 0], [2048, 5504, 300, 4096], [1000, 0, 688, 8191], [2048, 5504, 300, 4096]):
+        for o, m in zip(outs, masks):
+            o.fill_(7.0)
+            m.fill_(-1)
+        batch.run(ks, ws)
+        for W, o, n, m, k in zip(Ws, outs, norms, masks, ks):
+            ref_W, ref_mask = oracle.prune_unstructured(host(W), n.cpu().numpy(), k, "bf16")
+            assert_bits_equal(host(o), ref_W)
+            assert_bits_equal(m.cpu().numpy().view(np.uint32), ref_mask)
+
+
+def test_outlier_batch_reused():
+    shapes = [(300, 4096), (64, 688), (130, 11008)]
+    Ws = [make(r, c, "bf16", seed=950 + i, heavy=True) for i, (r, c) in enumerate(shapes)]
+    norms = [norms_for(c, 80 + i) for i, (r, c) in enumerate(shapes)]
+    counts = torch.full((len(shapes),), -5, dtype=torch.int64, device=DEV)
+    batch = api.OutlierBatch([(W, n, counts[i:i + 1], None) for i, (W, n) in enumerate(zip(Ws, norms))])
+    ws = api.Workspace(DEV)
+    for alpha in (5.0, 2.0, 5.0):
+        batch.run(alpha, ws)
+        got = counts.cpu().tolist()
+        for i, (W, n) in enumerate(zip(Ws, norms)):
+            ref = oracle.outlier_ratio(host(W), n.cpu().numpy(), alpha, "bf16")
+            assert ref["certified"] and got[i] == ref["count"], (alpha, i)
+
+
 # ------------------------------------------------------------------ structured
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("rows,cols,rg,cg,fr,fc", [(256, 688, 1, 1, 0.3, 0.3), (512, 1024, 64, 1, 0.25, 0.5),
