@@ -133,13 +133,12 @@ def accumulate_norms(st: ModelState, layer: int, X: dict, first: bool = True, la
             api.mosaic_act_norms(x, st.sumsq[layer, xk], st.norms[layer, xk] if last else None,
                                  api.RESET_ACCUM if first else 0, st.ws)
         return len(X)
-    if st.side is None:
-        st.side = [(torch.cuda.Stream(st.device), api.Workspace(st.device)) for _ in range(2)]
+    _side_streams(st, 2)
     need = max(api.lib().mosaic_act_norms_workspace_bytes(x.shape[0], x.shape[1]) for x in X.values())
     cur = torch.cuda.current_stream(st.device)
     fork = torch.cuda.Event()
     fork.record(cur)
-    for s, ws in st.side:
+    for s, ws in st.side[:2]:
         if ws.buf is None or ws.buf.numel() < need:   # grown before anything is in flight on the side stream
             s.synchronize()
             ws.get(need)
@@ -151,6 +150,15 @@ def accumulate_norms(st: ModelState, layer: int, X: dict, first: bool = True, la
     if join:
         join_side(st)
     return len(X)
+
+
+def _side_streams(st: ModelState, n: int) -> list:
+    """At least n (stream, workspace) pairs for calls that do not depend on one another."""
+    if st.side is None:
+        st.side = []
+    while len(st.side) < n:
+        st.side.append((torch.cuda.Stream(st.device), api.Workspace(st.device)))
+    return st.side[:n]
 
 
 def join_side(st: ModelState) -> None:
@@ -233,7 +241,7 @@ def _scores(W, norms, row_group, col_group, out, accumulate, ws):
 
 
 def prune_structured_coupled_layer(st: ModelState, layer: int, frac: float, source: dict | None = None,
-                                   use_norms: bool = True) -> dict:
+                                   use_norms: bool = True, ws: api.Workspace | None = None) -> dict:
     """Structured stage with the projections of a layer coupled the way the model's shapes require
     (Fig. "composite": nodes between projections are pruned as a group):
       * MLP channel c = row c of gate and up + column c of down, scored by the sum of the three;
@@ -243,7 +251,7 @@ def prune_structured_coupled_layer(st: ModelState, layer: int, frac: float, sour
     floor(frac * n_units) units are removed.  `source` gives the matrices to read (the masked
     weights in composite mode); returns {"W": {proj: compacted}, "mlp_keep", "attn_keep"}.
     """
-    cfg, dev, ws = st.cfg, st.device, st.ws
+    cfg, dev, ws = st.cfg, st.device, (st.ws if ws is None else ws)
     src = {pr: (source[pr] if source is not None else st.W[layer, pr]) for pr in PROJECTIONS}
     nrm = {pr: (st.norms[layer, cfg.x_key(pr)] if use_norms else None) for pr in PROJECTIONS}
     hd, n_kv = cfg.head_dim, cfg.n_kv_heads
@@ -299,7 +307,8 @@ def prune_structured_coupled_layer(st: ModelState, layer: int, frac: float, sour
     return out
 
 
-def prune_structured_independent(st: ModelState, layer: int, proj: str, frac: float, use_norms: bool = True):
+def prune_structured_independent(st: ModelState, layer: int, proj: str, frac: float, use_norms: bool = True,
+                                 ws: api.Workspace | None = None):
     """Every projection on its own: remove floor(frac*rows) rows and floor(frac*cols) columns
     (group 1) and write the dense compacted matrix.  Returns (W_compact, row_keep, col_keep)."""
     cfg, dev = st.cfg, st.device
@@ -310,5 +319,43 @@ def prune_structured_independent(st: ModelState, layer: int, proj: str, frac: fl
     ck = torch.empty(kc, dtype=torch.int32, device=dev)
     out = torch.empty(kr, kc, dtype=cfg.torch_dtype, device=dev)
     api.mosaic_prune_structured_compact(W, st.norms[layer, cfg.x_key(proj)] if use_norms else None, 1, 1, kr, kc, rk,
-                                        ck, 0, out, None, st.ws)
+                                        ck, 0, out, None, st.ws if ws is None else ws)
     return out, rk, ck
+
+
+def prune_structured_model(st: ModelState, frac: float, coupled: bool = True, sources: dict | None = None,
+                           use_norms: bool = True, n_streams: int = 4) -> dict:
+    """The structured stage over every owned layer.  Layers (coupled) or projections (independent)
+    do not depend on one another, so they go round-robin to `n_streams` side streams, each with its
+    own workspace: the ranking kernels - one or two CTAs each - then run beside the score and
+    compaction kernels of other matrices instead of holding the GPU alone.  `sources[layer]`, if
+    given, holds the matrices to read (the masked weights in composite mode).  Returns
+    {layer: result of prune_structured_coupled_layer} or {(layer, proj): (W_compact, row_keep,
+    col_keep)}; the current stream has waited for all of it."""
+    side = _side_streams(st, n_streams)
+    cur = torch.cuda.current_stream(st.device)
+    fork = torch.cuda.Event()
+    fork.record(cur)
+    for s, _ in side:
+        s.wait_event(fork)
+    out: dict = {}
+    i = 0
+    for layer in st.layers:
+        if coupled:
+            s, ws = side[i % n_streams]
+            i += 1
+            with torch.cuda.stream(s):      # buffers made here belong to s: freed ones are reused in s's order
+                out[layer] = prune_structured_coupled_layer(st, layer, frac, None if sources is None else sources[layer],
+                                                            use_norms, ws)
+        else:
+            for pr in PROJECTIONS:
+                s, ws = side[i % n_streams]
+                i += 1
+                with torch.cuda.stream(s):
+                    out[layer, pr] = prune_structured_independent(st, layer, pr, frac, use_norms, ws)
+    join_side(st)
+    for res in out.values():               # the results are used on the current stream from here on
+        tensors = list(res["W"].values()) + [res["mlp_keep"], res["attn_keep"]] if coupled else list(res)
+        for t in tensors:
+            t.record_stream(cur)
+    return out

@@ -203,3 +203,26 @@ def test_norm_calls_on_side_streams_match_the_serial_order():
     for key, ref in results[0].items():
         assert (ref > 0).all()
         assert bits_equal(results[1][key], ref) and bits_equal(results[2][key], ref), key
+
+
+def test_structured_model_over_side_streams_matches_layer_by_layer():
+    cfg = small("llama3_8b", hidden=640, n_heads=10, n_kv_heads=5, head_dim=64, intermediate=1728, n_layers=5, tokens=1500)
+    st = driver.alloc_model(cfg, DEV, outputs=False, masks=False)
+    for layer in st.layers:
+        driver.accumulate_norms(st, layer, driver.make_activations(cfg, layer, DEV))
+    for rep in range(2):   # the second pass reuses streams, workspaces and freed buffers
+        got = driver.prune_structured_model(st, 0.2, coupled=True)
+        torch.cuda.current_stream().synchronize()
+        for layer in st.layers:
+            ref = driver.prune_structured_coupled_layer(st, layer, 0.2)
+            assert torch.equal(got[layer]["mlp_keep"], ref["mlp_keep"]) and torch.equal(got[layer]["attn_keep"], ref["attn_keep"])
+            for pr in PROJECTIONS:
+                assert bits_equal(wl.to_numpy(got[layer]["W"][pr]), wl.to_numpy(ref["W"][pr])), (rep, layer, pr)
+        got = driver.prune_structured_model(st, 0.3, coupled=False)
+        torch.cuda.current_stream().synchronize()
+        for layer in st.layers:
+            for pr in PROJECTIONS:
+                out, rk, ck = driver.prune_structured_independent(st, layer, pr, 0.3)
+                g = got[layer, pr]
+                assert torch.equal(g[1], rk) and torch.equal(g[2], ck)
+                assert bits_equal(wl.to_numpy(g[0]), wl.to_numpy(out)), (rep, layer, pr)
