@@ -292,6 +292,25 @@ def test_prune_many_rows_per_cta(dtype, rows, cols):
         _check_prune(W, norms, k, dtype)
 
 
+@pytest.mark.parametrize("cols", [2048, 2056, 4104, 5128, 6152, 8200, 10248, 11264, 11272, 12296, 16384, 16392])
+def test_prune_bf16_every_cta_shape_with_a_ragged_last_vector_slot(cols):
+    # one row length per instantiation of the bf16 kernel (128 ... 512 threads) and just past each limit, so that
+    # some threads own vector slots beyond the end of the row; 16392 columns is beyond the kernel and takes the
+    # general one.  Batched (planned windows) and single (sampled windows) calls.
+    rows = 700
+    W = make(rows, cols, "bf16", seed=cols, heavy=(cols % 16 == 0))
+    norms = norms_for(cols, cols % 97)
+    for k in (cols // 2, 1, cols - 1):
+        _check_prune(W, norms, k, "bf16")
+    k = (3 * cols) // 10
+    out = torch.full_like(W, 3.0)
+    mask = torch.full((rows, (cols + 31) // 32), -1, dtype=torch.int32, device=DEV)
+    api.mosaic_prune_unstructured_batch([(W, out, norms, k, mask)])
+    ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, "bf16")
+    assert_bits_equal(host(out), ref_W)
+    assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_prune_rows_of_very_different_scale(dtype):
     # consecutive rows of a CTA differ by orders of magnitude, some are constant, some all zero,
