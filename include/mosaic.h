@@ -109,7 +109,7 @@ int mosaic_score(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dty
 
 /* ---------------------------------------------------------------------------
  * mosaic_outlier_ratio - Eq. 6 / the outlier-count step of Algorithm 1 for one projection:
- *     S = sum_ij (double) w_ij,  tau = (double)alpha * S / (rows*cols),
+ *     S = sum_ij (double) w_ij,  tau = (double)alpha * (S / (rows*cols)),   (fp64, in this order)
  *     O = #{ (i,j) : (double) w_ij > tau }                  (strict)
  *   outlier_count_out  device, 1 x int64
  *   score_sum_out      device, 1 x fp64, or NULL
@@ -165,7 +165,9 @@ int mosaic_outlier_ratio_batch(const mosaic_outlier_job *jobs, int64_t n_jobs, i
  *     regular call with your own buffer then.
  *   - The first call on each device looks up the array's device address (a
  *     host-side runtime query, with that device current).  Make that first
- *     call during start-up, outside any stream capture.
+ *     call during start-up, outside any stream capture.  The address belongs
+ *     to the device's context: after cudaDeviceReset() on a device this entry
+ *     point must not be used on it again in the same process.
  *   - All calls on one device share the one array.  Every call overwrites
  *     what it reads from it, so whatever an earlier call left there does no
  *     harm and back-to-back calls on one stream are fine; two calls that can overlap

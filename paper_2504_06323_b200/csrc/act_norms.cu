@@ -63,11 +63,11 @@ extern "C" int mosaic_act_norms(const void* X, int64_t tokens, int64_t cols, int
         splits = p.splits;
         dim3 grid((unsigned)((cols + kColTile - 1) / kColTile), (unsigned)p.splits);
         if (dtype == MOSAIC_BF16)
-            col_partial_kernel<MOSAIC_BF16, COL_SQUARE><<<grid, kColTile, 0, st>>>(
-                X, tokens, cols, ldx, nullptr, p.rows_per_split, static_cast<double*>(ws));
+            col_partial_kernel<MOSAIC_BF16><<<grid, kColTile, 0, st>>>(X, tokens, cols, ldx, p.rows_per_split,
+                                                                       static_cast<double*>(ws));
         else
-            col_partial_kernel<MOSAIC_F32, COL_SQUARE><<<grid, kColTile, 0, st>>>(
-                X, tokens, cols, ldx, nullptr, p.rows_per_split, static_cast<double*>(ws));
+            col_partial_kernel<MOSAIC_F32><<<grid, kColTile, 0, st>>>(X, tokens, cols, ldx, p.rows_per_split,
+                                                                      static_cast<double*>(ws));
         MOSAIC_LAUNCH_CHECK();
     }
     act_finish_kernel<<<(unsigned)((cols + kFinCols - 1) / kFinCols), kFinCols * kFinLanes, 0, st>>>(

@@ -5,22 +5,26 @@
 
 namespace mosaic {
 
-int sm_count() {
-    static int cached[64] = {0};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
         (void)cudaGetLastError();
-        return 148;
+        return -1;
     }
-    if (cached[dev] == 0) {
+    return dev;
+}
+
+int sm_count() {
+    static DeviceCache cached;
+    return cached.get([]() -> int {
         int n = 0;
-        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+        const int dev = current_device();
+        if (dev < 0 || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
             (void)cudaGetLastError();
             n = 148;
         }
-        cached[dev] = n;
-    }
-    return cached[dev];
+        return n;
+    });
 }
 
 int check_matrix(const void* p, int64_t rows, int64_t cols, int64_t ld, int dtype) {

@@ -6,8 +6,7 @@
 //            The 8 row lanes are combined in shared memory in lane order and
 //            one fp64 partial per (split, column) is written.
 //   stage 2: the caller adds the partials of a column in split order.
-// The value reduced is x^2 (activation norms, Eq. 5's ||A||_2 term); the COL_SCORE variant
-// (norm_j*|w_ij|) is kept for callers that want column sums of the weight metric alone.
+// The value reduced is x^2 (activation norms, Eq. 5's ||A||_2 term).
 #pragma once
 #include "common.cuh"
 
@@ -16,8 +15,6 @@ namespace mosaic {
 constexpr int kColTile = 256;   // columns per CTA
 constexpr int kRowLanes = 8;    // row lanes per CTA
 constexpr int kColUnroll = 4;   // rows in flight per thread
-
-enum ColOp { COL_SQUARE = 0, COL_SCORE = 1 };
 
 struct ColSplit {
     int splits;          // number of row splits (gridDim.y)
@@ -46,24 +43,19 @@ inline ColSplit col_split_plan(int64_t rows, int64_t cols) {
 
 #ifdef __CUDACC__
 
-template <int DT, int OP>
-__device__ __forceinline__ void col_accumulate(double (&acc)[kVec], const Raw8<DT>& r, const float (&nrm)[kVec]) {
+template <int DT>
+__device__ __forceinline__ void col_accumulate(double (&acc)[kVec], const Raw8<DT>& r) {
 #pragma unroll
     for (int e = 0; e < kVec; ++e) {
-        if (OP == COL_SQUARE) {
-            const double x = (double)r.f32(e);
-            acc[e] = fma(x, x, acc[e]);           // exact product, one rounding in the add
-        } else {
-            const float s = __fmul_rn(nrm[e], r.abs_f32(e));
-            acc[e] += (double)s;
-        }
+        const double x = (double)r.f32(e);
+        acc[e] = fma(x, x, acc[e]);           // exact product, one rounding in the add
     }
 }
 
-template <int DT, int OP>
+template <int DT>
 __global__ void __launch_bounds__(kColTile) col_partial_kernel(const void* __restrict__ M, int64_t rows, int64_t cols,
-                                                                int64_t ld, const float* __restrict__ norms,
-                                                                int rows_per_split, double* __restrict__ partial) {
+                                                                int64_t ld, int rows_per_split,
+                                                                double* __restrict__ partial) {
     __shared__ double sm[kRowLanes][kColTile + 2];
     const int cl = threadIdx.x & 31, rl = threadIdx.x >> 5;
     const int64_t c0 = (int64_t)blockIdx.x * kColTile + cl * kVec;
@@ -71,13 +63,8 @@ __global__ void __launch_bounds__(kColTile) col_partial_kernel(const void* __res
     const int64_t t1 = (t0 + rows_per_split < rows) ? t0 + rows_per_split : rows;
 
     double acc[kVec];
-    float nrm[kVec];
 #pragma unroll
-    for (int e = 0; e < kVec; ++e) {
-        acc[e] = 0.0;
-        nrm[e] = 1.0f;
-        if (OP == COL_SCORE && norms != nullptr && c0 + e < cols) nrm[e] = norms[c0 + e];
-    }
+    for (int e = 0; e < kVec; ++e) acc[e] = 0.0;
 
     if (c0 < cols) {
         int64_t t = t0 + rl;
@@ -86,12 +73,12 @@ __global__ void __launch_bounds__(kColTile) col_partial_kernel(const void* __res
 #pragma unroll
             for (int u = 0; u < kColUnroll; ++u) load_vec<DT, true>(r[u], M, (t + u * kRowLanes) * ld, c0, cols);
 #pragma unroll
-            for (int u = 0; u < kColUnroll; ++u) col_accumulate<DT, OP>(acc, r[u], nrm);
+            for (int u = 0; u < kColUnroll; ++u) col_accumulate<DT>(acc, r[u]);
         }
         for (; t < t1; t += kRowLanes) {
             Raw8<DT> r;
             load_vec<DT, true>(r, M, t * ld, c0, cols);
-            col_accumulate<DT, OP>(acc, r, nrm);
+            col_accumulate<DT>(acc, r);
         }
     }
 #pragma unroll

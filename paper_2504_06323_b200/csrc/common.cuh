@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/mosaic.h"
 
 namespace mosaic {
@@ -12,6 +14,29 @@ constexpr int kVec = 8;  // elements handled per thread per access: 16 B of bf16
 
 // ---------------------------------------------------------------- host side
 int sm_count();                        // SMs of the current device (148 if it cannot be queried)
+int current_device();                  // index of the current device, or -1 if it cannot be queried
+
+// One small non-zero integer remembered per device (occupancy of a kernel, "attribute set"):
+// function attributes and occupancy belong to one device's copy of a kernel, so a process that
+// drives several GPUs needs them once per device, not once per process.  get() runs `compute`
+// with the device current the first time that device asks; two host threads that race both
+// compute the same value.  A device index beyond the table is computed every time.
+constexpr int kMaxDevices = 64;
+class DeviceCache {
+    std::atomic<int> v_[kMaxDevices];   // static storage: starts at zero = "not computed yet"
+public:
+    template <class F>
+    int get(F compute) {
+        const int dev = current_device();
+        if (dev < 0 || dev >= kMaxDevices) return compute();
+        int x = v_[dev].load(std::memory_order_acquire);
+        if (x == 0) {
+            x = compute();
+            v_[dev].store(x, std::memory_order_release);
+        }
+        return x;
+    }
+};
 int check_matrix(const void* p, int64_t rows, int64_t cols, int64_t ld, int dtype);
 inline size_t elem_size(int dtype) { return dtype == MOSAIC_F32 ? 4 : 2; }
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

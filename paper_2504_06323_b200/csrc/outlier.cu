@@ -13,7 +13,9 @@
 //            and counts in fp32 against tau rounded toward -inf: for an fp32
 //            score s, (double)s > tau  <=>  s > fl32_down(tau).  It walks the
 //            tiles in reverse, starting on what sweep 1 touched last.
-#include <mutex>
+#include <atomic>
+#include <memory>
+#include <new>
 
 #include "common.cuh"
 
@@ -232,9 +234,8 @@ static int validate_outlier(const void* W, int64_t rows, int64_t cols, int64_t l
 
 template <int NJ>
 static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int dtype, cudaStream_t st) {
-    static int blocks_per_sm[2] = {0, 0};
-    int& bps = blocks_per_sm[dtype == MOSAIC_BF16 ? 1 : 0];
-    if (bps == 0) {
+    static DeviceCache blocks_per_sm[2];   // occupancy is a property of one device's copy of the kernels
+    const int bps = blocks_per_sm[dtype == MOSAIC_BF16 ? 1 : 0].get([&]() -> int {
         int n1 = 0, n2 = 0;
         cudaError_t e1, e2;
         if (dtype == MOSAIC_BF16) {
@@ -248,9 +249,9 @@ static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int d
             (void)cudaGetLastError();
             n1 = n2 = 4;
         }
-        bps = n1 < n2 ? n1 : n2;
-        if (bps < 1) bps = 1;
-    }
+        const int n = n1 < n2 ? n1 : n2;
+        return n < 1 ? 1 : n;
+    });
     int64_t grid = (int64_t)sm_count() * bps;
     if (grid > n_tiles) grid = n_tiles;
     if (dtype == MOSAIC_BF16) {
@@ -307,9 +308,10 @@ extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_
     if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
     if (ws_bytes < mosaic_outlier_ratio_batch_workspace_bytes(jobs, n_jobs)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    static OutlierJobList<kOutBatch> list;   // host staging of the kernel parameter (kept off the stack)
-    static std::mutex list_mutex;
-    std::lock_guard<std::mutex> lock(list_mutex);
+    // host staging of the kernel parameter (on the heap, one per call, so concurrent callers do not meet)
+    std::unique_ptr<OutlierJobList<kOutBatch>> list_mem(new (std::nothrow) OutlierJobList<kOutBatch>);
+    if (!list_mem) return MOSAIC_ERR_INVALID_ARG;
+    OutlierJobList<kOutBatch>& list = *list_mem;
     char* wsp = static_cast<char*>(ws);
     int64_t i = 0;
     while (i < n_jobs) {
@@ -349,19 +351,25 @@ static __device__ __align__(256) unsigned char g_outlier_scratch[kStaticScratchB
 // only a handle for the runtime, not something a kernel can dereference, so the address is asked
 // for once per device (with that device current) and remembered.
 static int static_scratch_address(void** out) {
-    static void* cached[64] = {nullptr};
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return MOSAIC_ERR_CUDA;
-    if (dev >= 0 && dev < 64 && cached[dev] != nullptr) {
-        *out = cached[dev];
-        return MOSAIC_OK;
+    // One slot per device.  Two host threads that race on a device's first call both look the
+    // address up and store the same value.  cudaDeviceReset() destroys the context the address
+    // belongs to: a process that resets a device must not call this entry point on it afterwards.
+    static std::atomic<void*> cached[kMaxDevices];
+    const int dev = current_device();
+    if (dev < 0) return MOSAIC_ERR_CUDA;
+    if (dev < kMaxDevices) {
+        void* hit = cached[dev].load(std::memory_order_acquire);
+        if (hit != nullptr) {
+            *out = hit;
+            return MOSAIC_OK;
+        }
     }
     void* p = nullptr;
     if (cudaGetSymbolAddress(&p, g_outlier_scratch) != cudaSuccess || p == nullptr) {
         (void)cudaGetLastError();
         return MOSAIC_ERR_CUDA;
     }
-    if (dev >= 0 && dev < 64) cached[dev] = p;
+    if (dev < kMaxDevices) cached[dev].store(p, std::memory_order_release);
     *out = p;
     return MOSAIC_OK;
 }
@@ -373,10 +381,9 @@ extern "C" size_t mosaic_outlier_ratio_static_max_workspace_bytes(void) { return
 extern "C" int mosaic_outlier_ratio_static(const void* W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
                                            const float* norms, float alpha, int64_t* outlier_count_out,
                                            double* score_sum_out, void* stream) {
-    // argument errors first, so that a bad call costs no CUDA work
-    int rc = check_matrix(W, rows, cols, ldw, dtype);
+    // every argument error first, so that a bad call costs no CUDA work at all
+    int rc = validate_outlier(W, rows, cols, ldw, dtype, norms, outlier_count_out, score_sum_out);
     if (rc != MOSAIC_OK) return rc;
-    if (rows == 0) return MOSAIC_ERR_INVALID_ARG;
     if (mosaic_outlier_ratio_workspace_bytes(rows, cols) > kStaticScratchBytes) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
     void* scratch = nullptr;
     rc = static_scratch_address(&scratch);

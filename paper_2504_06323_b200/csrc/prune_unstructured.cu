@@ -32,45 +32,21 @@
 //       between A_lo[j] and A_hi[j] - a few percent of the row - are the
 //       candidates, and only they get an exact fp32 score.
 //   prune_rows_kernel       any dtype, any shape; scores of all entries in fp32.
-#include <mutex>
+#include <memory>
+#include <new>
 #include <vector>
 
 #include "select.cuh"
 
-#ifndef MOSAIC_PRUNE_MINB_2X256
-#define MOSAIC_PRUNE_MINB_2X256 3
-#endif
-// Rows of a CTA resident in shared memory: the one being selected and the next one on its way from HBM.
-// A third (two in flight) was 2-4 % slower on every row length once the selection itself got faster.
-#ifndef MOSAIC_RING
-#define MOSAIC_RING 2
-#endif
-#ifndef MOSAIC_MINB_SMALL
-#define MOSAIC_MINB_SMALL 4
-#endif
-#ifndef MOSAIC_ROUND_GROUP
-#define MOSAIC_ROUND_GROUP 4
-#endif
-#ifndef MOSAIC_FAST_MAX_CTAS
-#define MOSAIC_FAST_MAX_CTAS 8
-#endif
-
 namespace mosaic {
 
-#ifdef MOSAIC_PRUNE_STATS   // development aid: how often each selection path ran
-__device__ unsigned long long g_prune_stats[8];
-#define MOSAIC_STAT(i) do { if (threadIdx.x == 0) atomicAdd(&g_prune_stats[i], 1ull); } while (0)
-#define MOSAIC_STAT_ADD(i, n) do { if (threadIdx.x == 0) atomicAdd(&g_prune_stats[i], (unsigned long long)(n)); } while (0)
-#else
-#define MOSAIC_STAT(i) do { } while (0)
-#define MOSAIC_STAT_ADD(i, n) do { } while (0)
-#endif
+// Rows of a CTA resident in shared memory: the one being selected and the next one on its way from HBM.
+// A third (two in flight) was 2-4 % slower on every row length once the selection itself got faster.
+constexpr int kRing = 2;
+constexpr int kFastMaxCtas = 8;   // resident CTAs per SM the bf16 kernel is launched with, at most
 
 constexpr int kListCap = kBins1;  // candidate list shares the histogram's storage
-#ifndef MOSAIC_TRACK_BITS
-#define MOSAIC_TRACK_BITS 21
-#endif
-constexpr int kTrackBits = MOSAIC_TRACK_BITS;    // width (log2, in key units) of a window carried from row to row
+constexpr int kTrackBits = 21;    // width (log2, in key units) of a window carried from row to row
 // The k-th score of a row scatters from row to row like 1/sqrt(cols): long rows get by with half the window
 // (half the candidates).
 __host__ __device__ constexpr int track_bits_for(int cols) { return cols >= 8192 ? kTrackBits - 1 : kTrackBits; }
@@ -211,9 +187,7 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
                     }
                 }
         __syncthreads();
-        MOSAIC_STAT_ADD(7, n_bin);
         if (n_bin == 1u) {
-            MOSAIC_STAT(6);
             T = sel.T;
             q = 1u;
             n_eq = 1u;
@@ -248,12 +222,9 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
 
         if (k > 0) {
             bool done = false;
-            MOSAIC_STAT(0);
             if (have_center) {
                 const uint32_t half = 1u << (kTrackBits - 1);
                 done = try_window(center > half ? center - half : 0u, kTrackBits);
-                MOSAIC_STAT(1);
-                if (done) MOSAIC_STAT(2);
             }
             if (!done) {
                 // window around the matching quantile of one key per thread
@@ -272,15 +243,12 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
                     }
                 }
                 __syncthreads();
-                MOSAIC_STAT(3);
                 if (sel.ok != 0u) {
                     const uint32_t lo = sel.lo;
                     done = try_window(lo, kSampleBits);
-                    if (done) MOSAIC_STAT(4);
                 }
             }
             if (!done) {
-                MOSAIC_STAT(5);
                 for (int b = tid; b < kBins1; b += NT) buf[b] = 0u;   // the list may have left entries
                 __syncthreads();
                 radix_select_row<V>(key_of, uk, buf, warp_tot, &sel3, NT, &T, &q, &n_eq);
@@ -302,7 +270,7 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
 // ---------------------------------------------------------------------------------------------
 constexpr int kFastV = 4;          // vectors (of 8 columns) per thread
 constexpr int kWinBins = 1024;     // histogram over the top 10 bits of a window
-constexpr int kRoundGroup = MOSAIC_ROUND_GROUP;   // candidate rounds of a warp whose loads are issued together
+constexpr int kRoundGroup = 4;            // candidate rounds of a warp whose loads are issued together
 constexpr int kQueueCap = 448;     // candidates a warp can queue (of its 1024 weights)
 constexpr int kBinListCap = 512;   // keys of one histogram bin that warp 0 will rank; also the sample size limit
 
@@ -738,7 +706,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         if (sel.ok == 0u) return 1;
         const uint32_t bin = sel.bin, r_bin = sel.q, n_bin = sel.n_eq;
         uint32_t T = sel.T;
-        MOSAIC_STAT_ADD(7, n_bin);
         if (n_bin > 1u) {
             if (n_bin > (uint32_t)kBinListCap) return 2;
             // collect the keys of that bin; warp 0 ranks them
@@ -785,8 +752,6 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 if (sel.ok == 0u) return 2;
                 T = sel.T;
             }
-        } else {
-            MOSAIC_STAT(6);
         }
 
         // prune: surely below lo, or a candidate whose exact key is <= T
@@ -887,22 +852,18 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
         }
         const int64_t row = r - row0;   // row inside the job
 
-        MOSAIC_STAT(0);
         int status = 1;
         uint32_t T_row = 0u;
         if (all_finite) {
             for (int tries = 0; tries < 2 && status == 1; ++tries) {
                 if (!win_valid || tries == 1) {
-                    MOSAIC_STAT(3);
                     set_window(sample_center(cur), kSampleBits);
                 }
                 if (!win_valid) break;
                 status = fast_attempt(cur, row, T_row);
-                if (status == 0) MOSAIC_STAT(win_w == track_bits ? 2 : 4);
             }
         }
         if (status != 0) {
-            MOSAIC_STAT(5);
             for (int b = tid; b < kWinBins; b += nt) slot[b] = 0u;
             __syncthreads();
             flush_mask();
@@ -988,21 +949,25 @@ static size_t fast_dyn_smem(int nt, int ring) {
 template <int MAXNT, int MINB, int NJ, int RING>
 static int launch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int nt, bool with_plan,
                              cudaStream_t st) {
-    static int blocks_per_sm[MAXNT / 32 + 1] = {0};
+    // The shared-memory opt-in and the occupancy belong to one device's copy of the kernel: both are
+    // looked up once per device and per CTA size (value -1: the opt-in was refused).
+    static DeviceCache blocks_per_sm[MAXNT / 32 + 1];
     const size_t dyn = fast_dyn_smem(nt, RING);
-    int& bps = blocks_per_sm[nt / 32];
-    if (bps == 0) {
+    const int bps = blocks_per_sm[nt / 32].get([&]() -> int {
         if (cudaFuncSetAttribute(prune_rows_bf16_kernel<MAXNT, MINB, NJ, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)fast_dyn_smem(MAXNT, RING)) != cudaSuccess)
-            return MOSAIC_ERR_CUDA;
+                                 (int)fast_dyn_smem(MAXNT, RING)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return -1;
+        }
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_bf16_kernel<MAXNT, MINB, NJ, RING>, nt, dyn) != cudaSuccess ||
             n < 1) {
             (void)cudaGetLastError();
             n = 1;
         }
-        bps = n > MOSAIC_FAST_MAX_CTAS ? MOSAIC_FAST_MAX_CTAS : n;
-    }
+        return n > kFastMaxCtas ? kFastMaxCtas : n;
+    });
+    if (bps < 0) return MOSAIC_ERR_CUDA;
     if (with_plan) {
         prune_plan_kernel<MAXNT, NJ><<<(unsigned)jobs.n, nt, 0, st>>>(jobs, cols);
         MOSAIC_LAUNCH_CHECK();
@@ -1019,12 +984,12 @@ static int dispatch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows,
                                cudaStream_t st) {
     // CTAs per SM are chosen so that a thread keeps about 128 registers where shared memory allows it: with the
     // thresholds in registers, a smaller budget spills them (rows of 5120 / 8192 columns ran 25 % slower at 80).
-    if (nt <= 128) return launch_prune_bf16<128, MOSAIC_MINB_SMALL, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 160) return launch_prune_bf16<160, 3, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 256) return launch_prune_bf16<256, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 352) return launch_prune_bf16<352, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
-    if (nt <= 384) return launch_prune_bf16<384, 2, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
-    return launch_prune_bf16<512, 1, NJ, MOSAIC_RING>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 128) return launch_prune_bf16<128, 4, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 160) return launch_prune_bf16<160, 3, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 256) return launch_prune_bf16<256, 2, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 352) return launch_prune_bf16<352, 2, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
+    if (nt <= 384) return launch_prune_bf16<384, 2, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
+    return launch_prune_bf16<512, 1, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
 }
 
 // Threads per CTA of the bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
@@ -1038,15 +1003,15 @@ static int fast_threads(int dtype, int64_t cols, int64_t k) {
 template <int DT, int V, int NT, int MINB>
 static int launch_prune(const void* W_in, void* W_out, int64_t rows, int cols, int64_t ldw, const float* norms, int k,
                         uint32_t* mask, cudaStream_t st) {
-    static int blocks_per_sm = 0;
-    if (blocks_per_sm == 0) {
+    static DeviceCache occupancy;
+    const int blocks_per_sm = occupancy.get([&]() -> int {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, prune_rows_kernel<DT, V, NT, MINB>, NT, 0) != cudaSuccess || n < 1) {
             (void)cudaGetLastError();
             n = 1;
         }
-        blocks_per_sm = n;
-    }
+        return n;
+    });
     int64_t grid = (int64_t)sm_count() * blocks_per_sm;
     if (grid > rows) grid = rows;
     const int words = (cols + 31) / 32;
@@ -1067,7 +1032,7 @@ static int dispatch_prune(const void* W_in, void* W_out, int64_t rows, int cols,
     if (nvec <= 64) MOSAIC_PRUNE_CASE(1, 64, 16);
     if (nvec <= 128) MOSAIC_PRUNE_CASE(1, 128, 8);
     if (nvec <= 256) MOSAIC_PRUNE_CASE(1, 256, 4);
-    if (nvec <= 2 * 256) MOSAIC_PRUNE_CASE(2, 256, MOSAIC_PRUNE_MINB_2X256);
+    if (nvec <= 2 * 256) MOSAIC_PRUNE_CASE(2, 256, 3);
     if (nvec <= 3 * 256) MOSAIC_PRUNE_CASE(3, 256, 3);
     if (nvec <= 2 * 512) MOSAIC_PRUNE_CASE(2, 512, 2);
     if (nvec <= 3 * 512) MOSAIC_PRUNE_CASE(3, 512, 1);
@@ -1083,17 +1048,6 @@ static int dispatch_prune(const void* W_in, void* W_out, int64_t rows, int cols,
 }  // namespace mosaic
 
 using namespace mosaic;
-
-#ifdef MOSAIC_PRUNE_STATS
-extern "C" int mosaic_debug_prune_stats(unsigned long long* host_out, int reset) {
-    if (cudaMemcpyFromSymbol(host_out, g_prune_stats, sizeof(unsigned long long) * 8) != cudaSuccess) return MOSAIC_ERR_CUDA;
-    if (reset) {
-        unsigned long long z[8] = {0};
-        if (cudaMemcpyToSymbol(g_prune_stats, z, sizeof(z)) != cudaSuccess) return MOSAIC_ERR_CUDA;
-    }
-    return MOSAIC_OK;
-}
-#endif
 
 extern "C" size_t mosaic_prune_unstructured_workspace_bytes(int64_t, int64_t) { return 0; }
 
@@ -1178,9 +1132,10 @@ extern "C" int mosaic_prune_unstructured_batch(const mosaic_prune_job* jobs, int
         plan_off[(size_t)i] = off;
         off += batch_plan_bytes(jobs[i], dtype);
     }
-    static PruneJobList<kBatchJobs> list;   // host staging of the kernel parameter (18 KB: kept off the stack)
-    static std::mutex list_mutex;
-    std::lock_guard<std::mutex> lock(list_mutex);
+    // host staging of the kernel parameter (18 KB: on the heap, one per call, so concurrent callers do not meet)
+    std::unique_ptr<PruneJobList<kBatchJobs>> list_mem(new (std::nothrow) PruneJobList<kBatchJobs>);
+    if (!list_mem) return MOSAIC_ERR_INVALID_ARG;
+    PruneJobList<kBatchJobs>& list = *list_mem;
     for (int64_t i = 0; i < n_jobs; ++i) {
         if (done[(size_t)i]) continue;
         const mosaic_prune_job& lead = jobs[i];

@@ -416,14 +416,15 @@ extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, i
 
     const size_t row_smem = align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
     if (row_smem > 200 * 1024) return MOSAIC_ERR_INVALID_ARG;   // a source row must fit in shared memory (cols <= 51200 fp32)
-    static bool attr_set[2] = {false, false};
-    if (!attr_set[dtype == MOSAIC_BF16]) {
+    static DeviceCache attr_set[2];   // the opt-in belongs to one device's copy of the kernel
+    const int opted = attr_set[dtype == MOSAIC_BF16].get([&]() -> int {
         const cudaError_t e = (dtype == MOSAIC_BF16)
             ? cudaFuncSetAttribute(compact_kernel<MOSAIC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
             : cudaFuncSetAttribute(compact_kernel<MOSAIC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) return MOSAIC_ERR_CUDA;
-        attr_set[dtype == MOSAIC_BF16] = true;
-    }
+        if (e != cudaSuccess) (void)cudaGetLastError();
+        return e == cudaSuccess ? 1 : -1;
+    });
+    if (opted < 0) return MOSAIC_ERR_CUDA;
     if (dtype == MOSAIC_BF16)
         compact_kernel<MOSAIC_BF16><<<(unsigned)out_rows, 256, row_smem, st>>>(W_in, cols, ldw, row_keep_units, n_ru, row_group,
                                                                               col_keep_units, n_cu, col_group, out_cols, W_out);

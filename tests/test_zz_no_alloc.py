@@ -16,7 +16,8 @@ import ctypes as C
 import pytest
 import torch
 
-from paper_2504_06323_b200 import api
+import oracle
+from paper_2504_06323_b200 import api, workloads as wl
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +56,8 @@ def test_static_scratch_matches_caller_workspace_twice_in_a_row():
         W, norms = _inputs(rows, cols, seed)
         want = _regular(W, norms, alpha)
         assert want[0] > 0                                   # the case does have outliers to count
+        ref = oracle.outlier_ratio(wl.to_numpy(W), norms.cpu().numpy(), alpha, "bf16")
+        assert ref["certified"] and want[0] == ref["count"]  # and both entry points agree with the CPU oracle
         assert _static_through_c_abi(W, norms, alpha) == want
         assert _static_through_c_abi(W, norms, alpha) == want
 
@@ -62,9 +65,19 @@ def test_static_scratch_matches_caller_workspace_twice_in_a_row():
 def test_static_scratch_refuses_what_does_not_fit():
     L = api.lib()
     assert L.mosaic_outlier_ratio_static_max_workspace_bytes() == 65536
-    # a row so wide that the first sweep needs more partial sums than the built-in array holds;
-    # refused from the sizes alone, before any pointer is touched
+    # rows so wide that the first sweep needs more partial sums than the built-in array holds:
+    # refused from the sizes alone.  Every pointer is a real device buffer of the right size, so
+    # that nothing could go wrong on the device even if the refusal were ever lost.
     cols = 16 * 1024 * 1024
     assert L.mosaic_outlier_ratio_workspace_bytes(8, cols) > 65536
-    rc = L.mosaic_outlier_ratio_static(256, 8, cols, cols, api.BF16, 256, C.c_float(5.0), 256, None, None)
+    W = torch.zeros(8, cols, dtype=torch.bfloat16, device="cuda")
+    norms = torch.ones(cols, dtype=torch.float32, device="cuda")
+    cnt = torch.full((1,), -7, dtype=torch.int64, device="cuda")
+    rc = L.mosaic_outlier_ratio_static(W.data_ptr(), 8, cols, cols, api.BF16, norms.data_ptr(), C.c_float(5.0),
+                                       cnt.data_ptr(), None, None)
     assert rc == -5, api.status_string(rc)
+    torch.cuda.synchronize()
+    assert cnt.item() == -7                                  # nothing was enqueued
+    # argument errors are reported before the scratch is even looked up
+    rc = L.mosaic_outlier_ratio_static(W.data_ptr(), 8, 4096, cols, api.BF16, None, C.c_float(5.0), cnt.data_ptr(), None, None)
+    assert rc == -2, api.status_string(rc)
