@@ -42,6 +42,7 @@ def lib():
     if _lib is None:
         _lib = C.CDLL(build())
         _lib.oracle_norm_certify.restype = C.c_int64
+        _lib.oracle_unit_scores_certify.restype = C.c_int64
         _lib.oracle_allocate_sparsity.restype = C.c_int
         _lib.oracle_num_threads.restype = C.c_int
     return _lib
@@ -168,6 +169,20 @@ def unit_scores(W: np.ndarray, norms, row_group: int = 1, col_group: int = 1, dt
     lib().oracle_unit_scores(_p(W), _i64(rows), _i64(cols), _i64(_ld(W)), code, _p(norms),
                              _i64(row_group), _i64(col_group), _p(rs), _p(cs))
     return rs, cs
+
+
+def unit_scores_certify(W: np.ndarray, norms, row_group: int = 1, col_group: int = 1, dtype=None):
+    """Per row unit and per column unit: True if no fp64 summation order can change the fp32 score."""
+    code = _code(W, dtype)
+    rows, cols = W.shape
+    assert rows % row_group == 0 and cols % col_group == 0
+    if norms is not None:
+        norms = np.ascontiguousarray(norms, np.float32)
+    r_ok = np.zeros(rows // row_group, np.uint8)
+    c_ok = np.zeros(cols // col_group, np.uint8)
+    lib().oracle_unit_scores_certify(_p(W), _i64(rows), _i64(cols), _i64(_ld(W)), code, _p(norms),
+                                     _i64(row_group), _i64(col_group), _p(r_ok), _p(c_ok))
+    return r_ok.astype(bool), c_ok.astype(bool)
 
 
 def rank_units(scores: np.ndarray, keep: int) -> np.ndarray:

@@ -363,6 +363,63 @@ void oracle_unit_scores(const void *W, int64_t rows, int64_t cols, int64_t ldw, 
 }
 
 /*
+ * Certification of the unit scores against summation order, in the manner of
+ * oracle_norm_certify: row_ok[u] / col_ok[v] = 1 iff the fp32 score of the unit
+ * is the same for the sequential fp64 sum above, for an extended-precision
+ * (long double) sum, and for that sum moved by +-n*2^-52 relative, n being the
+ * number of elements of the unit - i.e. no admissible order of the fp64
+ * additions can change the rounded score.  Either output may be NULL.  Returns
+ * the number of units NOT certified.
+ */
+static int unit_sum_certified(double s, long double e, double n_elems)
+{
+    double eps = n_elems * ldexp(1.0, -52);
+    float f0 = (float)s;
+    float f1 = (float)(double)e;
+    float f2 = (float)((double)e * (1.0 - eps));
+    float f3 = (float)((double)e * (1.0 + eps));
+    return float_bits(f0) == float_bits(f1) && float_bits(f1) == float_bits(f2) &&
+           float_bits(f1) == float_bits(f3);
+}
+
+int64_t oracle_unit_scores_certify(const void *W, int64_t rows, int64_t cols, int64_t ldw, int dtype,
+                                   const float *norms, int64_t row_group, int64_t col_group,
+                                   uint8_t *row_ok /* [rows/row_group] or NULL */,
+                                   uint8_t *col_ok /* [cols/col_group] or NULL */)
+{
+    int64_t n_ru = rows / row_group, n_cu = cols / col_group, bad = 0;
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+    for (int64_t u = 0; u < n_ru; ++u) {
+        double s = 0.0;
+        long double e = 0.0L;
+        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i)
+            for (int64_t j = 0; j < cols; ++j) {
+                double x = (double)weight_metric(norms ? norms[j] : 1.0f, load_elem(W, i * ldw + j, dtype));
+                s = s + x;
+                e = e + (long double)x;
+            }
+        int good = unit_sum_certified(s, e, (double)(row_group * cols));
+        if (row_ok) row_ok[u] = (uint8_t)good;
+        bad += good ? 0 : 1;
+    }
+#pragma omp parallel for schedule(static) reduction(+ : bad)
+    for (int64_t v = 0; v < n_cu; ++v) {
+        double s = 0.0;
+        long double e = 0.0L;
+        for (int64_t i = 0; i < rows; ++i)
+            for (int64_t j = v * col_group; j < (v + 1) * col_group; ++j) {
+                double x = (double)weight_metric(norms ? norms[j] : 1.0f, load_elem(W, i * ldw + j, dtype));
+                s = s + x;
+                e = e + (long double)x;
+            }
+        int good = unit_sum_certified(s, e, (double)(rows * col_group));
+        if (col_ok) col_ok[v] = (uint8_t)good;
+        bad += good ? 0 : 1;
+    }
+    return bad;
+}
+
+/*
  * Of n_units units, the (n_units - keep) that come first under (score
  * ascending, index ascending) are removed; keep_list receives the surviving
  * unit indices in ascending order.

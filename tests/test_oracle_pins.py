@@ -181,6 +181,53 @@ def test_outlier_planted_closed_form(dtype):
     assert oracle.outlier_ratio(Wc, ones, 1.0, dtype)["count"] == 0
 
 
+def test_outlier_certified_flags_a_score_on_or_next_to_the_threshold():
+    # four scores (1, 1, 1, x), alpha = 2: tau = (3 + x) / 2.
+    # x = 3 sits exactly on tau: not an outlier (strict), but any downward move of tau makes it
+    # one, so the count must NOT be certified.  x = the next fp32 above 3 clears tau by 2^-23,
+    # far more than the admissible C*2^-52: certified, one outlier.
+    ones = np.ones(4, np.float32)
+    r = oracle.outlier_ratio(np.array([[1, 1, 1, 3]], np.float32), ones, 2.0)
+    assert r["count"] == 0 and not r["certified"]
+    x = np.nextafter(np.float32(3), np.float32(4))
+    r = oracle.outlier_ratio(np.array([[1, 1, 1, x]], np.float32), ones, 2.0)
+    assert r["count"] == 1 and r["certified"]
+
+
+@pytest.mark.parametrize("log2_t,certified", [(-13, False), (-10, True)])
+def test_outlier_certified_margin_is_numel_times_2_pow_minus_52(log2_t, certified):
+    # C = 2^20 scores: all 1 except one 2 and one t = 2^log2_t, alpha = 2, so the sum C + t is
+    # exact in fp64 and tau = 2 (1 + t/C) lies t/C above the score 2 (relative).  The stated
+    # margin is C * 2^-52 = 2^-32: t/C = 2^-33 is inside it (not certified - a margin four times
+    # smaller would certify wrongly), t/C = 2^-30 is outside (certified - a margin four times
+    # larger would refuse wrongly).  Either way 2 is not above tau: no outliers.
+    n = 1024
+    W = np.ones((n, n), np.float32)
+    W[5, 7] = 2.0
+    W[900, 33] = np.float32(2.0 ** log2_t)
+    r = oracle.outlier_ratio(W, np.ones(n, np.float32), 2.0)
+    assert r["sum"] == float(n * n) + 2.0 ** log2_t
+    assert r["count"] == 0 and r["certified"] == certified
+
+
+def test_unit_scores_certify_flags_a_rounding_boundary():
+    # row 0: 1 + 2^-24 is exactly half way between the fp32 neighbours 1 and 1 + 2^-23 (the tie
+    # rounds to even, 1.0): any change of the fp64 sum flips the rounding - not certified.
+    # row 1: 1 + 2^-23 is an fp32 number: certified.  Columns: {1, 1}, {2^-24, 2^-23}, {0, 0}: exact.
+    W = np.array([[1.0, 2.0 ** -24, 0.0], [1.0, 2.0 ** -23, 0.0]], np.float32)
+    rs, cs = oracle.unit_scores(W, None)
+    r_ok, c_ok = oracle.unit_scores_certify(W, None)
+    assert rs[0] == np.float32(1.0) and rs[1] == np.float32(1.0 + 2.0 ** -23)
+    assert list(r_ok) == [False, True] and list(c_ok) == [True, True, True]
+    # as one row unit of two rows the sum is 2 + 3*2^-24 = 2 + 0.75 ulp(2): clear of a boundary
+    r_ok, c_ok = oracle.unit_scores_certify(W, None, 2, 3)
+    assert list(r_ok) == [True] and list(c_ok) == [True]
+    # norms enter the scores that are summed: with norm_1 = 1/2 row 0 is 1 + 2^-25 (clear of the
+    # boundary) and row 1 is 1 + 2^-24 (on it)
+    r_ok, _ = oracle.unit_scores_certify(W, np.array([1, 0.5, 1], np.float32))
+    assert list(r_ok) == [True, False]
+
+
 def test_outlier_uses_column_norms_not_row_norms():
     # 2 x 3 matrix of ones; norms (1, 1, 100): the outliers are the third COLUMN.
     W = np.ones((2, 3), np.float32)
