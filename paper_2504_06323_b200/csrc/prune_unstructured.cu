@@ -99,8 +99,10 @@ __global__ void __launch_bounds__(NT, MINB) prune_rows_kernel(const void* W_in, 
     // Score key of element (v, e) of the current row.  Columns past the end hold zero bits and
     // an infinite norm: their product is the canonical NaN 0x7FFFFFFF, the largest key there is,
     // and they come after every real column in the tie order, so no rank <= cols reaches them.
+    // (The sign bit is cleared: norms are >= +0 by contract, and a negative one must not index past
+    // the histograms - its rows then come out in an unspecified but memory-safe way.)
     auto key_of = [&](int v, int e) -> uint32_t {
-        return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e)));
+        return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))) & 0x7FFFFFFFu;
     };
 
     uint32_t center = 0u;
@@ -448,7 +450,7 @@ __device__ __noinline__ uint32_t generic_row_bf16(const uint4* my_vecs, int nt, 
             nrm[v][e] = (c < cols) ? __ldg(norms + c) : __int_as_float(0x7F800000);
         }
     }
-    auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))); };
+    auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))) & 0x7FFFFFFFu; };
     uint32_t T, q, n_eq, pruned[V];
     radix_select_row<V>(key_of, k, hist, warp_tot, sel3, nt, &T, &q, &n_eq);
     prune_flags<V>(key_of, T, q, n_eq, warp_tot, nt, pruned);
@@ -914,7 +916,7 @@ __global__ void __launch_bounds__(MAXNT, 1) prune_plan_kernel(const __grid_const
                 if (vec < nvec) raw[v].template load<true>(J.W_in + row * J.ldw + (int64_t)vec * kVec);
                 else raw[v].clear();
             }
-            auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))); };
+            auto key_of = [&](int v, int e) -> uint32_t { return __float_as_uint(__fmul_rn(nrm[v][e], raw[v].abs_f32(e))) & 0x7FFFFFFFu; };
             uint32_t q, n_eq;
             radix_select_row<V>(key_of, (uint32_t)J.k, hist, warp_tot, &sel3, nt, &Ts[s], &q, &n_eq);
         }
