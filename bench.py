@@ -11,9 +11,18 @@ selection + zeroing (+ keep bitmask) of every projection at 50 % average
 sparsity.  The metric is weight GB/s: bytes of weights scored and pruned per
 second of step time.  One JSON line is printed by rank 0.
 
-With N > 1 (torchrun, one process per GPU) every rank owns 32 layers of a
-32*N-layer model (weak scaling); the only exchange is one all_gather of the
-outlier counts between the two phases.
+With N > 1 every rank (one process per GPU) owns 32 layers of a 32*N-layer
+model (weak scaling); the only exchange is one all_gather of the outlier
+counts between the two phases.  Started as a single process with --gpus N,
+the script starts its N ranks itself (torch.distributed.run on 127.0.0.1);
+started by a launcher it finds RANK / WORLD_SIZE in the environment.
+
+After the headline region (N = 1 only) two more arms are timed and appended
+to the same JSON line: `structured` - rows and columns of every projection of
+the compaction-stress configuration ranked and compacted at f = 0.3 - and
+`composite` - one pass over the LLaMA-3-8B-shaped configuration: outlier
+sweeps, allocation, 50 % unstructured, then the coupled 20 % structured stage.
+--blocks chooses the arms (default: all).
 
 --impl reference times the CPU oracle (as it stands) on the host cores over a
 bounded sample of the same workload.
@@ -100,6 +109,17 @@ class ClockSampler:
         return out
 
 
+def cpu_model() -> str:
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 # --------------------------------------------------------------------------- CPU oracle sample
 def oracle_sample_inputs(cfg, frac_div: int, device):
     """1/frac_div of one layer: tokens/frac_div calibration tokens per input and rows/frac_div rows
@@ -169,6 +189,9 @@ def run_native(args, cfg):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    if world != args.gpus:
+        raise SystemExit(f"bench.py --gpus {args.gpus} is running as {world} rank(s): start it plainly (it launches its "
+                         f"ranks itself) or with --nproc-per-node equal to --gpus")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
@@ -196,6 +219,24 @@ def run_native(args, cfg):
     w_bytes = sum(st.W[l, p].numel() * cfg.itemsize for l in mine for p in PROJECTIONS)
     x_bytes_layer = sum(x.numel() * cfg.itemsize for x in X.values())
 
+    blocks = set(args.blocks.split(","))
+    if world == 1 and "headline" not in blocks:
+        # only the other arms (for profiling them alone): norms of one layer serve every layer
+        driver.accumulate_norms(st, mine[0], X)
+        for layer in mine[1:]:
+            for xk in cfg.x_keys():
+                st.norms[layer, xk].copy_(st.norms[mine[0], xk])
+        peak, _ = measured_peaks()
+        line = {"metric": METRIC, "n_gpus": 1, "note": "headline arm skipped (--blocks)"}
+        if "structured" in blocks:
+            line["structured"] = run_structured_block(args, st, peak)
+        del st, X
+        torch.cuda.empty_cache()
+        if "composite" in blocks:
+            line["composite"] = run_composite_block(args, dev, peak)
+        print(json.dumps(line), flush=True)
+        return
+
     def step(ev=None):
         """One pass of the whole path.  `ev`: five CUDA events recorded at the phase boundaries."""
         launches = 0
@@ -210,7 +251,7 @@ def run_native(args, cfg):
         _, k, _ = driver.plan_sparsity(total_cfg, counts)
         if ev: ev[3].record()
         driver.prune_unstructured_all(st, k)
-        launches += 2 * len({cfg.shape(p)[1] for p in PROJECTIONS})      # planning + pruning launch per distinct row length
+        launches += sum(prune_launches(c) for c in {cfg.shape(p)[1] for p in PROJECTIONS})
         if ev: ev[4].record()
         return launches
 
@@ -232,6 +273,9 @@ def run_native(args, cfg):
     barrier()
     total_ms = start.elapsed_time(end)
     phase_ms = [sum(ev[i].elapsed_time(ev[i + 1]) for ev in events) / args.steps for i in range(4)]
+    # per-step times: from one step's first event to the next step's (the last step ends at `end`)
+    step_ms = [events[i][0].elapsed_time(events[i + 1][0]) for i in range(args.steps - 1)] + [events[-1][0].elapsed_time(end)]
+    weight_ms = [ev[1].elapsed_time(ev[4]) for ev in events]
     clocks = sampler.stop() if rank == 0 else None
 
     t = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -251,14 +295,25 @@ def run_native(args, cfg):
         import oracle
         frac_div, reps = 2, 4
         Xs, Ws = oracle_sample_inputs(cfg, frac_div, dev)
+        threads = oracle.num_threads()
         t0 = time.perf_counter()
         nb = sum(oracle_sample_step(cfg, Xs, Ws) for _ in range(reps))
         dt = time.perf_counter() - t0
-        cpu = {"value": nb / dt / 1e9, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+        del Xs, Ws
+        # the same oracle on one thread, on a sample 16 times smaller
+        Xs, Ws = oracle_sample_inputs(cfg, 32, dev)
+        oracle.set_num_threads(1)
+        t1 = time.perf_counter()
+        nb1 = oracle_sample_step(cfg, Xs, Ws)
+        dt1 = time.perf_counter() - t1
+        oracle.set_num_threads(threads)
+        del Xs, Ws
+        cpu = {"value": nb / dt / 1e9, "unit": UNIT, "cores": threads, "kind": "oracle", "cpu_model": cpu_model(),
                "sample": f"{reps} passes over 1/{frac_div} of one layer: {cfg.tokens // frac_div} calibration tokens "
                          f"per input and rows/{frac_div} of each of the 7 projections ({nb / 1e6:.1f} MB of weights "
-                         f"in {dt:.1f} s)"}
-        del Xs, Ws
+                         f"in {dt:.1f} s)",
+               "one_thread": {"value": nb1 / dt1 / 1e9, "unit": UNIT, "cores": 1,
+                              "sample": f"1 pass over 1/32 of one layer ({nb1 / 1e6:.1f} MB of weights in {dt1:.1f} s)"}}
 
     if rank != 0:
         if world > 1:
@@ -289,6 +344,8 @@ def run_native(args, cfg):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
+        "ms_per_step_spread": {"min": min(step_ms), "median": statistics.median(step_ms), "max": max(step_ms),
+                               "note": "rank 0, CUDA events per step"},
         "config": {"workload": f"{cfg.name}: {n_layers} layers/GPU, hidden {cfg.hidden}, MLP {cfg.intermediate}, bf16 "
                                f"Student-t weights, {args.tokens or cfg.tokens} calibration tokens per projection input "
                                f"(one layer's activations resident and reused by every layer), alpha {cfg.alpha}, "
@@ -298,7 +355,8 @@ def run_native(args, cfg):
         "roofline": roofline, "cpu_baseline": cpu,
         "phases_ms": {"act_norms": phase_ms[0], "outlier_ratio": phase_ms[1], "counts_d2h_allocate": phase_ms[2],
                       "prune_unstructured": phase_ms[3]},
-        "weight_pass": {"ms": weight_pass_ms, "weight_GBps": w_bytes / (weight_pass_ms * 1e-3) / 1e9,
+        "weight_pass": {"ms": weight_pass_ms, "ms_min": min(weight_ms), "ms_median": statistics.median(weight_ms),
+                        "ms_max": max(weight_ms), "weight_GBps": w_bytes / (weight_pass_ms * 1e-3) / 1e9,
                         "compulsory_GBps": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9,
                         "frac_of_peak": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / peak,
                         "frac_of_8TBps": w_bytes * 6.125 / 2 / (weight_pass_ms * 1e-3) / 1e9 / 8000.0},
@@ -306,13 +364,123 @@ def run_native(args, cfg):
             {"kernel": "score_sum_kernel + outlier_count_kernel (two launches over all projections)", "bound": "hbm",
              "achieved": outl_gbs, "peak": peak, "unit": "GB/s", "frac": outl_gbs / peak,
              "algorithmic_bytes": "2 B/weight (the count sweep is a second read: 4 B/weight executed)"},
-            {"kernel": "prune_plan_kernel + prune_rows_bf16_kernel (one pair of launches per row length)", "bound": "hbm",
+            {"kernel": "prune_rows_warp_kernel (rows of 2048..8192 columns) + prune_plan_kernel / prune_rows_bf16_kernel (longer "
+                       "rows): one launch, or one pair, per row length", "bound": "hbm",
              "achieved": prune_gbs, "peak": peak, "unit": "GB/s", "frac": prune_gbs / peak,
              "algorithmic_bytes": "4.125 B/weight"}],
     }
+    # ---- the structured and the composite arm (N = 1): appended to the same line
+    if world == 1:
+        if "structured" in blocks:
+            line["structured"] = run_structured_block(args, st, peak)
+        del st, X
+        torch.cuda.empty_cache()
+        if "composite" in blocks:
+            line["composite"] = run_composite_block(args, dev, peak)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def prune_launches(cols: int) -> int:
+    """Kernel launches mosaic_prune_unstructured_batch makes for the jobs of one row length: the
+    warp-per-row kernel alone for rows of 2048..8192 columns, else a planning and a pruning launch."""
+    return 1 if 2048 <= cols <= 8192 else 2
+
+
+def _median_ms(fn, warmup=3, reps=5):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        fn()
+        e1.record()
+        torch.cuda.synchronize()
+        ts.append(e0.elapsed_time(e1))
+    return {"min": min(ts), "median": statistics.median(ts), "max": max(ts)}
+
+
+def run_structured_block(args, st, peak):
+    """Structured stage alone (steps C1-C3) on the compaction-stress shape: every projection of the
+    model on its own, floor(f*rows) rows and floor(f*cols) columns removed, dense compacted bf16 out.
+    Algorithmic bytes per weight: 2 (scores: W read once) + 2(1-f) (kept rows read) + 2(1-f)^2 (written)."""
+    from paper_2504_06323_b200 import driver
+    f = 0.3
+    t = _median_ms(lambda: driver.prune_structured_model(st, f, coupled=False))
+    w = sum(x.numel() for x in st.W.values())
+    nbytes = w * (2.0 + 2.0 * (1 - f) + 2.0 * (1 - f) ** 2)
+    gbs = nbytes / (t["median"] * 1e-3) / 1e9
+    return {"workload": f"llama7b_structured shape: {len(st.layers)} layers x 7 projections, rows and columns of every "
+                        f"projection independently, f = {f}", "ms": t["median"], "ms_min": t["min"], "ms_max": t["max"],
+            "algorithmic_bytes": nbytes, "bytes_per_weight": nbytes / w, "achieved": gbs, "unit": "GB/s", "peak": peak,
+            "frac": gbs / peak, "projections": len(st.W)}
+
+
+def run_composite_block(args, dev, peak):
+    """One pass over the LLaMA-3-8B-shaped configuration (GQA, MLP 14336) with the norms in place:
+    outlier sweeps, allocation, 50 % unstructured, coupled 20 % structured (MLP channels; KV groups)."""
+    from paper_2504_06323_b200 import driver
+    cfg = wl.CONFIGS["llama3_8b"]
+    n_layers = args.layers or cfg.n_layers
+    cfg_n = wl.scaled(cfg, n_layers=n_layers)
+    st = driver.alloc_model(cfg_n, dev)
+    X = driver.make_activations(cfg, 0, dev, tokens=min(args.tokens or 32768, 32768))   # norms only have to be realistic
+    driver.accumulate_norms(st, 0, X)
+    del X
+    for layer in st.layers[1:]:
+        for xk in cfg.x_keys():
+            st.norms[layer, xk].copy_(st.norms[0, xk])
+    frac = cfg.extra["structured_frac"]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+
+    def one_pass(record=False):
+        if record: ev[0].record()
+        driver.count_outliers_all(st)
+        if record: ev[1].record()
+        counts = driver.exchange_counts(st.counts, cfg_n.n_layers, 0, 1)
+        _, k, _ = driver.plan_sparsity(cfg_n, counts)
+        if record: ev[2].record()
+        driver.prune_unstructured_all(st, k)
+        if record: ev[3].record()
+        sources = {layer: {pr: st.W_out[layer, pr] for pr in PROJECTIONS} for layer in st.layers}
+        out = driver.prune_structured_model(st, frac, coupled=True, sources=sources)
+        if record: ev[4].record()
+        return out
+
+    for _ in range(3):
+        one_pass()
+    torch.cuda.synchronize()
+    runs = []
+    for _ in range(5):
+        one_pass(record=True)
+        torch.cuda.synchronize()
+        runs.append([ev[i].elapsed_time(ev[i + 1]) for i in range(4)])
+    med = [statistics.median(r[i] for r in runs) for i in range(4)]
+    w = sum(x.numel() for x in st.W.values())
+    # structured stage: scores read every weight once; compaction reads the kept rows whole and writes the kept part
+    keep = 1.0 - int(frac * cfg.intermediate) / cfg.intermediate
+    keep_a = 1.0 - int(frac * cfg.n_kv_heads) / cfg.n_kv_heads
+    c_bytes = 0.0
+    for layer in st.layers:
+        for pr in PROJECTIONS:
+            n = st.W[layer, pr].numel()
+            kr, kc = {"gate": (keep, 1.0), "up": (keep, 1.0), "down": (1.0, keep), "q": (keep_a, 1.0), "k": (keep_a, 1.0),
+                      "v": (keep_a, 1.0), "o": (1.0, keep_a)}[pr]
+            c_bytes += n * (2.0 + 2.0 * kr + 2.0 * kr * kc)
+    total = sum(med)
+    return {"workload": f"llama3_8b shape: {n_layers} layers, GQA 32/8 heads, MLP 14336; norms in place; p = {cfg.p}, "
+                        f"structured f = {frac} (coupled MLP channels and KV groups)",
+            "ms": total, "phases_ms": {"outlier_ratio": med[0], "counts_d2h_allocate": med[1], "prune_unstructured": med[2],
+                                       "structured_coupled": med[3]},
+            "algorithmic_bytes": {"outlier_ratio": 2.0 * w, "prune_unstructured": 4.125 * w, "structured_coupled": c_bytes},
+            "achieved": {"outlier_ratio": 2.0 * w / (med[0] * 1e-3) / 1e9, "prune_unstructured": 4.125 * w / (med[2] * 1e-3) / 1e9,
+                         "structured_coupled": c_bytes / (med[3] * 1e-3) / 1e9}, "unit": "GB/s", "peak": peak,
+            "frac": {"outlier_ratio": 2.0 * w / (med[0] * 1e-3) / 1e9 / peak,
+                     "prune_unstructured": 4.125 * w / (med[2] * 1e-3) / 1e9 / peak,
+                     "structured_coupled": c_bytes / (med[3] * 1e-3) / 1e9 / peak}}
 
 
 def run_e2e(args, cfg, total_cfg, st, mine, dev, rank, world, barrier):
@@ -417,12 +585,18 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--e2e-chunk", type=int, default=16384)
+    ap.add_argument("--blocks", default="headline,structured,composite",
+                    help="arms appended to the line at N = 1: headline, structured, composite")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]
     if args.impl == "reference":
         run_reference(args, cfg)
-    else:
-        run_native(args, cfg)
+        return
+    from paper_2504_06323_b200 import launch
+    if args.gpus > 1 and not launch.under_launcher():
+        # started plainly: become the launcher of our own N ranks (rank 0 prints the line)
+        sys.exit(launch.spawn_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
+    run_native(args, cfg)
 
 
 if __name__ == "__main__":

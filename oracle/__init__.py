@@ -73,6 +73,11 @@ def num_threads() -> int:
     return int(lib().oracle_num_threads())
 
 
+def set_num_threads(n: int) -> None:
+    """Threads of the oracle's parallel loops (for timing; results never depend on it)."""
+    lib().oracle_set_num_threads(C.c_int(int(n)))
+
+
 def act_sumsq(X: np.ndarray, sumsq: np.ndarray | None = None, dtype=None) -> np.ndarray:
     """sumsq[j] += sum_t X[t,j]^2 in fp64, t in order (the norm term of Eq. 5)."""
     code = _code(X, dtype)

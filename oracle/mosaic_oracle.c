@@ -465,6 +465,16 @@ void oracle_compact(const void *W, int64_t ldw, int dtype, const int32_t *row_ke
     }
 }
 
+/* Thread count of the parallel loops above (timing only: no result depends on it). */
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n > 0) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int oracle_num_threads(void)
 {
     int n = 1;

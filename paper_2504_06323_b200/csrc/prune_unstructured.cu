@@ -36,6 +36,7 @@
 #include <new>
 #include <vector>
 
+#include "prune_jobs.cuh"
 #include "select.cuh"
 
 namespace mosaic {
@@ -321,24 +322,6 @@ __device__ __forceinline__ int flag_elem(int b) {   // flag bit of comb_flags ->
     const int i = (15 | (half << 4)) - b;
     return (i << 1) | half;
 }
-
-// One matrix to prune, as the kernels see it.  A launch works through a list of them, all with
-// the same number of columns; rows are numbered across the list (row0 = first global row).
-struct PruneJob {
-    const uint16_t* W_in;
-    uint16_t* W_out;
-    const float* norms;
-    uint8_t* mask;          // keep bitmask as bytes, or nullptr
-    uint32_t* plan;         // window and thresholds prepared by prune_plan_kernel, or nullptr
-    int64_t rows, ldw, row0;
-    int k, mask_row_bytes;
-};
-template <int NJ>
-struct PruneJobList {
-    int n;
-    PruneJob job[NJ];
-};
-constexpr int kBatchJobs = 256;   // jobs per launch of the batched kernels (the list travels as a kernel parameter)
 
 // Layout of a plan (32-bit words): [0] valid, [1] window lo, [2] window width log2, [3] unused, then
 // for every vector slot vec = v*nt + tid eight words: Alo[0..3], Ahi[0..3].
@@ -790,7 +773,7 @@ __global__ void __launch_bounds__(MAXNT, MINB) prune_rows_bf16_kernel(const __gr
                 o.y = r.y & lane_mask_from_flags((r.y | 0x80008000u) - Alo[v][1]);
                 o.z = r.z & lane_mask_from_flags((r.z | 0x80008000u) - Alo[v][2]);
                 o.w = r.w & lane_mask_from_flags((r.w | 0x80008000u) - Alo[v][3]);
-                st_stream16(out_row + (int64_t)vec * kVec, o);
+                if (W_out != nullptr) st_stream16(out_row + (int64_t)vec * kVec, o);
             }
             if (mask_bytes != nullptr) {
                 uint32_t keep = 0u;
@@ -994,7 +977,12 @@ static int dispatch_prune_bf16(const PruneJobList<NJ>& jobs, int64_t total_rows,
     return launch_prune_bf16<512, 1, NJ, kRing>(jobs, total_rows, cols, nt, with_plan, st);
 }
 
-// Threads per CTA of the bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
+// True iff the warp-per-row kernel (prune_warp.cu) takes rows of this shape.
+static bool warp_kernel_takes(int dtype, int64_t cols, int64_t k) {
+    return dtype == MOSAIC_BF16 && cols % kVec == 0 && k > 0 && k < cols && cols >= kWarpMinCols && cols <= kWarpMaxCols;
+}
+
+// Threads per CTA of the CTA-per-row bf16 kernel for rows of `cols` columns, or 0 if the shape is not for it.
 static int fast_threads(int dtype, int64_t cols, int64_t k) {
     if (dtype != MOSAIC_BF16 || cols % kVec != 0 || k <= 0 || k >= cols) return 0;
     const int64_t nvec = cols / kVec;
@@ -1058,12 +1046,16 @@ static int validate_prune(const void* W_in, void* W_out, int64_t rows, int64_t c
                           const float* norms, int64_t k, uint32_t* mask_out) {
     int rc = check_matrix(W_in, rows, cols, ldw, dtype);
     if (rc != MOSAIC_OK) return rc;
-    rc = check_matrix(W_out, rows, cols, ldw, dtype);
-    if (rc != MOSAIC_OK) return rc;
+    if (W_out != nullptr) {   // W_out == NULL: mask-only mode, the keep bitmask is the only output
+        rc = check_matrix(W_out, rows, cols, ldw, dtype);
+        if (rc != MOSAIC_OK) return rc;
+    } else if (mask_out == nullptr) {
+        return MOSAIC_ERR_NULL_PTR;
+    }
     if (!norms) return MOSAIC_ERR_NULL_PTR;
     if ((reinterpret_cast<uintptr_t>(norms) & 3u) || (reinterpret_cast<uintptr_t>(mask_out) & 3u)) return MOSAIC_ERR_MISALIGNED;
     if (k < 0 || k > cols || cols > 65536) return MOSAIC_ERR_INVALID_ARG;
-    if (rows > 0 && W_in != W_out) {
+    if (rows > 0 && W_out != nullptr && W_in != W_out) {
         const size_t span = ((size_t)(rows - 1) * (size_t)ldw + (size_t)cols) * elem_size(dtype);
         const char *a = static_cast<const char*>(W_in), *b = static_cast<const char*>(W_out);
         if (a < b + span && b < a + span) return MOSAIC_ERR_ALIASING;
@@ -1080,6 +1072,14 @@ extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t 
     if (rc != MOSAIC_OK) return rc;
     if (rows == 0) return MOSAIC_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (warp_kernel_takes(dtype, cols, k)) {
+        PruneJobList<1> one;
+        one.n = 1;
+        one.job[0] = PruneJob{static_cast<const uint16_t*>(W_in), static_cast<uint16_t*>(W_out), norms,
+                              reinterpret_cast<uint8_t*>(mask_out), nullptr, rows, ldw, 0, (int)k,
+                              (int)((cols + 31) / 32) * 4};
+        return launch_prune_warp(one, rows, (int)cols, st);
+    }
     if (const int nt = fast_threads(dtype, cols, k)) {
         PruneJobList<1> one;
         one.n = 1;
@@ -1096,6 +1096,7 @@ extern "C" int mosaic_prune_unstructured(const void* W_in, void* W_out, int64_t 
 // Workspace of the batched call: one plan (window + per-column thresholds) per job that the bf16
 // kernel takes, 256-byte aligned, in job order.
 static size_t batch_plan_bytes(const mosaic_prune_job& j, int dtype) {
+    if (warp_kernel_takes(dtype, j.cols, j.k)) return 0;   // that kernel finds its windows itself
     const int nt = (j.rows > 0) ? fast_threads(dtype, j.cols, j.k) : 0;
     return nt ? align_up(plan_words(nt) * sizeof(uint32_t), 256) : 0;
 }
@@ -1141,8 +1142,33 @@ extern "C" int mosaic_prune_unstructured_batch(const mosaic_prune_job* jobs, int
     for (int64_t i = 0; i < n_jobs; ++i) {
         if (done[(size_t)i]) continue;
         const mosaic_prune_job& lead = jobs[i];
-        const int nt = (lead.rows > 0) ? fast_threads(dtype, lead.cols, lead.k) : 0;
-        if (nt == 0) {
+        const bool by_warp = lead.rows > 0 && warp_kernel_takes(dtype, lead.cols, lead.k);
+        const int nt = (lead.rows > 0 && !by_warp) ? fast_threads(dtype, lead.cols, lead.k) : 0;
+        if (by_warp) {   // all jobs of this row length that the warp-per-row kernel takes, kBatchJobs per launch
+            list.n = 0;
+            int64_t total_rows = 0;
+            for (int64_t m = i; m < n_jobs; ++m) {
+                const mosaic_prune_job& j = jobs[m];
+                if (done[(size_t)m] || j.cols != lead.cols || j.rows <= 0 || !warp_kernel_takes(dtype, j.cols, j.k)) continue;
+                done[(size_t)m] = 1;
+                list.job[list.n] = PruneJob{static_cast<const uint16_t*>(j.W_in), static_cast<uint16_t*>(j.W_out), j.norms,
+                                            reinterpret_cast<uint8_t*>(j.mask_out), nullptr, j.rows, j.ldw, total_rows,
+                                            (int)j.k, (int)((j.cols + 31) / 32) * 4};
+                total_rows += j.rows;
+                if (++list.n == kBatchJobs) {
+                    const int rc = launch_prune_warp(list, total_rows, (int)lead.cols, st);
+                    if (rc != MOSAIC_OK) return rc;
+                    list.n = 0;
+                    total_rows = 0;
+                }
+            }
+            if (list.n > 0) {
+                const int rc = launch_prune_warp(list, total_rows, (int)lead.cols, st);
+                if (rc != MOSAIC_OK) return rc;
+            }
+            continue;
+        }
+        if (nt == 0) {   // short or very long rows, fp32, k = 0 or k = cols: the general kernel, one launch per job
             done[(size_t)i] = 1;
             const int rc = mosaic_prune_unstructured(lead.W_in, lead.W_out, lead.rows, lead.cols, lead.ldw, dtype, lead.norms,
                                                      lead.k, lead.mask_out, nullptr, 0, stream);
@@ -1153,7 +1179,9 @@ extern "C" int mosaic_prune_unstructured_batch(const mosaic_prune_job* jobs, int
         int64_t total_rows = 0;
         for (int64_t m = i; m < n_jobs; ++m) {
             const mosaic_prune_job& j = jobs[m];
-            if (done[(size_t)m] || j.cols != lead.cols || j.rows <= 0 || fast_threads(dtype, j.cols, j.k) == 0) continue;
+            if (done[(size_t)m] || j.cols != lead.cols || j.rows <= 0 || warp_kernel_takes(dtype, j.cols, j.k) ||
+                fast_threads(dtype, j.cols, j.k) == 0)
+                continue;
             done[(size_t)m] = 1;
             list.job[list.n] = PruneJob{static_cast<const uint16_t*>(j.W_in), static_cast<uint16_t*>(j.W_out), j.norms,
                                         reinterpret_cast<uint8_t*>(j.mask_out),

@@ -217,7 +217,8 @@ __device__ __forceinline__ void prune_flags(KeyOf key_of, uint32_t T, uint32_t q
     }
 }
 
-// Write W' (pruned entries as +0, the others bit for bit) and the keep bitmask of one row.
+// Write W' (pruned entries as +0, the others bit for bit; skipped when W_out is null) and the keep
+// bitmask of one row.
 template <int DT, int V>
 __device__ __forceinline__ void store_row(Raw8<DT> (&raw)[V], const uint32_t (&pruned)[V], void* W_out, int64_t row_off,
                                           int cols, int nvec, int nt, uint8_t* mask_bytes, int64_t mask_off,
@@ -227,7 +228,7 @@ __device__ __forceinline__ void store_row(Raw8<DT> (&raw)[V], const uint32_t (&p
     for (int v = 0; v < V; ++v) {
         const int vec = v * nt + tid;
         const int c0 = vec * kVec;
-        if (vec < nvec) {
+        if (vec < nvec && W_out != nullptr) {
 #pragma unroll
             for (int e = 0; e < kVec; ++e)
                 if (pruned[v] & (1u << e)) raw[v].zero(e);

@@ -81,3 +81,22 @@ def test_two_ranks_agree_with_one_process():
         assert np.array_equal(np.array(s).view(np.uint64), s_ref.view(np.uint64))
         assert k == list(k_ref)
     assert len(set(results[0][4])) > 1
+
+
+def test_launcher_starts_two_ranks_that_agree_with_one_process(tmp_path):
+    # the launcher bench.py --gpus N uses (torch.distributed.run on 127.0.0.1), here with gloo ranks on CPU
+    import json
+    from paper_2504_06323_b200 import launch
+    build.build_library()
+    worker = os.path.join(os.path.dirname(os.path.abspath(__file__)), "rank_worker.py")
+    rc = launch.spawn_ranks(2, worker, [str(tmp_path)], timeout=300)
+    assert rc == 0
+    cfg = _cfg()
+    want_counts = _counts_for(cfg, list(range(cfg.n_layers)))
+    s_ref, k_ref, _ = op.plan(cfg, want_counts, cfg.n_layers)
+    for rank in range(2):
+        with open(tmp_path / f"rank{rank}.json") as f:
+            r = json.load(f)
+        assert r["world"] == 2 and r["mine"] == [l for l in range(cfg.n_layers) if l % 2 == rank]
+        assert r["counts"] == want_counts and r["k"] == list(k_ref)
+        assert np.array_equal(np.array(r["s"]).view(np.uint64), s_ref.view(np.uint64))
