@@ -7,7 +7,8 @@
 // for a window [lo, hi) of score keys that should contain every row's threshold, per column the
 // bf16 magnitude patterns A_lo[j] <= / A_hi[j] >= below / from which a weight's score is surely
 // under lo / at least hi (the score norm_j * |w| is monotone in |w|).  The window is centred on
-// the median of the exact thresholds of three rows of the job (first, middle, last).
+// the median of one estimate per warp: the matching quantile of the exact scores of a quarter of
+// one row of the job (rows spread evenly over the matrix), selected in registers.
 //
 // Each warp then works on whole rows by itself, with no block barrier on the row path:
 //   1. the row arrives in the warp's shared-memory buffer by cp.async;
@@ -296,7 +297,8 @@ __device__ __forceinline__ void thresholds_of_vector(const float* nrm8, float fl
 
 // blockDim.x = 32 * warps (warps >= 3); dynamic shared memory = off_warp0 + warps * per_warp of warp_layout(cols).
 // Every job: cols % 8 == 0, kWarpMinCols <= cols <= V * 256, 0 < k < cols.
-template <int V, int NJ>
+// FULL: cols == V * 256, so every vector slot v * 32 + lane is inside the row and no bounds test is needed.
+template <int V, int NJ, bool FULL>
 __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(const __grid_constant__ PruneJobList<NJ> jobs,
                                                                              int64_t total_rows, int cols) {
     extern __shared__ __align__(16) unsigned char smem[];
@@ -307,7 +309,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
     uint4* alo = reinterpret_cast<uint4*>(smem + L.off_alo);
     uint4* ahi = reinterpret_cast<uint4*>(smem + L.off_ahi);
     float* nrm = reinterpret_cast<float*>(smem + L.off_nrm);
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..2] sample thresholds
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates
     unsigned char* mine = smem + L.off_warp0 + (size_t)wid * L.per_warp;
     uint4* row = reinterpret_cast<uint4*>(mine);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(mine);
@@ -354,25 +356,60 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         bool valid = __syncthreads_and(fin ? 1 : 0) != 0;
         uint32_t lo = 0u;
         if (valid) {
-            for (int s = wid; s < 3; s += nwarps) {
-                const int64_t srow = (s == 0) ? 0 : (s == 1 ? J.rows / 2 : J.rows - 1);
+            // One estimate per warp: the k-th score of row (rows-1)*wid/(nwarps-1), taken as the matching
+            // quantile of the exact keys of four of each lane's vectors (a quarter of the row), which
+            // the lane keeps in registers through a 4 x 8-bit radix select.
+            {
+                const int64_t srow = (J.rows - 1) * wid / (nwarps > 1 ? nwarps - 1 : 1);
                 const uint16_t* src = J.W_in + srow * ldw;
+                uint32_t key[32];
+                uint32_t n_valid = 0u;
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const int vec = v * 32 + lane;
-                    if (vec < nvec) cp_async16(&row[vec], src + (int64_t)vec * kVec);
+                for (int i = 0; i < 4; ++i) {
+                    const int vec = (i * (V / 4)) * 32 + lane;
+                    if (FULL || vec < nvec) {
+                        const uint4 r = ld_stream16(src + (int64_t)vec * kVec);   // (in place, another CTA may be writing this row: any value will do for an estimate)
+                        const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
+                        const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = exact_key(r, n8, e);
+                        n_valid += 8u;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = 0xFFFFFFFFu;   // matches no prefix: in no histogram
+                    }
                 }
-                cp_async_commit_wait();
-                __syncwarp();
-                uint32_t T, q, n_eq;
-                warp_exact_select<V>(row, nrm, nvec, uk, hist, &T, &q, &n_eq);
-                if (lane == 0) misc[s] = T;
-                __syncwarp();
+                n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
+                uint32_t rank = (uint32_t)(((uint64_t)uk * n_valid + (uint32_t)cols / 2u) / (uint32_t)cols);
+                rank = rank < 1u ? 1u : (rank > n_valid ? n_valid : rank);
+                uint32_t prefix = 0u, pmask = 0u;
+#pragma unroll 1
+                for (int sh = 24; sh >= 0; sh -= 8) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if ((key[i] & pmask) == prefix && key[i] != 0xFFFFFFFFu) atomicAdd(&hist[(key[i] >> sh) & 0xFFu], 1u);
+                    __syncwarp();
+                    uint32_t bin = 0u, rr = 0u, cc = 0u;
+                    warp_find_bin(hist, 0u, rank, lane, &bin, &rr, &cc);
+                    prefix |= bin << sh;
+                    pmask |= 0xFFu << sh;
+                    rank = rr;
+                    __syncwarp();
+                }
+                if (lane == 0) misc[wid] = prefix;
             }
             __syncthreads();
-            const uint32_t t0 = misc[0], t1 = misc[1], t2 = misc[2];
-            const uint32_t mx = max(max(t0, t1), t2), mn = min(min(t0, t1), t2);
-            const uint32_t center = (uint32_t)((uint64_t)t0 + t1 + t2 - mx - mn);
+            // median of the estimates (every thread ranks them the same way: by value, then by warp)
+            uint32_t center = 0u;
+            for (int a = 0; a < nwarps; ++a) {
+                const uint32_t va = misc[a];
+                int less = 0;
+                for (int b = 0; b < nwarps; ++b) {
+                    const uint32_t vb = misc[b];
+                    less += (vb < va || (vb == va && b < a)) ? 1 : 0;
+                }
+                if (less == nwarps / 2) center = va;
+            }
             const uint32_t half = width >> 1;
             // refused where scores could be subnormal (lo < 2^24) or the window could reach inf
             valid = center >= (1u << 24) + half && center - half <= 0x7F7FFFFFu - width;
@@ -394,7 +431,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 const int vec = v * 32 + lane;
-                if (vec < nvec) cp_async16(&row[vec], src + (int64_t)vec * kVec);
+                if (FULL || vec < nvec) cp_async16(&row[vec], src + (int64_t)vec * kVec);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
@@ -416,7 +453,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const int vec = v * 32 + lane;
-                    if (vec < nvec) {
+                    if (FULL || vec < nvec) {
                         const uint4 rr = row[vec], a = alo[vec], h = ahi[vec];
                         const uint32_t x0 = rr.x | 0x80008000u, x1 = rr.y | 0x80008000u, x2 = rr.z | 0x80008000u,
                                        x3 = rr.w | 0x80008000u;
@@ -505,7 +542,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
 #pragma unroll
                         for (int v = 0; v < V; ++v) {
                             const int vec = v * 32 + lane;
-                            if (vec < nvec) {
+                            if (FULL || vec < nvec) {
                                 const uint4 rr = row[vec], a = alo[vec];
                                 const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
                                                t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
@@ -531,7 +568,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
     }
 }
 
-template <int V, int NJ>
+template <int V, int NJ, bool FULL>
 static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, cudaStream_t st) {
     const int warps = warps_for(cols);
     if (warps < 3) return MOSAIC_ERR_INVALID_ARG;
@@ -539,7 +576,7 @@ static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int c
     const size_t dyn = (size_t)L.off_warp0 + (size_t)warps * L.per_warp;
     static DeviceCache opted;   // the shared-memory opt-in belongs to one device's copy of the kernel
     const int ok = opted.get([&]() -> int {
-        if (cudaFuncSetAttribute(prune_rows_warp_kernel<V, NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(prune_rows_warp_kernel<V, NJ, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kWSmemBudget) != cudaSuccess) {
             (void)cudaGetLastError();
             return -1;
@@ -551,7 +588,7 @@ static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int c
     const int64_t need = (total_rows + warps - 1) / warps;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    prune_rows_warp_kernel<V, NJ><<<(unsigned)grid, warps * 32, dyn, st>>>(jobs, total_rows, cols);
+    prune_rows_warp_kernel<V, NJ, FULL><<<(unsigned)grid, warps * 32, dyn, st>>>(jobs, total_rows, cols);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
@@ -559,12 +596,18 @@ static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int c
 template <int NJ>
 static int launch_warp_any(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, cudaStream_t st) {
     const int v = (cols / 8 + 31) / 32;   // vectors per lane
-    if (v <= 8) return launch_warp_v<8, NJ>(jobs, total_rows, cols, st);
-    if (v <= 12) return launch_warp_v<12, NJ>(jobs, total_rows, cols, st);
-    if (v <= 16) return launch_warp_v<16, NJ>(jobs, total_rows, cols, st);
-    if (v <= 20) return launch_warp_v<20, NJ>(jobs, total_rows, cols, st);
-    if (v <= 24) return launch_warp_v<24, NJ>(jobs, total_rows, cols, st);
-    if (v <= 32) return launch_warp_v<32, NJ>(jobs, total_rows, cols, st);
+    const bool full = cols % 256 == 0;
+#define MOSAIC_WARP_CASE(V)                                                                       \
+    if (v <= V)                                                                                   \
+        return (full && cols == V * 256) ? launch_warp_v<V, NJ, true>(jobs, total_rows, cols, st) \
+                                         : launch_warp_v<V, NJ, false>(jobs, total_rows, cols, st)
+    MOSAIC_WARP_CASE(8);
+    MOSAIC_WARP_CASE(12);
+    MOSAIC_WARP_CASE(16);
+    MOSAIC_WARP_CASE(20);
+    MOSAIC_WARP_CASE(24);
+    MOSAIC_WARP_CASE(32);
+#undef MOSAIC_WARP_CASE
     return MOSAIC_ERR_INVALID_ARG;
 }
 
