@@ -364,8 +364,7 @@ def run_native(args, cfg):
             {"kernel": "score_sum_kernel + outlier_count_kernel (two launches over all projections)", "bound": "hbm",
              "achieved": outl_gbs, "peak": peak, "unit": "GB/s", "frac": outl_gbs / peak,
              "algorithmic_bytes": "2 B/weight (the count sweep is a second read: 4 B/weight executed)"},
-            {"kernel": "prune_rows_warp_kernel (rows of 2048..8192 columns) + prune_plan_kernel / prune_rows_bf16_kernel (longer "
-                       "rows): one launch, or one pair, per row length", "bound": "hbm",
+            {"kernel": "prune_rows_warp_kernel (one launch per row length)", "bound": "hbm",
              "achieved": prune_gbs, "peak": peak, "unit": "GB/s", "frac": prune_gbs / peak,
              "algorithmic_bytes": "4.125 B/weight"}],
     }
@@ -383,9 +382,9 @@ def run_native(args, cfg):
 
 
 def prune_launches(cols: int) -> int:
-    """Kernel launches mosaic_prune_unstructured_batch makes for the jobs of one row length: the
-    warp-per-row kernel alone for rows of 2048..8192 columns, else a planning and a pruning launch."""
-    return 1 if 2048 <= cols <= 8192 else 2
+    """Kernel launches mosaic_prune_unstructured_batch makes for the (<= 256) jobs of one row length:
+    one launch of the row-group kernel (bf16 rows of 2048..16384 columns)."""
+    return 1
 
 
 def _median_ms(fn, warmup=3, reps=5):

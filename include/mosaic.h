@@ -207,11 +207,14 @@ int mosaic_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numel
  * entries that come first under (w_ij ascending, j ascending) become +0; all
  * other entries keep their bits.
  *   W_in      device, [rows, cols]; W_out device, same shape/ld; W_out may be
- *             W_in exactly (in place); any other overlap -> MOSAIC_ERR_ALIASING
+ *             W_in exactly (in place); any other overlap -> MOSAIC_ERR_ALIASING.
+ *             W_out == NULL: mask-only mode, the keep bitmask is the only
+ *             output (mask_out is then required) and W_in is left untouched
  *   k         0 <= k <= cols
  *   mask_out  device, [rows, ceil(cols/32)] uint32 or NULL; bit j%32 of word
  *             j/32 is 1 for a kept entry; padding bits are 0
  *   cols      at most 65536
+ *   ws        unused (the call needs no scratch); may be NULL
  * ------------------------------------------------------------------------- */
 size_t mosaic_prune_unstructured_workspace_bytes(int64_t rows, int64_t cols);
 int mosaic_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64_t cols,
@@ -228,10 +231,12 @@ int mosaic_prune_unstructured(const void *W_in, void *W_out, int64_t rows, int64
  *            every pointer inside a descriptor is a device pointer with the
  *            meaning and alignment rules of mosaic_prune_unstructured
  *   dtype    one dtype for the whole list
- *   ws       device scratch, >= mosaic_prune_unstructured_batch_workspace_bytes
- *            for the same list; it receives, per job, the key window and the
- *            per-column thresholds a planning kernel derives from three rows
- * Jobs must not overlap each other's outputs.
+ *   ws       unused (the call needs no scratch; the query returns a token
+ *            256 bytes); may be NULL
+ * Jobs must not overlap each other's outputs.  With W_out == W_in (in place)
+ * the result is the same bits, but rows already pruned by one part of the
+ * launch can be sampled by another when it estimates a matrix's threshold,
+ * which only costs speed.
  * ------------------------------------------------------------------------- */
 typedef struct mosaic_prune_job {
     const void *W_in;

@@ -306,13 +306,24 @@ def mosaic_allocate_sparsity(outlier_counts, numels, cols, n_layers: int, n_proj
     return list(s), list(k), st == ERR_INFEASIBLE
 
 
-def mosaic_prune_unstructured(W_in: torch.Tensor, W_out: torch.Tensor, norms: torch.Tensor, k: int,
-                              mask_out: torch.Tensor | None = None, ws: Workspace | None = None, stream=None) -> None:
-    """Per row, zero the k entries first under (score asc, column asc); optional keep bitmask."""
-    p, rows, cols, ldw = _mat(W_in, "W_in")
+def _out_ptr(W_in: torch.Tensor, W_out: torch.Tensor | None, rows: int, cols: int, ldw: int):
+    """Pointer of the pruned-weights output, or None for mask-only mode."""
+    if W_out is None:
+        return None
     po, r2, c2, ld2 = _mat(W_out, "W_out")
     if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or (rows > 1 and ld2 != ldw):
         raise ValueError("W_out must match W_in in shape, dtype and leading dimension")
+    return po
+
+
+def mosaic_prune_unstructured(W_in: torch.Tensor, W_out: torch.Tensor | None, norms: torch.Tensor, k: int,
+                              mask_out: torch.Tensor | None = None, ws: Workspace | None = None, stream=None) -> None:
+    """Per row, zero the k entries first under (score asc, column asc); optional keep bitmask.
+    W_out None: mask-only mode (mask_out is then the only output)."""
+    p, rows, cols, ldw = _mat(W_in, "W_in")
+    po = _out_ptr(W_in, W_out, rows, cols, ldw)
+    if W_out is None and mask_out is None:
+        raise ValueError("mask-only mode needs mask_out")
     _dev(norms, "norms", torch.float32)
     if norms.numel() != cols:
         raise ValueError("norms must be [cols]")
@@ -332,7 +343,7 @@ class PruneJob(C.Structure):
 
 class PruneBatch:
     """The marshalled job list of mosaic_prune_unstructured_batch for a list of
-    (W_in, W_out, norms, k, mask_out or None).  Checked and laid out once; run() may replace
+    (W_in, W_out or None, norms, k, mask_out or None).  Checked and laid out once; run() may replace
     the per-row prune counts and then only makes the call.  The tensors are kept alive by the object."""
 
     def __init__(self, jobs):
@@ -343,9 +354,11 @@ class PruneBatch:
         dtype = self.jobs[0][0].dtype
         for i, (W_in, W_out, norms, k, mask_out) in enumerate(self.jobs):
             p, rows, cols, ldw = _mat(W_in, "W_in")
-            po, r2, c2, ld2 = _mat(W_out, "W_out")
-            if (r2, c2) != (rows, cols) or W_out.dtype != W_in.dtype or W_in.dtype != dtype or (rows > 1 and ld2 != ldw):
-                raise ValueError("W_out must match W_in in shape, dtype and leading dimension; one dtype per batch")
+            po = _out_ptr(W_in, W_out, rows, cols, ldw)
+            if W_in.dtype != dtype:
+                raise TypeError("one dtype per batch")
+            if W_out is None and mask_out is None:
+                raise ValueError("mask-only mode needs mask_out")
             _dev(norms, "norms", torch.float32)
             if norms.numel() != cols:
                 raise ValueError("norms must be [cols]")

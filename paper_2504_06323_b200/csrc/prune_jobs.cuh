@@ -12,7 +12,6 @@ struct PruneJob {
     uint16_t* W_out;        // or nullptr: only the keep bitmask is written
     const float* norms;
     uint8_t* mask;          // keep bitmask as bytes, or nullptr
-    uint32_t* plan;         // window and thresholds prepared by prune_plan_kernel, or nullptr
     int64_t rows, ldw, row0;
     int k, mask_row_bytes;
 };
@@ -23,9 +22,10 @@ struct PruneJobList {
 };
 constexpr int kBatchJobs = 256;   // jobs per launch of the batched kernels (the list travels as a kernel parameter)
 
-// Warp-per-row kernel (prune_warp.cu): bf16 rows of kWarpMinCols..kWarpMaxCols columns, cols % 8 == 0,
+// Row-group kernel (prune_warp.cu): bf16 rows of kWarpMinCols..kWarpMaxCols columns, cols % 8 == 0,
 // 0 < k < cols for every job.  Enqueues one launch; returns a mosaic_status.
-constexpr int kWarpMinCols = 2048, kWarpMaxCols = 8192;
+constexpr int kWarpMinCols = 2048, kWarpMaxCols = 16384;
+bool prune_warp_takes(int64_t cols);   // true iff a launch shape exists for rows of this length
 int launch_prune_warp(const PruneJobList<1>& jobs, int64_t total_rows, int cols, cudaStream_t st);
 int launch_prune_warp(const PruneJobList<kBatchJobs>& jobs, int64_t total_rows, int cols, cudaStream_t st);
 

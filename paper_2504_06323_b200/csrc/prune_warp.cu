@@ -1,31 +1,37 @@
-// Warp-per-row kernel of mosaic_prune_unstructured[_batch] for bf16 rows of 2048..8192 columns
-// (Section 4.1.3, unstructured projection pruning; weight metric of Eq. 5): per output row, the k
-// entries first under (score ascending, column ascending) become +0, fused with the keep bitmask.
+// Per-row selection kernel of mosaic_prune_unstructured[_batch] for bf16 rows of 2048..16384
+// columns (Section 4.1.3, unstructured projection pruning; weight metric of Eq. 5): per output
+// row, the k entries first under (score ascending, column ascending) become +0, fused with the
+// keep bitmask.
 //
 // One persistent CTA per SM.  A CTA takes a contiguous range of the launch's rows, so it changes
-// matrix (job) only a few times; per job it keeps three tables in shared memory - the norms and,
-// for a window [lo, hi) of score keys that should contain every row's threshold, per column the
-// bf16 magnitude patterns A_lo[j] <= / A_hi[j] >= below / from which a weight's score is surely
-// under lo / at least hi (the score norm_j * |w| is monotone in |w|).  The window is centred on
-// the median of one estimate per warp: the matching quantile of the exact scores of a quarter of
-// one row of the job (rows spread evenly over the matrix), selected in registers.
+// matrix (job) only a few times; per job it keeps two tables in shared memory: the norms and, for
+// a window [lo, hi) of score keys that should contain every row's threshold, per column the bf16
+// magnitude pattern A_lo[j] such that a weight below it scores surely under lo, while a weight
+// from A_lo[j] + D up scores surely at least hi (the score norm_j * |w| is monotone in |w|; D is
+// one depth for the whole job).  The window is centred on the median of one estimate per warp:
+// the matching quantile of the exact scores of a quarter of one row of the job (rows spread
+// evenly over the matrix), selected in registers.
 //
-// Each warp then works on whole rows by itself, with no block barrier on the row path:
-//   1. the row arrives in the warp's shared-memory buffer by cp.async;
+// A row is worked on by a group of G warps (G = 1 for short rows: a warp per row and no barrier at
+// all on the row path; longer rows take 2, 4 or 8 warps so that 16 warps stay resident).  Every
+// warp owns a fixed set of the row's 16-byte vectors from the copy into shared memory to the final
+// store; the warps of a group only meet on the row's histogram:
+//   1. the warp's vectors arrive in the group's row buffer by cp.async;
 //   2. classification, two weights per integer subtract: (w | 0x8000) - A has bit 15 set iff the
-//      magnitude is >= A.  Weights under A_lo are pruned for sure, weights from A_hi up are kept
-//      for sure, the few per cent in between are the row's candidates;
-//   3. the candidates are queued (their columns), get their exact fp32 score key from the row and
-//      the norm table, and go into a 256-bin histogram of the window;
-//   4. a warp scan finds the bin that holds rank k; the keys of that bin are ranked under
-//      (key, column), which is the oracle's total order, so ties need no special case;
-//   5. candidates at or below the threshold are zeroed in the row buffer.  A zeroed weight has
-//      magnitude 0 < A_lo, so the store pass - which masks everything under A_lo - writes both the
-//      sure and the selected zeros and the keep bits from one classification.
-// A row whose threshold falls outside the window, whose candidates overflow the queue, or whose
-// bin holds more than 32 keys, and every row of a job whose window is unusable (non-finite norms,
-// thresholds near zero or overflow) takes slow_row(): a full 4 x 8-bit radix select by the warp on
-// exact keys.  All paths give the oracle's bits.
+//      magnitude is >= A.  Weights under A_lo are pruned for sure, weights from A_lo + D up are
+//      kept for sure, the few per cent in between are the row's candidates;
+//   3. the warp queues its candidates (their columns), forms their exact fp32 score keys from the
+//      row buffer and the norm table, and adds them to the group's 256-bin histogram of the window;
+//   4. (group barrier) every warp finds the bin that holds rank k; the keys of that bin are
+//      collected (group barrier) and ranked under (key, column), which is the oracle's total
+//      order, so ties need no special case;
+//   5. the warp zeroes its candidates at or below the threshold in the row buffer.  A zeroed weight
+//      has magnitude 0 < A_lo, so the store pass - which masks everything under A_lo - writes both
+//      the sure and the selected zeros and the keep bits from one classification.
+// A row whose threshold falls outside the window, whose candidates overflow a queue, or whose bin
+// holds more than 32 keys, and every row of a job whose window is unusable (non-finite norms,
+// norms outside [2^-100, 2^100], thresholds near zero or overflow) takes slow_row(): a radix
+// select by the group on exact (key, column) pairs.  All paths give the oracle's bits.
 #include "prune_jobs.cuh"
 
 namespace mosaic {
@@ -33,52 +39,52 @@ namespace mosaic {
 constexpr int kWMaxWarps = 16;
 constexpr int kWBins = 256;
 constexpr int kWBinList = 32;
+constexpr uint32_t kWOverflow = 0xFFFFFFFFu;   // a warp's "my queue overflowed" in place of its count of sure-below weights
 
-// Shared-memory carve-up for rows of `cols` columns (host and device agree on it).
+// Shared-memory carve-up for rows of `cols` columns worked on by groups of G warps (host and
+// device agree on it).  Groups of several warps alternate between two histograms / bin lists /
+// count slots from row to row, so that a warp may start the next row while another still reads.
 struct WarpLayout {
-    int nvec, qcap, nwords;
-    uint32_t off_alo, off_ahi, off_nrm, off_misc, off_warp0, per_warp;   // bytes
-    uint32_t o_qkey, o_qcol, o_hist, o_mbytes, o_bkey, o_bcol;           // bytes inside a warp's block
+    int nvec, nwords, qcap;   // qcap: candidates one warp may queue
+    uint32_t off_alo, off_nrm, off_misc, off_group0, per_group;                      // bytes
+    uint32_t o_queue, per_queue, o_qcol, o_hist, o_mbytes, o_bkey, o_bcol, o_ctl;   // bytes inside a group's block
 };
-__host__ __device__ inline WarpLayout warp_layout(int cols) {
+__host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
     WarpLayout L;
+    const uint32_t sets = G == 1 ? 1u : 2u;
     L.nvec = cols >> 3;
     L.nwords = (cols + 31) >> 5;
-    L.qcap = ((cols >> 3) + 31) & ~31;                 // candidates a row may have (1/8 of it) before it goes the slow way
+    L.qcap = (((cols >> 3) * 15 / 16 + G - 1) / G + 31) & ~31;   // about an eighth of the warp's share of the row
     uint32_t o = 0;
     L.off_alo = o;   o += (uint32_t)L.nvec * 16u;
-    L.off_ahi = o;   o += (uint32_t)L.nvec * 16u;
     L.off_nrm = o;   o += (uint32_t)cols * 4u;
-    L.off_misc = o;  o += 64u;
-    L.off_warp0 = o;
+    L.off_misc = o;  o += 128u;
+    L.off_group0 = o;
     uint32_t w = (uint32_t)L.nvec * 16u;               // the row
-    L.o_qkey = w;    w += (uint32_t)L.qcap * 4u;
-    L.o_qcol = w;    w += (uint32_t)L.qcap * 2u;
+    L.o_queue = w;                                     // per warp: qcap keys (4 B) then qcap columns (2 B)
+    L.o_qcol = (uint32_t)L.qcap * 4u;
+    L.per_queue = (uint32_t)L.qcap * 6u;
+    w += L.per_queue * (uint32_t)G;
     w = (w + 15u) & ~15u;
-    L.o_hist = w;    w += kWBins * 4u;
+    L.o_hist = w;    w += sets * kWBins * 4u;
     L.o_mbytes = w;  w += ((uint32_t)L.nwords * 4u + 15u) & ~15u;
-    L.o_bkey = w;    w += kWBinList * 4u;
-    L.o_bcol = w;    w += kWBinList * 4u;
-    L.per_warp = (w + 15u) & ~15u;
+    L.o_bkey = w;    w += sets * kWBinList * 4u;
+    L.o_bcol = w;    w += sets * kWBinList * 4u;
+    L.o_ctl = w;     w += G == 1 ? 16u : 256u;         // [p*16 + sub] sure-below counts, [32 + p] bin-list fill
+    L.per_group = (w + 15u) & ~15u;
     return L;
 }
-constexpr uint32_t kWSmemBudget = 227u * 1024u - 1024u;   // dynamic shared memory a CTA may use (static arrays need a little)
-
-// Warps per CTA for rows of `cols` columns: as many as shared memory holds, at most kWMaxWarps.
-static int warps_for(int cols) {
-    const WarpLayout L = warp_layout(cols);
-    if (L.off_warp0 + 3u * L.per_warp > kWSmemBudget) return 0;
-    int w = (int)((kWSmemBudget - L.off_warp0) / L.per_warp);
-    return w > kWMaxWarps ? kWMaxWarps : w;
-}
+constexpr uint32_t kWSmemBudget = 227u * 1024u - 256u;   // dynamic shared memory a CTA may use (static arrays need a little)
 
 __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem)), "l"(gmem)
                  : "memory");
 }
-__device__ __forceinline__ void cp_async_commit_wait() {
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
+// Barrier among the 32*G threads of a row group (G == 1: the warp).  Barrier 0 is the CTA's.
+template <int G>
+__device__ __forceinline__ void group_barrier(int gid) {
+    if (G == 1) __syncwarp();
+    else asm volatile("bar.sync %0, %1;" ::"r"(gid + 1), "r"(32 * G) : "memory");
 }
 
 // With x = word | 0x80008000 (each 16-bit lane = 0x8000 + magnitude) and A two 16-bit thresholds
@@ -90,12 +96,12 @@ __device__ __forceinline__ uint32_t flags8(uint32_t t0, uint32_t t1, uint32_t t2
     const uint32_t b = __byte_perm(t2, t3, 0x7531);   // elements 4, 5, 6, 7
     return (a & 0x80808080u) | ((b >> 1) & 0x40404040u);
 }
-// flags8 word -> byte with bit e = flag of element e.  ((f >> 7) & 0x01010101) holds elements 0..3
-// on bits 0, 8, 16, 24; times 0x01020408 brings them to bits 24..27 in order (no two partial
-// products meet on a bit, so nothing carries).
+// flags8 word -> byte with bit e = flag of element e.  (f & 0x80808080) holds elements 0..3 on bits
+// 7, 15, 23, 31; the high word of its product with 2^25 + 2^18 + 2^11 + 2^4 has them on bits 0..3
+// (no two partial products meet on a bit, so nothing carries).
 __device__ __forceinline__ uint32_t byte_of_flags(uint32_t f) {
-    const uint32_t lo = (((f >> 7) & 0x01010101u) * 0x01020408u) >> 24;
-    const uint32_t hi = (((f >> 6) & 0x01010101u) * 0x01020408u) >> 24;
+    const uint32_t lo = __umulhi(f & 0x80808080u, 0x02040810u) & 0xFu;
+    const uint32_t hi = __umulhi((f << 1) & 0x80808080u, 0x02040810u) & 0xFu;
     return lo | (hi << 4);
 }
 // 0xFFFF over each 16-bit lane of t whose top bit is set (prmt replicates the sign of the selected byte).
@@ -119,13 +125,16 @@ __device__ __forceinline__ uint32_t warp_incl_scan(uint32_t v, int lane) {
 }
 
 // The bin of hist[0..256) that holds rank `rank` (1-based) when `base0` entries come before bin 0.
-// Warp-wide; clears the histogram.  Returns false if no bin holds the rank.
+// Warp-wide; CLEAR leaves the histogram zeroed.  Returns false if no bin holds the rank.
+template <bool CLEAR>
 __device__ __forceinline__ bool warp_find_bin(uint32_t* hist, uint32_t base0, uint32_t rank, int lane, uint32_t* bin,
                                               uint32_t* rank_in_bin, uint32_t* count) {
     uint4* h4 = reinterpret_cast<uint4*>(hist);
     const uint4 a = h4[lane * 2], b = h4[lane * 2 + 1];
-    h4[lane * 2] = make_uint4(0u, 0u, 0u, 0u);
-    h4[lane * 2 + 1] = make_uint4(0u, 0u, 0u, 0u);
+    if (CLEAR) {
+        h4[lane * 2] = make_uint4(0u, 0u, 0u, 0u);
+        h4[lane * 2 + 1] = make_uint4(0u, 0u, 0u, 0u);
+    }
     const uint32_t c[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
     uint32_t sum = 0u;
 #pragma unroll
@@ -150,102 +159,80 @@ __device__ __forceinline__ bool warp_find_bin(uint32_t* hist, uint32_t base0, ui
     *count = __shfl_sync(0xFFFFFFFFu, cc, src);
     return true;
 }
+__device__ __forceinline__ void warp_clear_hist(uint32_t* hist, int lane) {
+    uint4* h4 = reinterpret_cast<uint4*>(hist);
+    h4[lane * 2] = make_uint4(0u, 0u, 0u, 0u);
+    h4[lane * 2 + 1] = make_uint4(0u, 0u, 0u, 0u);
+}
 
-// Exact score key of element e of vector `vec` of the row (sign bit cleared: norms are >= +0 by
-// contract, and a negative one must not index past a histogram).
+// Exact score key of element e of a vector (sign bit cleared: norms are >= +0 by contract, and a
+// negative one must not index past a histogram).
 __device__ __forceinline__ uint32_t exact_key(const uint4& r, const float* nrm8, int e) {
     return __float_as_uint(__fmul_rn(nrm8[e], mag_f32(word_of(r, e >> 1), e & 1))) & 0x7FFFFFFFu;
 }
 
-// Exact k-th smallest key of the row in `row` (1 <= k <= cols) by the warp: 4 x 8-bit radix select
-// from the top.  T = the key, n_eq = keys equal to it, q = how many of those are among the k
-// smallest.  hist must be zero on entry and is zero on exit.
-template <int V>
-__device__ __noinline__ void warp_exact_select(const uint4* row, const float* nrm, int nvec, uint32_t k, uint32_t* hist,
-                                               uint32_t* T, uint32_t* q, uint32_t* n_eq) {
+// The always-exact treatment of one row by its group: radix select (8-bit digits from the top) of
+// the k-th smallest key T, then - if only q of the n_eq keys equal to T are among the k smallest -
+// of the q-th smallest column among those; every entry at or below (T, column) is pruned.  Stores
+// the warp's vectors and leaves their keep bits as bytes in mbytes.  `hist` may hold a failed
+// attempt's counts on entry and is zero on exit.  Called by all warps of the group together.
+template <int V, int G>
+__device__ __noinline__ void slow_row(const uint4* row, const float* nrm, int nvec, uint32_t k, uint32_t* hist, uint8_t* mbytes,
+                                      uint16_t* out_row, int gid, int sub) {
     const int lane = threadIdx.x & 31;
-    uint32_t prefix = 0u, pmask = 0u, rank = k, cnt = 0u;
-#pragma unroll 1
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    const int gl = sub * 32 + lane;
+    group_barrier<G>(gid);
+    if (sub == 0) warp_clear_hist(hist, lane);
+    group_barrier<G>(gid);
+    uint32_t T = 0u, q = 0u, n_eq = 0u, colT = 0xFFFFu;
+    // phase 0: the key, four digits; phase 1: the column among the keys equal to T, two digits
+    for (int phase = 0; phase < 2; ++phase) {
+        uint32_t prefix = 0u, pmask = 0u, rank = phase == 0 ? k : q, cnt = 0u;
+        for (int shift = phase == 0 ? 24 : 8; shift >= 0; shift -= 8) {
 #pragma unroll 2
-        for (int v = 0; v < V; ++v) {
-            const int vec = v * 32 + lane;
-            if (vec < nvec) {
-                const uint4 r = row[vec];
-                const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
-                const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+            for (int v = 0; v < V; ++v) {
+                const int vec = v * 32 * G + gl;
+                if (vec < nvec) {
+                    const uint4 r = row[vec];
+                    const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
+                    const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
 #pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    const uint32_t key = exact_key(r, n8, e);
-                    if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFFu], 1u);
-                }
-            }
-        }
-        __syncwarp();
-        uint32_t bin = 0u, rr = 0u, cc = 0u;
-        warp_find_bin(hist, 0u, rank, lane, &bin, &rr, &cc);   // always found: 1 <= rank <= keys that match the prefix
-        prefix |= bin << shift;
-        pmask |= 0xFFu << shift;
-        rank = rr;
-        cnt = cc;
-        __syncwarp();
-    }
-    *T = prefix;
-    *q = rank;
-    *n_eq = cnt;
-}
-
-// The always-exact treatment of one row by its warp: full select, ties by column, store, keep bits.
-// Leaves the keep bits of the row as bytes in mbytes (one per vector).
-template <int V>
-__device__ __noinline__ void slow_row(uint4* row, const float* nrm, int nvec, uint32_t k, uint32_t* hist, uint8_t* mbytes,
-                                      uint16_t* out_row) {
-    const int lane = threadIdx.x & 31;
-    uint32_t T, q, n_eq;
-    warp_exact_select<V>(row, nrm, nvec, k, hist, &T, &q, &n_eq);
-    // column of the q-th key equal to T in column order (a lane's vectors v*32 + lane ascend with v, then lane)
-    uint32_t colT = 0xFFFFFFFFu;
-    if (q < n_eq) {
-        uint32_t before = 0u;
-        bool found = false;
-#pragma unroll 1
-        for (int v = 0; v < V && !found; ++v) {
-            const int vec = v * 32 + lane;
-            uint32_t eq = 0u;
-            if (vec < nvec) {
-                const uint4 r = row[vec];
-                const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
-                const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) eq |= (exact_key(r, n8, e) == T) ? (1u << e) : 0u;
-            }
-            const uint32_t mine = (uint32_t)__popc(eq);
-            const uint32_t incl = warp_incl_scan(mine, lane);
-            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            if (before + tot >= q) {
-                const uint32_t excl = before + incl - mine;
-                const unsigned m = __ballot_sync(0xFFFFFFFFu, excl < q && q <= excl + mine);
-                const int src = __ffs(m) - 1;
-                uint32_t col = 0u;
-                if (lane == src) {
-                    uint32_t need = q - excl;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        if ((eq >> e) & 1u) {
-                            if (--need == 0u) col = (uint32_t)(vec * 8 + e);
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t key = exact_key(r, n8, e);
+                        if (phase == 0) {
+                            if ((key & pmask) == prefix) atomicAdd(&hist[(key >> shift) & 0xFFu], 1u);
+                        } else {
+                            const uint32_t col = (uint32_t)(vec * 8 + e);
+                            if (key == T && (col & pmask) == prefix) atomicAdd(&hist[(col >> shift) & 0xFFu], 1u);
                         }
+                    }
                 }
-                colT = __shfl_sync(0xFFFFFFFFu, col, src);
-                found = true;
             }
-            before += tot;
+            group_barrier<G>(gid);
+            uint32_t bin = 0u, rr = 0u, cc = 0u;
+            warp_find_bin<false>(hist, 0u, rank, lane, &bin, &rr, &cc);   // always found: 1 <= rank <= matching entries
+            group_barrier<G>(gid);
+            if (sub == 0) warp_clear_hist(hist, lane);
+            group_barrier<G>(gid);
+            prefix |= bin << shift;
+            pmask |= 0xFFu << shift;
+            rank = rr;
+            cnt = cc;
+        }
+        if (phase == 0) {
+            T = prefix;
+            q = rank;
+            n_eq = cnt;
+            if (q == n_eq) break;   // every key equal to T is pruned: colT stays above all columns
+        } else {
+            colT = prefix;
         }
     }
 #pragma unroll 2
     for (int v = 0; v < V; ++v) {
-        const int vec = v * 32 + lane;
+        const int vec = v * 32 * G + gl;
         if (vec < nvec) {
-            uint4 r = row[vec];
+            const uint4 r = row[vec];
             const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
             const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
             uint32_t pruned = 0u;
@@ -266,67 +253,72 @@ __device__ __noinline__ void slow_row(uint4* row, const float* nrm, int nvec, ui
     }
 }
 
-// Thresholds of the window [lo, lo + 2^w) for one vector of 8 columns.  For column j with norm n:
+// Thresholds of the window [lo, hi) for one vector of 8 columns: A_lo per column (packed like the
+// row's words); returns the largest A_hi - A_lo of the vector.  For column j with norm n:
 //   magnitude pattern a <  A_lo  =>  score key < lo;      a >= A_hi  =>  score key >= hi.
 // With x = fl(l / n) (correctly rounded) and g = its top 16 bits (the bf16 pattern at or just
 // below x), patterns <= g-2 are more than a bf16 step (2^-8 relative) below l/n, so their product
 // with n rounds below l; patterns >= g+2 are above it.  A_lo >= 1 always: a zero weight scores +0,
-// under any usable lo.  Norm 0: every finite weight scores 0 (sure below), inf/NaN weights are
-// candidates.  Norms outside [2^-100, 2^100]: every non-zero weight is a candidate.
-__device__ __forceinline__ void thresholds_of_vector(const float* nrm8, float flo, float fhi, uint4* alo, uint4* ahi) {
-    uint32_t al[8], ah[8];
+// under any usable lo.  Norm 0: every finite weight scores 0 (sure below); inf and NaN weights
+// (patterns from 0x7F80) become candidates.  The caller has checked 2^-100 <= n <= 2^100 or n == 0.
+__device__ __forceinline__ uint32_t thresholds_of_vector(const float* nrm8, float flo, float fhi, uint4* alo) {
+    uint32_t al[8], depth = 2u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         const float n = nrm8[e];
         if (n == 0.0f) {
             al[e] = 0x7F80u;
-            ah[e] = 0x7F82u;
-        } else if (!(n >= 0x1p-100f && n <= 0x1p100f)) {
-            al[e] = 1u;
-            ah[e] = 0x8000u;
         } else {
             const uint32_t gl = __float_as_uint(__fdiv_rn(flo, n)) >> 16;
             const uint32_t gh = __float_as_uint(__fdiv_rn(fhi, n)) >> 16;
             al[e] = gl > 3u ? gl - 2u : 1u;
-            ah[e] = gh + 2u < 0x8000u ? gh + 2u : 0x8000u;
+            const uint32_t ah = gh + 2u < 0x8000u ? gh + 2u : 0x8000u;
+            depth = max(depth, ah - al[e]);
         }
     }
     *alo = make_uint4(al[0] | (al[1] << 16), al[2] | (al[3] << 16), al[4] | (al[5] << 16), al[6] | (al[7] << 16));
-    *ahi = make_uint4(ah[0] | (ah[1] << 16), ah[2] | (ah[3] << 16), ah[4] | (ah[5] << 16), ah[6] | (ah[7] << 16));
+    return depth;
 }
 
-// blockDim.x = 32 * warps (warps >= 3); dynamic shared memory = off_warp0 + warps * per_warp of warp_layout(cols).
-// Every job: cols % 8 == 0, kWarpMinCols <= cols <= V * 256, 0 < k < cols.
-// FULL: cols == V * 256, so every vector slot v * 32 + lane is inside the row and no bounds test is needed.
-template <int V, int NJ, bool FULL>
+// blockDim.x = 32 * G * groups; dynamic shared memory = off_group0 + groups * per_group of warp_layout(cols, G).
+// Every job: cols % 8 == 0, cols <= V * 256 * G, 0 < k < cols.  FULL: cols == V * 256 * G, so every
+// vector slot is inside the row and no bounds test is needed.
+template <int V, int G, int NJ, bool FULL>
 __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(const __grid_constant__ PruneJobList<NJ> jobs,
                                                                              int64_t total_rows, int cols) {
     extern __shared__ __align__(16) unsigned char smem[];
-    __shared__ uint16_t flagtab[32];   // bit of a packed candidate word -> column offset (vector within the group of 4) * 256 + element
-    const WarpLayout L = warp_layout(cols);
+    __shared__ uint16_t flagtab[32];   // bit of a packed candidate word -> (vector within its group of 4) * 256 * G + element
+    constexpr int TG = 32 * G;         // threads of a row group
+    constexpr int NW = (V + 3) / 4;    // packed candidate words per thread
+    const WarpLayout L = warp_layout(cols, G);
     const int nvec = L.nvec, nwords = L.nwords;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5, nwarps = blockDim.x >> 5, nthreads = blockDim.x;
+    const int gid = wid / G, sub = wid % G, ngroups = nwarps / G;
+    const int gl = sub * 32 + lane;    // thread within the row group: owns the vectors v * TG + gl
     uint4* alo = reinterpret_cast<uint4*>(smem + L.off_alo);
-    uint4* ahi = reinterpret_cast<uint4*>(smem + L.off_ahi);
     float* nrm = reinterpret_cast<float*>(smem + L.off_nrm);
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates
-    unsigned char* mine = smem + L.off_warp0 + (size_t)wid * L.per_warp;
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates, [16] window depth
+    unsigned char* mine = smem + L.off_group0 + (size_t)gid * L.per_group;
     uint4* row = reinterpret_cast<uint4*>(mine);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(mine);
-    uint32_t* qkey = reinterpret_cast<uint32_t*>(mine + L.o_qkey);
-    uint16_t* qcol = reinterpret_cast<uint16_t*>(mine + L.o_qcol);
-    uint32_t* hist = reinterpret_cast<uint32_t*>(mine + L.o_hist);
+    uint32_t* qkey = reinterpret_cast<uint32_t*>(mine + L.o_queue + (size_t)sub * L.per_queue);
+    uint16_t* qcol = reinterpret_cast<uint16_t*>(mine + L.o_queue + (size_t)sub * L.per_queue + L.o_qcol);
+    uint32_t* hist0 = reinterpret_cast<uint32_t*>(mine + L.o_hist);
     uint8_t* mbytes = mine + L.o_mbytes;
-    uint32_t* bkey = reinterpret_cast<uint32_t*>(mine + L.o_bkey);
-    uint32_t* bcol = reinterpret_cast<uint32_t*>(mine + L.o_bcol);
+    uint32_t* bkey0 = reinterpret_cast<uint32_t*>(mine + L.o_bkey);
+    uint32_t* bcol0 = reinterpret_cast<uint32_t*>(mine + L.o_bcol);
+    uint32_t* ctl = reinterpret_cast<uint32_t*>(mine + L.o_ctl);
 
     if (tid < 32) {
         const int p = tid & 7, s = (7 - p) >> 1;
         const int e = (tid >> 3) + ((p & 1) ? 0 : 4);
-        flagtab[tid] = (uint16_t)(s * 256 + e);
+        flagtab[tid] = (uint16_t)(s * 8 * TG + e);
     }
-    for (int b = lane; b < kWBins; b += 32) hist[b] = 0u;
-    for (int b = lane; b < nwords * 4; b += 32) mbytes[b] = 0u;   // the bytes past the row's last vector stay zero: mask padding
+    if (sub == 0) {
+        for (int b = lane; b < (G == 1 ? 1 : 2) * kWBins; b += 32) hist0[b] = 0u;
+        for (int b = lane; b < nwords * 4; b += 32) mbytes[b] = 0u;   // the bytes past the row's last vector stay zero: mask padding
+        for (int b = lane; b < (G == 1 ? 4 : 64); b += 32) ctl[b] = 0u;
+    }
     __syncthreads();
 
     const int win_bits = cols >= 8192 ? 20 : 21;   // the k-th score of a row scatters like 1/sqrt(cols)
@@ -337,6 +329,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
     const int64_t cta_begin = (int64_t)blockIdx.x * rows_per_cta;
     const int64_t cta_end = cta_begin + rows_per_cta < total_rows ? cta_begin + rows_per_cta : total_rows;
     int j = 0;
+    uint32_t parity = 0u;   // which histogram / bin list / count slots the group's current row uses (G > 1)
     for (int64_t seg = cta_begin; seg < cta_end;) {
         while (seg >= jobs.job[j].row0 + jobs.job[j].rows) ++j;
         const PruneJob& J = jobs.job[j];
@@ -351,14 +344,15 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         for (int c = tid; c < cols; c += nthreads) {
             const float n = __ldg(J.norms + c);
             nrm[c] = n;
-            fin = fin && (n >= 0.0f) && (n <= 3.402823466e38f);
+            fin = fin && (n == 0.0f || (n >= 0x1p-100f && n <= 0x1p100f));   // false for NaN, inf and negative norms too
         }
+        if (tid == 0) misc[16] = 0u;
         bool valid = __syncthreads_and(fin ? 1 : 0) != 0;
-        uint32_t lo = 0u;
+        uint32_t lo = 0u, DD = 0u;
         if (valid) {
             // One estimate per warp: the k-th score of row (rows-1)*wid/(nwarps-1), taken as the matching
-            // quantile of the exact keys of four of each lane's vectors (a quarter of the row), which
-            // the lane keeps in registers through a 4 x 8-bit radix select.
+            // quantile of the exact keys of a quarter of the row (four evenly spaced vectors per lane),
+            // which the lane keeps in registers through a 4 x 8-bit radix select.
             {
                 const int64_t srow = (J.rows - 1) * wid / (nwarps > 1 ? nwarps - 1 : 1);
                 const uint16_t* src = J.W_in + srow * ldw;
@@ -366,9 +360,10 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 uint32_t n_valid = 0u;
 #pragma unroll
                 for (int i = 0; i < 4; ++i) {
-                    const int vec = (i * (V / 4)) * 32 + lane;
+                    const int vec = (i * (V * G / 4)) * 32 + lane;
                     if (FULL || vec < nvec) {
-                        const uint4 r = ld_stream16(src + (int64_t)vec * kVec);   // (in place, another CTA may be writing this row: any value will do for an estimate)
+                        // (in place, another CTA may be writing this row: any value will do for an estimate)
+                        const uint4 r = ld_stream16(src + (int64_t)vec * kVec);
                         const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
                         const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
 #pragma unroll
@@ -376,25 +371,30 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                         n_valid += 8u;
                     } else {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = 0xFFFFFFFFu;   // matches no prefix: in no histogram
+                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = 0xFFFFFFFFu;   // in no histogram
                     }
                 }
                 n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
                 uint32_t rank = (uint32_t)(((uint64_t)uk * n_valid + (uint32_t)cols / 2u) / (uint32_t)cols);
                 rank = rank < 1u ? 1u : (rank > n_valid ? n_valid : rank);
                 uint32_t prefix = 0u, pmask = 0u;
+                for (int turn = 0; turn < G; ++turn) {   // the warps of a group share a histogram: one after the other
+                    if (turn == sub) {
 #pragma unroll 1
-                for (int sh = 24; sh >= 0; sh -= 8) {
+                        for (int sh = 24; sh >= 0; sh -= 8) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if ((key[i] & pmask) == prefix && key[i] != 0xFFFFFFFFu) atomicAdd(&hist[(key[i] >> sh) & 0xFFu], 1u);
-                    __syncwarp();
-                    uint32_t bin = 0u, rr = 0u, cc = 0u;
-                    warp_find_bin(hist, 0u, rank, lane, &bin, &rr, &cc);
-                    prefix |= bin << sh;
-                    pmask |= 0xFFu << sh;
-                    rank = rr;
-                    __syncwarp();
+                            for (int i = 0; i < 32; ++i)
+                                if ((key[i] & pmask) == prefix && key[i] != 0xFFFFFFFFu) atomicAdd(&hist0[(key[i] >> sh) & 0xFFu], 1u);
+                            __syncwarp();
+                            uint32_t bin = 0u, rr = 0u, cc = 0u;
+                            warp_find_bin<true>(hist0, 0u, rank, lane, &bin, &rr, &cc);
+                            prefix |= bin << sh;
+                            pmask |= 0xFFu << sh;
+                            rank = rr;
+                            __syncwarp();
+                        }
+                    }
+                    if (G > 1) group_barrier<G>(gid);
                 }
                 if (lane == 0) misc[wid] = prefix;
             }
@@ -416,65 +416,82 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
             if (valid) {
                 lo = center - half;
                 const float flo = __uint_as_float(lo), fhi = __uint_as_float(lo + width);
+                uint32_t depth = 2u;
                 for (int vec = tid; vec < nvec; vec += nthreads) {
                     const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
                     const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-                    thresholds_of_vector(n8, flo, fhi, &alo[vec], &ahi[vec]);
+                    depth = max(depth, thresholds_of_vector(n8, flo, fhi, &alo[vec]));
                 }
+                depth = __reduce_max_sync(0xFFFFFFFFu, depth);
+                if (lane == 0) atomicMax(&misc[16], depth);
             }
         }
         __syncthreads();
+        if (valid) {
+            // One depth for all columns: A_hi = A_lo + D.  D <= 128 keeps A_lo + D <= 0x8000 for every
+            // column (A_lo <= 0x7F80), which the borrow-free subtraction needs; a window of 2^21 keys is
+            // at most 32 bf16 steps deep, so the bound holds with room to spare for every usable window.
+            const uint32_t depth = misc[16];
+            valid = depth <= 128u;
+            DD = depth | (depth << 16);
+        }
 
-        // ---------------- rows of the segment, one per warp at a time
-        auto fetch = [&](int64_t rr) {   // this warp's copy of global row rr into its buffer (one cp.async group)
+        // ---------------- rows of the segment, one per group at a time
+        auto fetch = [&](int64_t rr) {   // this warp's vectors of global row rr into the group's buffer (one cp.async group)
             const uint16_t* src = J.W_in + (rr - J.row0) * ldw;
 #pragma unroll
             for (int v = 0; v < V; ++v) {
-                const int vec = v * 32 + lane;
+                const int vec = v * TG + gl;
                 if (FULL || vec < nvec) cp_async16(&row[vec], src + (int64_t)vec * kVec);
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         };
-        if (seg + wid < seg_end) fetch(seg + wid);
-        for (int64_t r = seg + wid; r < seg_end; r += nwarps) {
+        if (seg + gid < seg_end) fetch(seg + gid);
+        for (int64_t r = seg + gid; r < seg_end; r += ngroups, parity ^= (G == 1 ? 0u : 1u)) {
             const int64_t lrow = r - J.row0;
             uint16_t* out_row = J.W_out != nullptr ? J.W_out + lrow * ldw : nullptr;
             uint32_t* mask_row = J.mask != nullptr ? reinterpret_cast<uint32_t*>(J.mask + lrow * J.mask_row_bytes) : nullptr;
+            uint32_t* hist = hist0 + parity * kWBins;
+            uint32_t* bkey = bkey0 + parity * kWBinList;
+            uint32_t* bcol = bcol0 + parity * kWBinList;
+            uint32_t* below_of = ctl + parity * 16u;   // [sub]   (G > 1)
+            uint32_t* fill = ctl + 32u + parity;       //         (G > 1)
             asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncwarp();
+            __syncwarp();   // a warp reads only the vectors it copied itself
 
             bool done = false;
             if (valid) {
                 // ---- classification
-                uint32_t candw[(V + 3) / 4];
+                uint32_t candw[NW];
 #pragma unroll
-                for (int w = 0; w < (V + 3) / 4; ++w) candw[w] = 0u;
+                for (int w = 0; w < NW; ++w) candw[w] = 0u;
                 uint32_t below = 0u;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
-                    const int vec = v * 32 + lane;
+                    const int vec = v * TG + gl;
                     if (FULL || vec < nvec) {
-                        const uint4 rr = row[vec], a = alo[vec], h = ahi[vec];
-                        const uint32_t x0 = rr.x | 0x80008000u, x1 = rr.y | 0x80008000u, x2 = rr.z | 0x80008000u,
-                                       x3 = rr.w | 0x80008000u;
-                        const uint32_t keepf = flags8(x0 - a.x, x1 - a.y, x2 - a.z, x3 - a.w);
-                        const uint32_t above = flags8(x0 - h.x, x1 - h.y, x2 - h.z, x3 - h.w);
+                        const uint4 rr = row[vec], a = alo[vec];
+                        const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
+                                       t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
+                        const uint32_t keepf = flags8(t0, t1, t2, t3);
+                        const uint32_t above = flags8(t0 - DD, t1 - DD, t2 - DD, t3 - DD);
                         candw[v >> 2] |= (keepf & ~above) >> (2 * (v & 3));
                         below += 8u - (uint32_t)__popc(keepf);
                     }
                 }
-                // ---- queue the candidates' columns
+                // ---- queue the warp's candidates (their columns)
                 uint32_t cnt = 0u;
 #pragma unroll
-                for (int w = 0; w < (V + 3) / 4; ++w) cnt += (uint32_t)__popc(candw[w]);
+                for (int w = 0; w < NW; ++w) cnt += (uint32_t)__popc(candw[w]);
                 const uint32_t incl = warp_incl_scan(cnt, lane);
                 const uint32_t qn = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                if (qn <= (uint32_t)L.qcap) {
+                const bool fits = qn <= (uint32_t)L.qcap;
+                if (fits) {
                     uint32_t off = incl - cnt;
 #pragma unroll
-                    for (int w = 0; w < (V + 3) / 4; ++w)
+                    for (int w = 0; w < NW; ++w)
                         for (uint32_t c = candw[w]; c != 0u; c &= c - 1u)
-                            qcol[off++] = (uint16_t)(w * 1024 + lane * 8 + flagtab[__ffs(c) - 1]);
+                            qcol[off++] = (uint16_t)(w * 32 * TG + gl * 8 + flagtab[__ffs(c) - 1]);
                     __syncwarp();
                     // ---- exact keys of the candidates, four rounds of 32 at a time
                     for (uint32_t base = lane; base < qn; base += 128u) {
@@ -483,7 +500,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
                             const uint32_t i = base + 32u * g;
-                            col[g] = i < qn ? (uint32_t)qcol[i] : 0u;
+                            col[g] = i < qn ? (uint32_t)qcol[i] : (uint32_t)(gl * 8);   // a spare slot reads a column of its own
                         }
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
@@ -502,81 +519,128 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                             }
                         }
                     }
-                    below = __reduce_add_sync(0xFFFFFFFFu, below);
-                    __syncwarp();
-                    // ---- the bin that holds rank k, then the rank inside it under (key, column)
-                    uint32_t bin = 0u, r_bin = 0u, n_bin = 0u;
-                    const bool hit = warp_find_bin(hist, below, uk, lane, &bin, &r_bin, &n_bin);
-                    if (hit && n_bin <= (uint32_t)kWBinList) {
-                        uint32_t nl = 0u;
-                        for (uint32_t base = 0u; base < qn; base += 32u) {
-                            const uint32_t i = base + lane;
-                            const uint32_t key = i < qn ? qkey[i] : 0u;
-                            const bool in = i < qn && ((key - lo) >> shift) == bin;
-                            const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
-                            if (in) {
-                                const uint32_t pos = nl + (uint32_t)__popc(m & ((1u << lane) - 1u));
-                                bkey[pos] = key;
-                                bcol[pos] = (uint32_t)qcol[i];
-                            }
-                            nl += (uint32_t)__popc(m);
-                        }
-                        __syncwarp();
-                        const bool have = (uint32_t)lane < n_bin;
-                        const uint32_t mk = have ? bkey[lane] : 0xFFFFFFFFu, mc = have ? bcol[lane] : 0xFFFFFFFFu;
-                        uint32_t less = 0u;
-                        for (uint32_t jj = 0u; jj < n_bin; ++jj) {
-                            const uint32_t ok = __shfl_sync(0xFFFFFFFFu, mk, (int)jj), oc = __shfl_sync(0xFFFFFFFFu, mc, (int)jj);
-                            less += (ok < mk || (ok == mk && oc < mc)) ? 1u : 0u;
-                        }
-                        const unsigned sel = __ballot_sync(0xFFFFFFFFu, have && less + 1u == r_bin);
-                        const int src_l = __ffs(sel) - 1;   // exactly one entry holds rank r_bin: the pairs are distinct
-                        const uint32_t T = __shfl_sync(0xFFFFFFFFu, mk, src_l), colT = __shfl_sync(0xFFFFFFFFu, mc, src_l);
-                        // ---- zero the selected candidates in the row buffer
-                        for (uint32_t i = lane; i < qn; i += 32u) {
-                            const uint32_t key = qkey[i], col = (uint32_t)qcol[i];
-                            if (key < T || (key == T && col <= colT)) row16[col] = (uint16_t)0;
-                        }
-                        __syncwarp();
-                        // ---- store: everything under A_lo (the sure ones and the zeroed candidates) becomes +0
+                }
+                below = __reduce_add_sync(0xFFFFFFFFu, below);
+                bool ok = fits;
+                if (G > 1) {   // the group's count of sure-below weights, and whether every warp's queue held
+                    if (lane == 0) below_of[sub] = fits ? below : kWOverflow;
+                    group_barrier<G>(gid);
+                    below = 0u;
 #pragma unroll
-                        for (int v = 0; v < V; ++v) {
-                            const int vec = v * 32 + lane;
-                            if (FULL || vec < nvec) {
-                                const uint4 rr = row[vec], a = alo[vec];
-                                const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
-                                               t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
-                                if (out_row != nullptr)
-                                    st_stream16(out_row + (int64_t)vec * kVec,
-                                                make_uint4(rr.x & lane_mask(t0), rr.y & lane_mask(t1), rr.z & lane_mask(t2),
-                                                           rr.w & lane_mask(t3)));
-                                mbytes[vec] = (uint8_t)byte_of_flags(flags8(t0, t1, t2, t3));
-                            }
-                        }
-                        done = true;
+                    for (int g = 0; g < G; ++g) {
+                        const uint32_t b = below_of[g];
+                        ok = ok && b != kWOverflow;
+                        below += b;
                     }
+                } else {
+                    __syncwarp();
+                }
+                // ---- the bin that holds rank k, then the rank inside it under (key, column)
+                uint32_t bin = 0u, r_bin = 0u, n_bin = 0u;
+                if (ok) ok = warp_find_bin<G == 1>(hist, below, uk, lane, &bin, &r_bin, &n_bin) && n_bin <= (uint32_t)kWBinList;
+                if (ok) {
+                    uint32_t nl = 0u;
+                    for (uint32_t base = 0u; base < qn; base += 32u) {
+                        const uint32_t i = base + lane;
+                        const uint32_t key = i < qn ? qkey[i] : 0u;
+                        const bool in = i < qn && ((key - lo) >> shift) == bin;
+                        const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
+                        if (G > 1 && m != 0u) {   // the group's list is filled by all its warps: take a range of it
+                            uint32_t first = 0u;
+                            if (lane == 0) first = atomicAdd(fill, (uint32_t)__popc(m));
+                            nl = __shfl_sync(0xFFFFFFFFu, first, 0);
+                        }
+                        if (in) {
+                            const uint32_t pos = nl + (uint32_t)__popc(m & ((1u << lane) - 1u));
+                            bkey[pos] = key;
+                            bcol[pos] = (uint32_t)qcol[i];
+                        }
+                        if (G == 1) nl += (uint32_t)__popc(m);
+                    }
+                    group_barrier<G>(gid);
+                    const bool have = (uint32_t)lane < n_bin;
+                    const uint32_t mk = have ? bkey[lane] : 0xFFFFFFFFu, mc = have ? bcol[lane] : 0xFFFFFFFFu;
+                    uint32_t less = 0u;
+                    for (uint32_t jj = 0u; jj < n_bin; ++jj) {
+                        const uint32_t ok2 = __shfl_sync(0xFFFFFFFFu, mk, (int)jj), oc = __shfl_sync(0xFFFFFFFFu, mc, (int)jj);
+                        less += (ok2 < mk || (ok2 == mk && oc < mc)) ? 1u : 0u;
+                    }
+                    const unsigned sel = __ballot_sync(0xFFFFFFFFu, have && less + 1u == r_bin);
+                    const int src_l = __ffs(sel) - 1;   // exactly one entry holds rank r_bin: the pairs are distinct
+                    const uint32_t T = __shfl_sync(0xFFFFFFFFu, mk, src_l), colT = __shfl_sync(0xFFFFFFFFu, mc, src_l);
+                    if (G > 1 && sub == 0) {   // every warp has read this row's histogram: clean for the row after next
+                        warp_clear_hist(hist, lane);
+                        if (lane == 0) *fill = 0u;
+                    }
+                    // ---- zero the warp's selected candidates in the row buffer
+                    for (uint32_t i = lane; i < qn; i += 32u) {
+                        const uint32_t key = qkey[i], col = (uint32_t)qcol[i];
+                        if (key < T || (key == T && col <= colT)) row16[col] = (uint16_t)0;
+                    }
+                    __syncwarp();
+                    // ---- store: everything under A_lo (the sure ones and the zeroed candidates) becomes +0
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        const int vec = v * TG + gl;
+                        if (FULL || vec < nvec) {
+                            const uint4 rr = row[vec], a = alo[vec];
+                            const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
+                                           t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
+                            if (out_row != nullptr)
+                                st_stream16(out_row + (int64_t)vec * kVec,
+                                            make_uint4(rr.x & lane_mask(t0), rr.y & lane_mask(t1), rr.z & lane_mask(t2),
+                                                       rr.w & lane_mask(t3)));
+                            mbytes[vec] = (uint8_t)byte_of_flags(flags8(t0, t1, t2, t3));
+                        }
+                    }
+                    done = true;
                 }
             }
-            if (!done) slow_row<V>(row, nrm, nvec, uk, hist, mbytes, out_row);
-            __syncwarp();   // the row buffer is free, the keep bytes are complete
-            if (r + nwarps < seg_end) fetch(r + nwarps);   // the next row travels while the keep words leave
-            if (mask_row != nullptr)
-                for (int w = lane; w < nwords; w += 32) mask_row[w] = reinterpret_cast<const uint32_t*>(mbytes)[w];
+            if (!done) slow_row<V, G>(row, nrm, nvec, uk, hist, mbytes, out_row, gid, sub);
+            __syncwarp();   // the warp's part of the row buffer is free, its keep bytes are complete
+            if (r + ngroups < seg_end) fetch(r + ngroups);   // the next row travels while the keep words leave
+            if (mask_row != nullptr) {
+                // the warp's vectors v*TG + sub*32 .. +31 are 32 keep bytes = 8 keep words per v
+                for (int idx = lane; idx < V * 8; idx += 32) {
+                    const int w = ((idx >> 3) * TG + sub * 32) / 4 + (idx & 7);
+                    if (w < nwords) mask_row[w] = reinterpret_cast<const uint32_t*>(mbytes)[w];
+                }
+            }
             __syncwarp();
         }
         seg = seg_end;
     }
 }
 
-template <int V, int NJ, bool FULL>
-static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, cudaStream_t st) {
-    const int warps = warps_for(cols);
-    if (warps < 3) return MOSAIC_ERR_INVALID_ARG;
-    const WarpLayout L = warp_layout(cols);
-    const size_t dyn = (size_t)L.off_warp0 + (size_t)warps * L.per_warp;
+// Group size, group count and vectors per thread for rows of `cols` columns: the most resident
+// warps shared memory allows (at most kWMaxWarps), the smaller group on a tie.
+struct WarpShape {
+    int G, groups, V;
+};
+static WarpShape shape_for(int cols) {
+    WarpShape best{0, 0, 0};
+    const int nvec = cols / 8;
+    for (int G = 1; G <= 8; G *= 2) {
+        const int v = (nvec + 32 * G - 1) / (32 * G);
+        const int V = v <= 8 ? 8 : (v <= 10 ? 10 : (v <= 12 ? 12 : (v <= 14 ? 14 : (v <= 16 ? 16 : (v <= 20 ? 20 : 0)))));
+        if (V == 0) continue;
+        const WarpLayout L = warp_layout(cols, G);
+        if (L.off_group0 + L.per_group > kWSmemBudget) continue;
+        int groups = (int)((kWSmemBudget - L.off_group0) / L.per_group);
+        if (groups > kWMaxWarps / G) groups = kWMaxWarps / G;
+        if (groups * G < 3) continue;
+        if (groups * G > best.groups * best.G) best = WarpShape{G, groups, V};
+    }
+    return best;
+}
+
+template <int V, int G, int NJ, bool FULL>
+static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, int groups, cudaStream_t st) {
+    const WarpLayout L = warp_layout(cols, G);
+    const size_t dyn = (size_t)L.off_group0 + (size_t)groups * L.per_group;
     static DeviceCache opted;   // the shared-memory opt-in belongs to one device's copy of the kernel
     const int ok = opted.get([&]() -> int {
-        if (cudaFuncSetAttribute(prune_rows_warp_kernel<V, NJ, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(prune_rows_warp_kernel<V, G, NJ, FULL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kWSmemBudget) != cudaSuccess) {
             (void)cudaGetLastError();
             return -1;
@@ -585,30 +649,47 @@ static int launch_warp_v(const PruneJobList<NJ>& jobs, int64_t total_rows, int c
     });
     if (ok < 0) return MOSAIC_ERR_CUDA;
     int64_t grid = sm_count();
-    const int64_t need = (total_rows + warps - 1) / warps;
+    const int64_t need = (total_rows + groups - 1) / groups;
     if (grid > need) grid = need;
     if (grid < 1) grid = 1;
-    prune_rows_warp_kernel<V, NJ, FULL><<<(unsigned)grid, warps * 32, dyn, st>>>(jobs, total_rows, cols);
+    prune_rows_warp_kernel<V, G, NJ, FULL><<<(unsigned)grid, groups * G * 32, dyn, st>>>(jobs, total_rows, cols);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
 
 template <int NJ>
 static int launch_warp_any(const PruneJobList<NJ>& jobs, int64_t total_rows, int cols, cudaStream_t st) {
-    const int v = (cols / 8 + 31) / 32;   // vectors per lane
-    const bool full = cols % 256 == 0;
-#define MOSAIC_WARP_CASE(V)                                                                       \
-    if (v <= V)                                                                                   \
-        return (full && cols == V * 256) ? launch_warp_v<V, NJ, true>(jobs, total_rows, cols, st) \
-                                         : launch_warp_v<V, NJ, false>(jobs, total_rows, cols, st)
-    MOSAIC_WARP_CASE(8);
-    MOSAIC_WARP_CASE(12);
-    MOSAIC_WARP_CASE(16);
-    MOSAIC_WARP_CASE(20);
-    MOSAIC_WARP_CASE(24);
-    MOSAIC_WARP_CASE(32);
+    const WarpShape s = shape_for(cols);
+    if (s.G == 0) return MOSAIC_ERR_INVALID_ARG;
+    const bool full = cols == s.V * 256 * s.G;
+#define MOSAIC_WARP_CASE(VV, GG)                                                                  \
+    if (s.V == VV && s.G == GG)                                                                   \
+        return full ? launch_warp_v<VV, GG, NJ, true>(jobs, total_rows, cols, s.groups, st)       \
+                    : launch_warp_v<VV, GG, NJ, false>(jobs, total_rows, cols, s.groups, st)
+    MOSAIC_WARP_CASE(8, 1);
+    MOSAIC_WARP_CASE(10, 1);
+    MOSAIC_WARP_CASE(12, 1);
+    MOSAIC_WARP_CASE(14, 1);
+    MOSAIC_WARP_CASE(16, 1);
+    MOSAIC_WARP_CASE(20, 1);
+    MOSAIC_WARP_CASE(8, 2);
+    MOSAIC_WARP_CASE(10, 2);
+    MOSAIC_WARP_CASE(12, 2);
+    MOSAIC_WARP_CASE(14, 2);
+    MOSAIC_WARP_CASE(16, 2);
+    MOSAIC_WARP_CASE(20, 2);
+    MOSAIC_WARP_CASE(8, 4);
+    MOSAIC_WARP_CASE(10, 4);
+    MOSAIC_WARP_CASE(12, 4);
+    MOSAIC_WARP_CASE(14, 4);
+    MOSAIC_WARP_CASE(16, 4);
+    MOSAIC_WARP_CASE(8, 8);
 #undef MOSAIC_WARP_CASE
     return MOSAIC_ERR_INVALID_ARG;
+}
+
+bool prune_warp_takes(int64_t cols) {
+    return cols >= kWarpMinCols && cols <= kWarpMaxCols && cols % 8 == 0 && shape_for((int)cols).G != 0;
 }
 
 int launch_prune_warp(const PruneJobList<1>& jobs, int64_t total_rows, int cols, cudaStream_t st) {

@@ -293,11 +293,12 @@ def test_prune_many_rows_per_cta(dtype, rows, cols):
         _check_prune(W, norms, k, dtype)
 
 
-@pytest.mark.parametrize("cols", [2048, 2056, 4104, 5128, 6152, 8200, 10248, 11264, 11272, 12296, 16384, 16392])
+@pytest.mark.parametrize("cols", [2048, 2056, 2560, 3072, 3584, 4104, 5120, 5128, 6152, 7168, 8192, 8200, 10248, 11264, 11272,
+                                  12296, 13824, 14336, 16384, 16392])
 def test_prune_bf16_every_cta_shape_with_a_ragged_last_vector_slot(cols):
-    # one row length per instantiation of the bf16 kernel (128 ... 512 threads) and just past each limit, so that
-    # some threads own vector slots beyond the end of the row; 16392 columns is beyond the kernel and takes the
-    # general one.  Batched (planned windows) and single (sampled windows) calls.
+    # one row length per shape of the row-group kernel (1, 2, 4 or 8 warps per row; 8 ... 20 vectors per thread) and
+    # just past each limit, so that some threads own vector slots beyond the end of the row; 16392 columns is beyond
+    # the kernel and takes the general one.  Single and batched calls.
     rows = 700
     W = make(rows, cols, "bf16", seed=cols, heavy=(cols % 16 == 0))
     norms = norms_for(cols, cols % 97)
@@ -310,6 +311,29 @@ def test_prune_bf16_every_cta_shape_with_a_ragged_last_vector_slot(cols):
     ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, "bf16")
     assert_bits_equal(host(out), ref_W)
     assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+
+
+@pytest.mark.parametrize("dtype,rows,cols", [("bf16", 300, 4096), ("bf16", 90, 11008), ("bf16", 40, 688), ("f32", 64, 1000),
+                                             ("bf16", 50, 16392)])
+def test_prune_mask_only_mode(dtype, rows, cols):
+    # W_out == NULL: the keep bitmask is the only output, the input stays as it was
+    W = make(rows, cols, dtype, seed=rows + cols, heavy=True)
+    before = W.clone()
+    norms = norms_for(cols, 44)
+    for k in (0, cols // 2, cols - 1):
+        ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, dtype)
+        mask = torch.full((rows, (cols + 31) // 32), -1, dtype=torch.int32, device=DEV)
+        api.mosaic_prune_unstructured(W, None, norms, k, mask)
+        assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+        mask2 = torch.full_like(mask, -1)
+        api.mosaic_prune_unstructured_batch([(W, None, norms, k, mask2)])
+        assert_bits_equal(mask2.cpu().numpy().view(np.uint32), ref_mask)
+        assert torch.equal(W.view(torch.int16 if dtype == "bf16" else torch.int32),
+                           before.view(torch.int16 if dtype == "bf16" else torch.int32))
+    L = api.lib()
+    rc = L.mosaic_prune_unstructured(W.data_ptr(), None, rows, cols, W.stride(0), api.BF16 if dtype == "bf16" else api.F32,
+                                     norms.data_ptr(), 1, None, None, 0, None)
+    assert rc == -2                                     # no output at all: refused
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
