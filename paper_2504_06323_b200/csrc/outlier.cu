@@ -13,6 +13,17 @@
 //            and counts in fp32 against tau rounded toward -inf: for an fp32
 //            score s, (double)s > tau  <=>  s > fl32_down(tau).  It walks the
 //            tiles in reverse, starting on what sweep 1 touched last.
+//
+// bf16 matrices whose rows are whole 16-byte vectors (cols % 8 == 0: every projection of a
+// model) take two leaner kernels with the same partial sums and the same results:
+//   score_sum_bf16_kernel     the sweep above without the ragged-edge handling, 4 loads in flight
+//                             and few enough registers for 32+ resident warps per SM;
+//   outlier_count_bf16_kernel counts without forming a score: for a fixed column the predicate
+//                             fl32(norm_j * |w|) > tau is monotone in the 15 magnitude bits of
+//                             w, so per column there is one bf16 pattern A_j - found exactly, by
+//                             bisection on that very predicate - with  score > tau  <=>  |w| >= A_j,
+//                             and a row is counted two weights per integer subtract:
+//                             (w | 0x8000) - A_j has bit 15 set iff the magnitude is >= A_j.
 #include <atomic>
 #include <memory>
 #include <new>
@@ -36,6 +47,7 @@ struct OutlierJob {
     int64_t rows, cols, ldw;
     int tile0;             // first global tile
     int chunks;            // tiles per row band
+    int ctile0;            // first global tile of the bf16 count sweep (taller tiles)
 };
 template <int NJ>
 struct OutlierJobList {
@@ -46,6 +58,11 @@ struct OutlierJobList {
 
 __host__ __device__ inline int64_t outlier_tiles(int64_t rows, int64_t cols) {
     return ((cols + kOutChunk - 1) / kOutChunk) * ((rows + kOutTileRows - 1) / kOutTileRows);
+}
+
+constexpr int kCntTileRows = 256;   // rows per tile of the bf16 count sweep: the per-column thresholds are found once per tile
+__host__ __device__ inline int64_t outlier_count_tiles(int64_t rows, int64_t cols) {
+    return ((cols + kOutChunk - 1) / kOutChunk) * ((rows + kCntTileRows - 1) / kCntTileRows);
 }
 
 // Tiles [t_begin, t_end) of this CTA: an equal share of the n_tiles, contiguous.
@@ -179,6 +196,164 @@ __global__ void __launch_bounds__(kOutThreads) outlier_count_kernel(const __grid
     if (j_tau >= 0) flush(j_tau);
 }
 
+// ------------------------------------------------------------------------------------------
+// bf16, cols % 8 == 0
+// ------------------------------------------------------------------------------------------
+// The eight scores of one 16-byte vector added to four fp64 accumulators (element e to acc[e & 3]).
+__device__ __forceinline__ void add_scores(const uint4& v, const float (&nrm)[kVec], double (&acc)[4]) {
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16), hi = __uint_as_float(w[i] & 0xFFFF0000u);
+        acc[(2 * i) & 3] += (double)__fmul_rn(nrm[2 * i], fabsf(lo));
+        acc[(2 * i + 1) & 3] += (double)__fmul_rn(nrm[2 * i + 1], fabsf(hi));
+    }
+}
+
+template <int NJ>
+__global__ void __launch_bounds__(kOutThreads, 8) score_sum_bf16_kernel(const __grid_constant__ OutlierJobList<NJ> jobs,
+                                                                        int n_tiles) {
+    __shared__ double red[32];
+    int t_begin, t_end;
+    tile_share(n_tiles, &t_begin, &t_end);
+    int j = 0;
+    for (int tile = t_begin; tile < t_end; ++tile) {
+        while (j + 1 < jobs.n && tile >= jobs.job[j + 1].tile0) ++j;
+        const OutlierJob& J = jobs.job[j];
+        const int local = tile - J.tile0;
+        if (local == 0 && threadIdx.x == 0) *J.count_out = 0ull;   // the count sweep is a later launch
+        const int chunk = local % J.chunks, band = local / J.chunks;
+        const int c0 = chunk * kOutChunk + (int)threadIdx.x * kVec;
+        const int64_t r0 = (int64_t)band * kOutTileRows;
+        const int n_rows = (int)((r0 + kOutTileRows < J.rows ? r0 + kOutTileRows : J.rows) - r0);
+        double acc[4] = {0.0, 0.0, 0.0, 0.0};
+        if (c0 < (int)J.cols) {
+            float nrm[kVec];
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) nrm[e] = __ldg(J.norms + c0 + e);
+            const size_t stride = (size_t)J.ldw * 2u;
+            const char* p = static_cast<const char*>(J.W) + ((size_t)r0 * (size_t)J.ldw + (size_t)c0) * 2u;
+            int r = 0;
+            for (; r + 4 <= n_rows; r += 4, p += 4 * stride) {
+                const uint4 v0 = ld_stream16_ro(p), v1 = ld_stream16_ro(p + stride), v2 = ld_stream16_ro(p + 2 * stride),
+                            v3 = ld_stream16_ro(p + 3 * stride);
+                add_scores(v0, nrm, acc);
+                add_scores(v1, nrm, acc);
+                add_scores(v2, nrm, acc);
+                add_scores(v3, nrm, acc);
+            }
+            for (; r < n_rows; ++r, p += stride) add_scores(ld_stream16_ro(p), nrm, acc);
+        }
+        const double blk = block_sum((acc[0] + acc[1]) + (acc[2] + acc[3]), red);
+        if (threadIdx.x == 0) J.partial[local] = blk;
+    }
+}
+
+// Smallest bf16 magnitude pattern a in [0, 0x7F80] with  fl32(n * value(a)) > tau  (0x8000 if there
+// is none: n = 0, n or tau not a number, tau = +inf).  The predicate is evaluated exactly as the
+// score is defined (one fp32 multiply, compared with tau already rounded toward -inf) and is
+// monotone in a for n >= 0, so bisection finds the exact boundary; it starts from the bracket
+// [g-2, g+2] around the pattern of tau / n, which holds it except in odd corners (subnormals,
+// overflow), where the whole range is searched.
+__device__ __forceinline__ uint32_t outlier_pattern(float n, float tau) {
+    auto above = [&](uint32_t a) -> bool { return __fmul_rn(n, __uint_as_float(a << 16)) > tau; };
+    if (!above(0x7F80u)) return 0x8000u;
+    if (above(0u)) return 0u;
+    uint32_t lo = 0u, hi = 0x7F80u;   // above(lo) false, above(hi) true
+    const uint32_t g = __float_as_uint(__fdiv_rn(tau, n)) >> 16;   // tau >= 0 and n > 0 here
+    if (g >= 2u && g + 2u <= 0x7F80u && !above(g - 2u) && above(g + 2u)) {
+        lo = g - 2u;
+        hi = g + 2u;
+    }
+    while (hi - lo > 1u) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (above(mid)) hi = mid;
+        else lo = mid;
+    }
+    return hi;
+}
+
+// Flags of (magnitude >= threshold) of a vector's eight elements, counted.  See prune_warp.cu for
+// the borrow-free subtraction: t = (w | 0x80008000) - A, thresholds A <= 0x8000 per 16-bit lane.
+__device__ __forceinline__ uint32_t count_at_or_above(const uint4& v, const uint4& A) {
+    const uint32_t t0 = (v.x | 0x80008000u) - A.x, t1 = (v.y | 0x80008000u) - A.y, t2 = (v.z | 0x80008000u) - A.z,
+                   t3 = (v.w | 0x80008000u) - A.w;
+    const uint32_t a = __byte_perm(t0, t1, 0x7531), b = __byte_perm(t2, t3, 0x7531);   // flag = top bit of every byte
+    return (uint32_t)__popc(a & 0x80808080u) + (uint32_t)__popc(b & 0x80808080u);
+}
+
+template <int NJ>
+__global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(const __grid_constant__ OutlierJobList<NJ> jobs,
+                                                                            int n_tiles) {
+    __shared__ double red[32];
+    __shared__ unsigned int cred[32];
+    __shared__ float tau_sh;
+    int t_begin, t_end;
+    tile_share(n_tiles, &t_begin, &t_end);
+    int j = jobs.n - 1, j_tau = -1;
+    float tau = 0.0f;
+    unsigned int cnt = 0;
+    auto flush = [&](int job) {   // add this CTA's count for `job` (block-uniform call)
+        cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+        __syncthreads();
+        if (lane == 0) cred[wid] = cnt;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long tot = 0;
+            for (int i = 0; i < kOutThreads / 32; ++i) tot += cred[i];
+            if (tot) atomicAdd(jobs.job[job].count_out, tot);   // integer: exact in any order
+        }
+        cnt = 0;
+    };
+    for (int t2 = t_begin; t2 < t_end; ++t2) {
+        const int tile = n_tiles - 1 - t2;   // reverse order of the sum sweep
+        while (tile < jobs.job[j].ctile0) --j;
+        const OutlierJob& J = jobs.job[j];
+        if (j != j_tau) {
+            if (j_tau >= 0) flush(j_tau);
+            // this matrix's partials in tile order: thread-strided, then a fixed tree (as in the general kernel)
+            const int nt_j = (int)outlier_tiles(J.rows, J.cols);
+            double s = 0.0;
+            for (int i = threadIdx.x; i < nt_j; i += kOutThreads) s += __ldcg(&J.partial[i]);
+            const double total = block_sum(s, red);
+            if (threadIdx.x == 0) {
+                const double mean = total / (double)(J.rows * J.cols);
+                const double tau_d = (double)jobs.alpha * mean;
+                tau_sh = __double2float_rd(tau_d);
+                const int last = J.ctile0 + (int)outlier_count_tiles(J.rows, J.cols) - 1;
+                if (tile == last && J.sum_out) *J.sum_out = total;   // once: by the CTA that owns the matrix's last tile
+            }
+            __syncthreads();
+            tau = tau_sh;
+            j_tau = j;
+        }
+        const int local = tile - J.ctile0;
+        const int chunk = local % J.chunks, band = local / J.chunks;
+        const int c0 = chunk * kOutChunk + (int)threadIdx.x * kVec;
+        const int64_t r0 = (int64_t)band * kCntTileRows;
+        const int n_rows = (int)((r0 + kCntTileRows < J.rows ? r0 + kCntTileRows : J.rows) - r0);
+        if (c0 < (int)J.cols) {
+            uint32_t A[kVec];
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) A[e] = outlier_pattern(__ldg(J.norms + c0 + e), tau);
+            const uint4 A4 = make_uint4(A[0] | (A[1] << 16), A[2] | (A[3] << 16), A[4] | (A[5] << 16), A[6] | (A[7] << 16));
+            const size_t stride = (size_t)J.ldw * 2u;
+            const char* p = static_cast<const char*>(J.W) + ((size_t)r0 * (size_t)J.ldw + (size_t)c0) * 2u;
+            int r = 0;
+            for (; r + 8 <= n_rows; r += 8, p += 8 * stride) {
+                uint4 v[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) v[u] = ld_stream16_ro(p + u * stride);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) cnt += count_at_or_above(v[u], A4);
+            }
+            for (; r < n_rows; ++r, p += stride) cnt += count_at_or_above(ld_stream16_ro(p), A4);
+        }
+    }
+    if (j_tau >= 0) flush(j_tau);
+}
+
 template <int DT>
 __global__ void score_kernel(const void* __restrict__ W, int64_t rows, int64_t cols, int64_t ldw,
                              const float* __restrict__ norms, float* __restrict__ out) {
@@ -232,36 +407,49 @@ static int validate_outlier(const void* W, int64_t rows, int64_t cols, int64_t l
     return MOSAIC_OK;
 }
 
-template <int NJ>
-static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int dtype, cudaStream_t st) {
-    static DeviceCache blocks_per_sm[2];   // occupancy is a property of one device's copy of the kernels
-    const int bps = blocks_per_sm[dtype == MOSAIC_BF16 ? 1 : 0].get([&]() -> int {
-        int n1 = 0, n2 = 0;
-        cudaError_t e1, e2;
-        if (dtype == MOSAIC_BF16) {
-            e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n1, score_sum_kernel<MOSAIC_BF16, NJ>, kOutThreads, 0);
-            e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, outlier_count_kernel<MOSAIC_BF16, NJ>, kOutThreads, 0);
-        } else {
-            e1 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n1, score_sum_kernel<MOSAIC_F32, NJ>, kOutThreads, 0);
-            e2 = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n2, outlier_count_kernel<MOSAIC_F32, NJ>, kOutThreads, 0);
-        }
-        if (e1 != cudaSuccess || e2 != cudaSuccess) {
+// Resident CTAs per SM of a kernel, looked up once per device.
+template <class K>
+static int cached_occupancy(DeviceCache& cache, K kernel) {
+    return cache.get([&]() -> int {
+        int n = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, kOutThreads, 0) != cudaSuccess || n < 1) {
             (void)cudaGetLastError();
-            n1 = n2 = 4;
+            n = 4;
         }
-        const int n = n1 < n2 ? n1 : n2;
-        return n < 1 ? 1 : n;
+        return n;
     });
-    int64_t grid = (int64_t)sm_count() * bps;
-    if (grid > n_tiles) grid = n_tiles;
-    if (dtype == MOSAIC_BF16) {
-        score_sum_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+}
+
+// `lean`: every job is bf16 with cols % 8 == 0 (n_ctiles = tiles of the bf16 count sweep).
+template <int NJ>
+static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int64_t n_ctiles, int dtype, bool lean,
+                          cudaStream_t st) {
+    static DeviceCache occ[6];   // occupancy is a property of one device's copy of a kernel
+    int64_t g1, g2;
+    if (lean) {
+        g1 = (int64_t)sm_count() * cached_occupancy(occ[0], score_sum_bf16_kernel<NJ>);
+        g2 = (int64_t)sm_count() * cached_occupancy(occ[1], outlier_count_bf16_kernel<NJ>);
+        if (g1 > n_tiles) g1 = n_tiles;
+        if (g2 > n_ctiles) g2 = n_ctiles;
+        score_sum_bf16_kernel<NJ><<<(unsigned)g1, kOutThreads, 0, st>>>(list, (int)n_tiles);
         MOSAIC_LAUNCH_CHECK();
-        outlier_count_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        outlier_count_bf16_kernel<NJ><<<(unsigned)g2, kOutThreads, 0, st>>>(list, (int)n_ctiles);
+    } else if (dtype == MOSAIC_BF16) {
+        g1 = (int64_t)sm_count() * cached_occupancy(occ[2], score_sum_kernel<MOSAIC_BF16, NJ>);
+        g2 = (int64_t)sm_count() * cached_occupancy(occ[3], outlier_count_kernel<MOSAIC_BF16, NJ>);
+        if (g1 > n_tiles) g1 = n_tiles;
+        if (g2 > n_tiles) g2 = n_tiles;
+        score_sum_kernel<MOSAIC_BF16, NJ><<<(unsigned)g1, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        MOSAIC_LAUNCH_CHECK();
+        outlier_count_kernel<MOSAIC_BF16, NJ><<<(unsigned)g2, kOutThreads, 0, st>>>(list, (int)n_tiles);
     } else {
-        score_sum_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        g1 = (int64_t)sm_count() * cached_occupancy(occ[4], score_sum_kernel<MOSAIC_F32, NJ>);
+        g2 = (int64_t)sm_count() * cached_occupancy(occ[5], outlier_count_kernel<MOSAIC_F32, NJ>);
+        if (g1 > n_tiles) g1 = n_tiles;
+        if (g2 > n_tiles) g2 = n_tiles;
+        score_sum_kernel<MOSAIC_F32, NJ><<<(unsigned)g1, kOutThreads, 0, st>>>(list, (int)n_tiles);
         MOSAIC_LAUNCH_CHECK();
-        outlier_count_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, kOutThreads, 0, st>>>(list, (int)n_tiles);
+        outlier_count_kernel<MOSAIC_F32, NJ><<<(unsigned)g2, kOutThreads, 0, st>>>(list, (int)n_tiles);
     }
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
@@ -284,8 +472,9 @@ extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, i
     one.n = 1;
     one.alpha = alpha;
     one.job[0] = OutlierJob{W, norms, reinterpret_cast<unsigned long long*>(outlier_count_out), score_sum_out,
-                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk)};
-    return launch_outlier<1>(one, outlier_tiles(rows, cols), dtype, static_cast<cudaStream_t>(stream));
+                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk), 0};
+    return launch_outlier<1>(one, outlier_tiles(rows, cols), outlier_count_tiles(rows, cols), dtype,
+                             dtype == MOSAIC_BF16 && cols % kVec == 0, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" size_t mosaic_outlier_ratio_batch_workspace_bytes(const mosaic_outlier_job* jobs, int64_t n_jobs) {
@@ -313,23 +502,26 @@ extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_
     if (!list_mem) return MOSAIC_ERR_INVALID_ARG;
     OutlierJobList<kOutBatch>& list = *list_mem;
     char* wsp = static_cast<char*>(ws);
+    bool lean = dtype == MOSAIC_BF16;
+    for (int64_t m = 0; m < n_jobs; ++m) lean = lean && jobs[m].cols % kVec == 0;
     int64_t i = 0;
     while (i < n_jobs) {
         list.n = 0;
         list.alpha = alpha;
-        int64_t tiles = 0;
+        int64_t tiles = 0, ctiles = 0;
         while (i < n_jobs && list.n < kOutBatch) {
             const mosaic_outlier_job& j = jobs[i];
             const int64_t nt = outlier_tiles(j.rows, j.cols);
             if (tiles + nt > 0x3FFFFFFF) break;
             list.job[list.n++] = OutlierJob{j.W, j.norms, reinterpret_cast<unsigned long long*>(j.outlier_count_out),
                                             j.score_sum_out, reinterpret_cast<double*>(wsp), j.rows, j.cols, j.ldw,
-                                            (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk)};
+                                            (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk), (int)ctiles};
             wsp += mosaic_outlier_ratio_workspace_bytes(j.rows, j.cols);
             tiles += nt;
+            ctiles += outlier_count_tiles(j.rows, j.cols);
             ++i;
         }
-        const int rc = launch_outlier<kOutBatch>(list, tiles, dtype, st);
+        const int rc = launch_outlier<kOutBatch>(list, tiles, ctiles, dtype, lean, st);
         if (rc != MOSAIC_OK) return rc;
     }
     return MOSAIC_OK;

@@ -8,9 +8,11 @@
 // a window [lo, hi) of score keys that should contain every row's threshold, per column the bf16
 // magnitude pattern A_lo[j] such that a weight below it scores surely under lo, while a weight
 // from A_lo[j] + D up scores surely at least hi (the score norm_j * |w| is monotone in |w|; D is
-// one depth for the whole job).  The window is centred on the median of one estimate per warp:
+// one depth for the whole job).  Both patterns are exact: they are found by bisection on the very
+// product that defines a score.  The window is centred on the median of one estimate per warp -
 // the matching quantile of the exact scores of a quarter of one row of the job (rows spread
-// evenly over the matrix), selected in registers.
+// evenly over the matrix), selected in registers - and made just wide enough, judged by the same
+// samples, to hold the ranks a row's threshold can scatter over.
 //
 // A row is worked on by a group of G warps (G = 1 for short rows: a warp per row and no barrier at
 // all on the row path; longer rows take 2, 4 or 8 warps so that 16 warps stay resident).  Every
@@ -21,7 +23,8 @@
 //      magnitude is >= A.  Weights under A_lo are pruned for sure, weights from A_lo + D up are
 //      kept for sure, the few per cent in between are the row's candidates;
 //   3. the warp queues its candidates (their columns), forms their exact fp32 score keys from the
-//      row buffer and the norm table, and adds them to the group's 256-bin histogram of the window;
+//      row buffer and the norm table (again whenever it needs them: a queue of columns alone is a
+//      third the size), and adds them to the group's histogram of the window (up to 256 bins);
 //   4. (group barrier) every warp finds the bin that holds rank k; the keys of that bin are
 //      collected (group barrier) and ranked under (key, column), which is the oracle's total
 //      order, so ties need no special case;
@@ -29,9 +32,9 @@
 //      has magnitude 0 < A_lo, so the store pass - which masks everything under A_lo - writes both
 //      the sure and the selected zeros and the keep bits from one classification.
 // A row whose threshold falls outside the window, whose candidates overflow a queue, or whose bin
-// holds more than 32 keys, and every row of a job whose window is unusable (non-finite norms,
-// norms outside [2^-100, 2^100], thresholds near zero or overflow) takes slow_row(): a radix
-// select by the group on exact (key, column) pairs.  All paths give the oracle's bits.
+// holds more than 32 keys, and every row of a job whose window is unusable (norms that are not
+// finite and >= 0, a threshold at zero or at overflow) takes slow_row(): a radix select by the
+// group on exact (key, column) pairs.  All paths give the oracle's bits.
 #include "prune_jobs.cuh"
 
 namespace mosaic {
@@ -54,16 +57,16 @@ __host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
     const uint32_t sets = G == 1 ? 1u : 2u;
     L.nvec = cols >> 3;
     L.nwords = (cols + 31) >> 5;
-    L.qcap = (((cols >> 3) * 15 / 16 + G - 1) / G + 31) & ~31;   // about an eighth of the warp's share of the row
+    L.qcap = (((cols >> 3) * 3 / 2 + G - 1) / G + 31) & ~31;     // 3/16 of the warp's share of the row
     uint32_t o = 0;
     L.off_alo = o;   o += (uint32_t)L.nvec * 16u;
     L.off_nrm = o;   o += (uint32_t)cols * 4u;
-    L.off_misc = o;  o += 128u;
+    L.off_misc = o;  o += 256u;
     L.off_group0 = o;
     uint32_t w = (uint32_t)L.nvec * 16u;               // the row
-    L.o_queue = w;                                     // per warp: qcap keys (4 B) then qcap columns (2 B)
-    L.o_qcol = (uint32_t)L.qcap * 4u;
-    L.per_queue = (uint32_t)L.qcap * 6u;
+    L.o_queue = w;                                     // per warp: the columns of its candidates (2 B each)
+    L.o_qcol = 0u;
+    L.per_queue = (uint32_t)L.qcap * 2u;
     w += L.per_queue * (uint32_t)G;
     w = (w + 15u) & ~15u;
     L.o_hist = w;    w += sets * kWBins * 4u;
@@ -253,28 +256,39 @@ __device__ __noinline__ void slow_row(const uint4* row, const float* nrm, int nv
     }
 }
 
-// Thresholds of the window [lo, hi) for one vector of 8 columns: A_lo per column (packed like the
-// row's words); returns the largest A_hi - A_lo of the vector.  For column j with norm n:
-//   magnitude pattern a <  A_lo  =>  score key < lo;      a >= A_hi  =>  score key >= hi.
-// With x = fl(l / n) (correctly rounded) and g = its top 16 bits (the bf16 pattern at or just
-// below x), patterns <= g-2 are more than a bf16 step (2^-8 relative) below l/n, so their product
-// with n rounds below l; patterns >= g+2 are above it.  A_lo >= 1 always: a zero weight scores +0,
-// under any usable lo.  Norm 0: every finite weight scores 0 (sure below); inf and NaN weights
-// (patterns from 0x7F80) become candidates.  The caller has checked 2^-100 <= n <= 2^100 or n == 0.
-__device__ __forceinline__ uint32_t thresholds_of_vector(const float* nrm8, float flo, float fhi, uint4* alo) {
-    uint32_t al[8], depth = 2u;
+// Smallest bf16 magnitude pattern a in [0, 0x7F80] whose score key with norm n is >= key_t
+// (1 <= key_t <= 0x7F800000; n >= 0 and finite).  The key of pattern a is the bit pattern of the one
+// fp32 product that defines the score, which is monotone in a, so bisection finds the exact
+// boundary:  magnitude < result  <=>  score key < key_t.  It starts from the bracket [g-2, g+2]
+// around the pattern of t / n, which holds the boundary except in odd corners (subnormal or
+// overflowing quotients), where the whole range is searched.  n = 0: every finite weight scores 0,
+// the result is 0x7F80 (inf and NaN weights score NaN, the largest key).
+__device__ __forceinline__ uint32_t pattern_at_key(float n, uint32_t key_t) {
+    auto at_or_above = [&](uint32_t a) -> bool {
+        return (__float_as_uint(__fmul_rn(n, __uint_as_float(a << 16))) & 0x7FFFFFFFu) >= key_t;
+    };
+    uint32_t lo = 0u, hi = 0x7F80u;   // at_or_above(0) is false (key 0 < key_t); at_or_above(0x7F80) is true (inf or NaN)
+    const uint32_t g = __float_as_uint(__fdiv_rn(__uint_as_float(key_t), n)) >> 16;
+    if (g >= 2u && g + 2u <= 0x7F80u && !at_or_above(g - 2u) && at_or_above(g + 2u)) {
+        lo = g - 2u;
+        hi = g + 2u;
+    }
+    while (hi - lo > 1u) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (at_or_above(mid)) hi = mid;
+        else lo = mid;
+    }
+    return hi;
+}
+
+// A_lo of one vector of 8 columns for the window [lo, hi) of keys (packed like the row's words);
+// returns the largest A_hi - A_lo of the vector.
+__device__ __forceinline__ uint32_t thresholds_of_vector(const float* nrm8, uint32_t lo, uint32_t hi, uint4* alo) {
+    uint32_t al[8], depth = 0u;
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
-        const float n = nrm8[e];
-        if (n == 0.0f) {
-            al[e] = 0x7F80u;
-        } else {
-            const uint32_t gl = __float_as_uint(__fdiv_rn(flo, n)) >> 16;
-            const uint32_t gh = __float_as_uint(__fdiv_rn(fhi, n)) >> 16;
-            al[e] = gl > 3u ? gl - 2u : 1u;
-            const uint32_t ah = gh + 2u < 0x8000u ? gh + 2u : 0x8000u;
-            depth = max(depth, ah - al[e]);
-        }
+        al[e] = pattern_at_key(nrm8[e], lo);
+        depth = max(depth, pattern_at_key(nrm8[e], hi) - al[e]);
     }
     *alo = make_uint4(al[0] | (al[1] << 16), al[2] | (al[3] << 16), al[4] | (al[5] << 16), al[6] | (al[7] << 16));
     return depth;
@@ -297,12 +311,12 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
     const int gl = sub * 32 + lane;    // thread within the row group: owns the vectors v * TG + gl
     uint4* alo = reinterpret_cast<uint4*>(smem + L.off_alo);
     float* nrm = reinterpret_cast<float*>(smem + L.off_nrm);
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates, [16] window depth
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates, [16] window depth,
+                                                                       // [17] samples taken, [32..63] samples by distance from the centre
     unsigned char* mine = smem + L.off_group0 + (size_t)gid * L.per_group;
     uint4* row = reinterpret_cast<uint4*>(mine);
     uint16_t* row16 = reinterpret_cast<uint16_t*>(mine);
-    uint32_t* qkey = reinterpret_cast<uint32_t*>(mine + L.o_queue + (size_t)sub * L.per_queue);
-    uint16_t* qcol = reinterpret_cast<uint16_t*>(mine + L.o_queue + (size_t)sub * L.per_queue + L.o_qcol);
+    uint16_t* qcol = reinterpret_cast<uint16_t*>(mine + L.o_queue + (size_t)sub * L.per_queue);
     uint32_t* hist0 = reinterpret_cast<uint32_t*>(mine + L.o_hist);
     uint8_t* mbytes = mine + L.o_mbytes;
     uint32_t* bkey0 = reinterpret_cast<uint32_t*>(mine + L.o_bkey);
@@ -320,10 +334,6 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         for (int b = lane; b < (G == 1 ? 4 : 64); b += 32) ctl[b] = 0u;
     }
     __syncthreads();
-
-    const int win_bits = cols >= 8192 ? 20 : 21;   // the k-th score of a row scatters like 1/sqrt(cols)
-    const int shift = win_bits - 8;
-    const uint32_t width = 1u << win_bits;
 
     const int64_t rows_per_cta = (total_rows + gridDim.x - 1) / gridDim.x;
     const int64_t cta_begin = (int64_t)blockIdx.x * rows_per_cta;
@@ -344,37 +354,38 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         for (int c = tid; c < cols; c += nthreads) {
             const float n = __ldg(J.norms + c);
             nrm[c] = n;
-            fin = fin && (n == 0.0f || (n >= 0x1p-100f && n <= 0x1p100f));   // false for NaN, inf and negative norms too
+            fin = fin && n >= 0.0f && n <= 3.402823466e38f;   // false for NaN, inf and negative norms
         }
-        if (tid == 0) misc[16] = 0u;
+        if (tid < 64) misc[tid] = 0u;
         bool valid = __syncthreads_and(fin ? 1 : 0) != 0;
-        uint32_t lo = 0u, DD = 0u;
+        uint32_t lo = 0u, width = 0u, DD = 0u;
+        int shift = 0;
         if (valid) {
             // One estimate per warp: the k-th score of row (rows-1)*wid/(nwarps-1), taken as the matching
             // quantile of the exact keys of a quarter of the row (four evenly spaced vectors per lane),
             // which the lane keeps in registers through a 4 x 8-bit radix select.
-            {
-                const int64_t srow = (J.rows - 1) * wid / (nwarps > 1 ? nwarps - 1 : 1);
-                const uint16_t* src = J.W_in + srow * ldw;
-                uint32_t key[32];
-                uint32_t n_valid = 0u;
+            const int64_t srow = (J.rows - 1) * wid / (nwarps > 1 ? nwarps - 1 : 1);
+            const uint16_t* src = J.W_in + srow * ldw;
+            uint32_t key[32];
+            uint32_t n_valid = 0u;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int vec = (i * (V * G / 4)) * 32 + lane;
-                    if (FULL || vec < nvec) {
-                        // (in place, another CTA may be writing this row: any value will do for an estimate)
-                        const uint4 r = ld_stream16(src + (int64_t)vec * kVec);
-                        const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
-                        const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
+            for (int i = 0; i < 4; ++i) {
+                const int vec = (i * (V * G / 4)) * 32 + lane;
+                if (FULL || vec < nvec) {
+                    // (in place, another CTA may be writing this row: any value will do for an estimate)
+                    const uint4 r = ld_stream16(src + (int64_t)vec * kVec);
+                    const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
+                    const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = exact_key(r, n8, e);
-                        n_valid += 8u;
-                    } else {
+                    for (int e = 0; e < 8; ++e) key[i * 8 + e] = exact_key(r, n8, e);
+                    n_valid += 8u;
+                } else {
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) key[i * 8 + e] = 0xFFFFFFFFu;   // in no histogram
-                    }
+                    for (int e = 0; e < 8; ++e) key[i * 8 + e] = 0xFFFFFFFFu;   // in no histogram
                 }
-                n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
+            }
+            n_valid = __reduce_add_sync(0xFFFFFFFFu, n_valid);
+            {
                 uint32_t rank = (uint32_t)(((uint64_t)uk * n_valid + (uint32_t)cols / 2u) / (uint32_t)cols);
                 rank = rank < 1u ? 1u : (rank > n_valid ? n_valid : rank);
                 uint32_t prefix = 0u, pmask = 0u;
@@ -396,7 +407,10 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                     }
                     if (G > 1) group_barrier<G>(gid);
                 }
-                if (lane == 0) misc[wid] = prefix;
+                if (lane == 0) {
+                    misc[wid] = prefix;
+                    atomicAdd(&misc[17], n_valid);
+                }
             }
             __syncthreads();
             // median of the estimates (every thread ranks them the same way: by value, then by warp)
@@ -410,17 +424,56 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 }
                 if (less == nwarps / 2) center = va;
             }
-            const uint32_t half = width >> 1;
-            // refused where scores could be subnormal (lo < 2^24) or the window could reach inf
-            valid = center >= (1u << 24) + half && center - half <= 0x7F7FFFFFu - width;
+            // How wide must the window be?  A row's threshold scatters over about +-3.25 sigma ranks around the
+            // typical one, sigma^2 = k (1 - k/cols), and the centre itself is only an estimate (allow cols/64
+            // ranks).  The samples tell how many keys lie how far from the centre: misc[32 + b] counts those
+            // whose distance has bit length b, i.e. lies in [2^(b-1), 2^b).
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (key[i] != 0xFFFFFFFFu) {
+                    const uint32_t dist = key[i] > center ? key[i] - center : center - key[i];
+                    atomicAdd(&misc[32 + (32 - __clz(dist))], 1u);   // dist < 2^31: bit length 0..31
+                }
+            __syncthreads();
+            {
+                const double p = (double)uk / (double)cols;
+                const double want_row = 6.5 * sqrt((double)cols * p * (1.0 - p)) + (double)cols / 64.0 + 16.0;
+                const uint32_t n_samples = misc[17];
+                const double want = want_row * (double)n_samples / (double)cols;   // ... among the samples
+                // smallest half-width h with  #{distance < h} >= want, interpolated inside the bit-length class
+                double below = 0.0, half_w = 0.0;
+                bool found = false;
+                for (int b = 0; b < 32 && !found; ++b) {
+                    const double c = (double)misc[32 + b];
+                    if (below + c >= want) {
+                        const double base = b == 0 ? 0.0 : ldexp(1.0, b - 1), span = b == 0 ? 1.0 : ldexp(1.0, b - 1);
+                        half_w = base + span * (c > 0.0 ? (want - below) / c : 1.0);
+                        found = true;
+                    }
+                    below += c;
+                }
+                if (!found) half_w = 2147483648.0;
+                double w_d = 2.0 * half_w;
+                if (w_d < 4096.0) w_d = 4096.0;
+                valid = w_d <= 8388608.0;   // a window of more than an octave of keys is no window
+                if (valid) {
+                    uint32_t w_u = (uint32_t)w_d;
+                    shift = 32 - __clz(w_u) - 8;                                  // at most 256 bins of 2^shift keys
+                    shift = shift < 0 ? 0 : shift;
+                    const uint32_t nb = (w_u + (1u << shift) - 1u) >> shift;     // 128 < nb <= 256
+                    width = nb << shift;
+                    const uint32_t half = width >> 1;
+                    // the window must start above key 0 (a zero weight has to be below it) and end at or below +inf
+                    valid = center > half && center - half <= 0x7F800000u - width;
+                    lo = center - half;
+                }
+            }
             if (valid) {
-                lo = center - half;
-                const float flo = __uint_as_float(lo), fhi = __uint_as_float(lo + width);
-                uint32_t depth = 2u;
+                uint32_t depth = 0u;
                 for (int vec = tid; vec < nvec; vec += nthreads) {
                     const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
                     const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-                    depth = max(depth, thresholds_of_vector(n8, flo, fhi, &alo[vec]));
+                    depth = max(depth, thresholds_of_vector(n8, lo, lo + width, &alo[vec]));
                 }
                 depth = __reduce_max_sync(0xFFFFFFFFu, depth);
                 if (lane == 0) atomicMax(&misc[16], depth);
@@ -429,8 +482,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         __syncthreads();
         if (valid) {
             // One depth for all columns: A_hi = A_lo + D.  D <= 128 keeps A_lo + D <= 0x8000 for every
-            // column (A_lo <= 0x7F80), which the borrow-free subtraction needs; a window of 2^21 keys is
-            // at most 32 bf16 steps deep, so the bound holds with room to spare for every usable window.
+            // column (A_lo <= 0x7F80), which the borrow-free subtraction needs.
             const uint32_t depth = misc[16];
             valid = depth <= 128u;
             DD = depth | (depth << 16);
@@ -512,7 +564,6 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                             const uint32_t i = base + 32u * g;
                             if (i < qn) {
                                 const uint32_t key = __float_as_uint(__fmul_rn(n[g], __uint_as_float(a[g])));
-                                qkey[i] = key;
                                 const uint32_t d = key - lo;   // key < lo wraps to >= 2^31 (key, lo < 2^31)
                                 if (d < width) atomicAdd(&hist[d >> shift], 1u);
                                 else below += d >> 31;
@@ -542,7 +593,9 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                     uint32_t nl = 0u;
                     for (uint32_t base = 0u; base < qn; base += 32u) {
                         const uint32_t i = base + lane;
-                        const uint32_t key = i < qn ? qkey[i] : 0u;
+                        const uint32_t col = i < qn ? (uint32_t)qcol[i] : (uint32_t)(gl * 8);
+                        const uint32_t key =
+                            __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
                         const bool in = i < qn && ((key - lo) >> shift) == bin;
                         const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
                         if (G > 1 && m != 0u) {   // the group's list is filled by all its warps: take a range of it
@@ -553,7 +606,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                         if (in) {
                             const uint32_t pos = nl + (uint32_t)__popc(m & ((1u << lane) - 1u));
                             bkey[pos] = key;
-                            bcol[pos] = (uint32_t)qcol[i];
+                            bcol[pos] = col;
                         }
                         if (G == 1) nl += (uint32_t)__popc(m);
                     }
@@ -574,7 +627,9 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                     }
                     // ---- zero the warp's selected candidates in the row buffer
                     for (uint32_t i = lane; i < qn; i += 32u) {
-                        const uint32_t key = qkey[i], col = (uint32_t)qcol[i];
+                        const uint32_t col = (uint32_t)qcol[i];
+                        const uint32_t key =
+                            __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
                         if (key < T || (key == T && col <= colT)) row16[col] = (uint16_t)0;
                     }
                     __syncwarp();
