@@ -300,6 +300,67 @@ int mosaic_rank_units(const float *scores, int64_t n_units, int64_t keep, int32_
  * ------------------------------------------------------------------------- */
 int mosaic_sum_unit_scores(float *dst, const float *src, int64_t n_units, void *stream);
 
+/* ---------------------------------------------------------------------------
+ * Batched forms of the structured steps (Section 4.1.3 structured; Section 2.3):
+ * the same arithmetic as steps 1-3 of mosaic_prune_structured_compact, bit for
+ * bit, for a HOST list of matrices in one launch per step - a model has N*M
+ * projections (Section 3.1) and each is only microseconds of work.  Every
+ * pointer inside a descriptor is a device pointer; the lists are read during
+ * the call only.  Coupled projections (Fig. "composite": nodes between
+ * projections are pruned as a group) are handled by the caller: score all
+ * matrices, add the scores of the coupled units, rank once, compact each matrix
+ * with the shared keep list.
+ * ------------------------------------------------------------------------- */
+
+/* Step 1, unit scores.  row_scores_out [rows/row_group] and col_scores_out
+ * [cols/col_group] are fp32 outputs (overwritten); either may be NULL.
+ * norms == NULL means norm = 1.  ws: device scratch, 256-byte aligned, >= the
+ * query for the same list. */
+typedef struct mosaic_unit_score_job {
+    const void *W;
+    int64_t rows, cols, ldw;
+    const float *norms;
+    int64_t row_group, col_group;
+    float *row_scores_out;
+    float *col_scores_out;
+} mosaic_unit_score_job;
+size_t mosaic_unit_scores_batch_workspace_bytes(const mosaic_unit_score_job *jobs, int64_t n_jobs);
+int mosaic_unit_scores_batch(const mosaic_unit_score_job *jobs, int64_t n_jobs, int dtype, void *ws,
+                             size_t ws_bytes, void *stream);
+
+/* dst[u] = fl32(a[u] + b[u]), u < n, for every item: the running total of the
+ * scores of coupled units.  dst may be a or b exactly; the items of one call
+ * must not write what another item reads. */
+typedef struct mosaic_add_job {
+    float *dst;
+    const float *a;
+    const float *b;
+    int64_t n;
+} mosaic_add_job;
+int mosaic_add_unit_scores_batch(const mosaic_add_job *jobs, int64_t n_jobs, void *stream);
+
+/* Step 2, mosaic_rank_units for a list of score arrays. */
+typedef struct mosaic_rank_job {
+    const float *scores;
+    int64_t n_units, keep;
+    int32_t *keep_out;
+} mosaic_rank_job;
+int mosaic_rank_units_batch(const mosaic_rank_job *jobs, int64_t n_jobs, void *stream);
+
+/* Step 3, dense compaction with given keep lists (ascending unit indices; an
+ * out-of-range index is clamped).  W_out is dense
+ * [row_units_keep*row_group, col_units_keep*col_group] and must not overlap W_in. */
+typedef struct mosaic_compact_job {
+    const void *W_in;
+    int64_t rows, cols, ldw;
+    const int32_t *row_keep_units;
+    int64_t row_units_keep, row_group;
+    const int32_t *col_keep_units;
+    int64_t col_units_keep, col_group;
+    void *W_out;
+} mosaic_compact_job;
+int mosaic_compact_batch(const mosaic_compact_job *jobs, int64_t n_jobs, int dtype, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -37,6 +37,8 @@ SYMBOLS = (
     "mosaic_prune_unstructured_batch_workspace_bytes", "mosaic_prune_unstructured_batch",
     "mosaic_prune_structured_compact_workspace_bytes", "mosaic_prune_structured_compact",
     "mosaic_rank_units", "mosaic_sum_unit_scores",
+    "mosaic_unit_scores_batch_workspace_bytes", "mosaic_unit_scores_batch", "mosaic_add_unit_scores_batch",
+    "mosaic_rank_units_batch", "mosaic_compact_batch",
 )
 
 
@@ -101,6 +103,16 @@ def lib() -> C.CDLL:
         L.mosaic_rank_units.argtypes = [vp, i64, i64, vp, vp]
         L.mosaic_sum_unit_scores.restype = ci
         L.mosaic_sum_unit_scores.argtypes = [vp, vp, i64, vp]
+        L.mosaic_unit_scores_batch_workspace_bytes.restype = sz
+        L.mosaic_unit_scores_batch_workspace_bytes.argtypes = [vp, i64]
+        L.mosaic_unit_scores_batch.restype = ci
+        L.mosaic_unit_scores_batch.argtypes = [vp, i64, ci, vp, sz, vp]
+        L.mosaic_add_unit_scores_batch.restype = ci
+        L.mosaic_add_unit_scores_batch.argtypes = [vp, i64, vp]
+        L.mosaic_rank_units_batch.restype = ci
+        L.mosaic_rank_units_batch.argtypes = [vp, i64, vp]
+        L.mosaic_compact_batch.restype = ci
+        L.mosaic_compact_batch.argtypes = [vp, i64, ci, vp]
         _lib = L
     return _lib
 
@@ -439,3 +451,157 @@ def mosaic_sum_unit_scores(dst: torch.Tensor, src: torch.Tensor, stream=None) ->
         raise ValueError("dst and src must be contiguous and of equal length")
     _check(lib().mosaic_sum_unit_scores(dst.data_ptr(), src.data_ptr(), dst.numel(), _stream(stream)),
            "mosaic_sum_unit_scores")
+
+
+# --------------------------------------------------------------------------- batched structured steps
+class UnitScoreJob(C.Structure):
+    """mosaic_unit_score_job of include/mosaic.h."""
+    _fields_ = [("W", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ldw", C.c_int64), ("norms", C.c_void_p),
+                ("row_group", C.c_int64), ("col_group", C.c_int64), ("row_scores_out", C.c_void_p),
+                ("col_scores_out", C.c_void_p)]
+
+
+class AddJob(C.Structure):
+    """mosaic_add_job of include/mosaic.h."""
+    _fields_ = [("dst", C.c_void_p), ("a", C.c_void_p), ("b", C.c_void_p), ("n", C.c_int64)]
+
+
+class RankJob(C.Structure):
+    """mosaic_rank_job of include/mosaic.h."""
+    _fields_ = [("scores", C.c_void_p), ("n_units", C.c_int64), ("keep", C.c_int64), ("keep_out", C.c_void_p)]
+
+
+class CompactJob(C.Structure):
+    """mosaic_compact_job of include/mosaic.h."""
+    _fields_ = [("W_in", C.c_void_p), ("rows", C.c_int64), ("cols", C.c_int64), ("ldw", C.c_int64),
+                ("row_keep_units", C.c_void_p), ("row_units_keep", C.c_int64), ("row_group", C.c_int64),
+                ("col_keep_units", C.c_void_p), ("col_units_keep", C.c_int64), ("col_group", C.c_int64),
+                ("W_out", C.c_void_p)]
+
+
+class UnitScoreBatch:
+    """The marshalled job list of mosaic_unit_scores_batch for a list of (W, norms or None, row_group,
+    col_group, row_scores_out or None, col_scores_out or None).  Checked and laid out once; run() only
+    makes the call.  The tensors are kept alive by the object."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (UnitScoreJob * len(self.jobs))()
+        dtype = self.jobs[0][0].dtype
+        for i, (W, norms, rg, cg, rs, cs) in enumerate(self.jobs):
+            p, rows, cols, ldw = _mat(W, "W")
+            if W.dtype != dtype:
+                raise TypeError("one dtype per batch")
+            if norms is not None:
+                _dev(norms, "norms", torch.float32)
+            for t, nm, n in ((rs, "row_scores_out", rows // rg), (cs, "col_scores_out", cols // cg)):
+                if t is not None:
+                    _dev(t, nm, torch.float32)
+                    if t.numel() < n or not t.is_contiguous():
+                        raise ValueError(f"{nm} must be contiguous with one entry per unit")
+            self.arr[i] = UnitScoreJob(p, rows, cols, ldw, _ptr(norms), int(rg), int(cg), _ptr(rs), _ptr(cs))
+        self.code = _dtype_code(self.jobs[0][0])
+        self.device = self.jobs[0][0].device
+        self.ws_bytes = lib().mosaic_unit_scores_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs))
+
+    def run(self, ws: Workspace | None = None, stream=None) -> None:
+        wp, wn = _ws(ws, self.device).get(self.ws_bytes)
+        _check(lib().mosaic_unit_scores_batch(C.addressof(self.arr), len(self.jobs), self.code, wp, wn, _stream(stream)),
+               "mosaic_unit_scores_batch")
+
+
+class AddBatch:
+    """The marshalled list of mosaic_add_unit_scores_batch for (dst, a, b) fp32 vectors of equal length."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (AddJob * len(self.jobs))()
+        for i, (dst, a, b) in enumerate(self.jobs):
+            for t, nm in ((dst, "dst"), (a, "a"), (b, "b")):
+                _dev(t, nm, torch.float32)
+                if not t.is_contiguous() or t.numel() != dst.numel():
+                    raise ValueError("dst, a and b must be contiguous and of equal length")
+            self.arr[i] = AddJob(dst.data_ptr(), a.data_ptr(), b.data_ptr(), dst.numel())
+
+    def run(self, stream=None) -> None:
+        _check(lib().mosaic_add_unit_scores_batch(C.addressof(self.arr), len(self.jobs), _stream(stream)),
+               "mosaic_add_unit_scores_batch")
+
+
+class RankBatch:
+    """The marshalled list of mosaic_rank_units_batch for (scores, keep, keep_out)."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (RankJob * len(self.jobs))()
+        for i, (scores, keep, keep_out) in enumerate(self.jobs):
+            _dev(scores, "scores", torch.float32)
+            _dev(keep_out, "keep_out", torch.int32)
+            if keep_out.numel() < keep or not scores.is_contiguous():
+                raise ValueError("keep_out too short or scores not contiguous")
+            self.arr[i] = RankJob(scores.data_ptr(), scores.numel(), int(keep), keep_out.data_ptr())
+
+    def run(self, stream=None) -> None:
+        _check(lib().mosaic_rank_units_batch(C.addressof(self.arr), len(self.jobs), _stream(stream)), "mosaic_rank_units_batch")
+
+
+class CompactBatch:
+    """The marshalled list of mosaic_compact_batch for (W_in, row_keep_units, row_units_keep, row_group,
+    col_keep_units, col_units_keep, col_group, W_out)."""
+
+    def __init__(self, jobs):
+        self.jobs = list(jobs)
+        if not self.jobs:
+            raise ValueError("empty batch")
+        self.arr = (CompactJob * len(self.jobs))()
+        dtype = self.jobs[0][0].dtype
+        for i, (W_in, rk, n_rk, rg, ck, n_ck, cg, W_out) in enumerate(self.jobs):
+            p, rows, cols, ldw = _mat(W_in, "W_in")
+            if W_in.dtype != dtype:
+                raise TypeError("one dtype per batch")
+            _dev(rk, "row_keep_units", torch.int32)
+            _dev(ck, "col_keep_units", torch.int32)
+            _dev(W_out, "W_out", W_in.dtype)
+            if rk.numel() < n_rk or ck.numel() < n_ck:
+                raise ValueError("keep list shorter than the number of kept units")
+            if not W_out.is_contiguous() or W_out.numel() < n_rk * rg * n_ck * cg:
+                raise ValueError("W_out must be contiguous and hold the compacted matrix")
+            self.arr[i] = CompactJob(p, rows, cols, ldw, rk.data_ptr(), int(n_rk), int(rg), ck.data_ptr(), int(n_ck), int(cg),
+                                     W_out.data_ptr())
+        self.code = _dtype_code(self.jobs[0][0])
+
+    def run(self, stream=None) -> None:
+        _check(lib().mosaic_compact_batch(C.addressof(self.arr), len(self.jobs), self.code, _stream(stream)),
+               "mosaic_compact_batch")
+
+
+def mosaic_unit_scores_batch(jobs, ws: Workspace | None = None, stream=None) -> None:
+    """Unit scores of a list of (W, norms or None, row_group, col_group, row_scores_out or None,
+    col_scores_out or None) in two launches."""
+    if jobs:
+        UnitScoreBatch(jobs).run(ws, stream)
+
+
+def mosaic_add_unit_scores_batch(jobs, stream=None) -> None:
+    """dst[u] = fl32(a[u] + b[u]) for a list of (dst, a, b): fp32 vectors of equal length."""
+    if jobs:
+        AddBatch(jobs).run(stream)
+
+
+def mosaic_rank_units_batch(jobs, stream=None) -> None:
+    """mosaic_rank_units for a list of (scores, keep, keep_out) in one launch."""
+    if jobs:
+        RankBatch(jobs).run(stream)
+
+
+def mosaic_compact_batch(jobs, stream=None) -> None:
+    """Dense compaction of a list of (W_in, row_keep_units, row_units_keep, row_group, col_keep_units,
+    col_units_keep, col_group, W_out) in one launch."""
+    if jobs:
+        CompactBatch(jobs).run(stream)

@@ -1,144 +1,216 @@
-// mosaic_prune_structured_compact / mosaic_rank_units: structured projection
-// pruning (Section 4.1.3; Section 2.3) - unit scores, exact ranking of units,
-// dense compaction.
+// Structured projection pruning (Section 4.1.3: remove the lowest-magnitude heads and channels;
+// Section 2.3: structured pruning leaves smaller dense matrices): unit scores, exact ranking of
+// units, dense compaction - as single calls and as batched calls that take a host list of
+// matrices and do each step for all of them in one launch (a model has N*M projections; one
+// launch chain per projection is bound by launch latency and by the host).
 //
-//   scores : one sweep over W in tiles of 256 columns x 256 rows.  A lane owns 8
-//            adjacent columns: it adds every score to its column accumulators
-//            and to the row's partial sum (fp64); a row's partial over a chunk
-//            is combined by a fixed butterfly, the chunks of a row in chunk
-//            order, the warps' and the bands' column partials in index order.  One fp64 sum per unit over its rows / columns in
-//            index order follows, rounded once to fp32.
-//   rank   : one CTA per dimension; 4 x 8-bit radix select on the fp32 score
-//            bits finds the threshold key and tie quota; an ordered block scan
-//            then emits the ascending keep list (ties: lowest index removed
-//            first).
-//   compact: one CTA per output row: the source row is staged in shared memory
-//            with coalesced 16-byte loads, every thread then gathers 8 output
-//            elements from it through the kept-column list and stores 16 bytes.
+//   scores : one sweep over W in tiles of 512 columns x 256 rows.  A warp covers the tile's 512
+//            columns (a lane owns two vectors of 8 adjacent columns) and takes every fourth row:
+//            every score goes to the lane's column accumulators and to the row's partial sum
+//            (fp64); a row's partial over the tile is combined by a fixed butterfly, the tiles of
+//            a row in column order, the warps' and the row bands' column partials in index order.
+//            One fp64 sum per unit over its rows / columns in index order follows, rounded once
+//            to fp32.  Nothing depends on the launch shape.
+//   rank   : one CTA per list of units; 4 x 8-bit radix select on the fp32 score bits finds the
+//            threshold key and tie quota; an ordered block scan then emits the ascending keep
+//            list (ties: lowest index removed first).
+//   compact: CTAs walk the output rows of all matrices.  Kept columns that come in whole 16-byte
+//            vectors (every column kept, or column units of a multiple of 8 columns) are copied
+//            vector by vector straight from global memory; otherwise the source row is staged in
+//            shared memory and gathered through the kept-column list.
+#include <memory>
+#include <new>
+
 #include "common.cuh"
 
 namespace mosaic {
 
 constexpr int kRankThreads = 1024;
-
-constexpr int kSTileCols = 256;    // columns per tile: one warp row of 32 lanes x 8 columns
+constexpr int kSTileCols = 512;    // columns per tile: a warp row of 32 lanes x 2 vectors of 8 columns
 constexpr int kSTileRows = 256;    // rows per tile, dealt round-robin to the CTA's warps
 constexpr int kSThreads = 128;
 constexpr int kSWarps = kSThreads / 32;
+constexpr int kStructBatch = 128;  // matrices per launch (the list travels as a kernel parameter)
 
-struct StructWs {  // carve-up of the caller's workspace
-    double* row_partial;  // [chunks, rows]
-    double* col_partial;  // [bands, cols]
-    float* scores;        // [n_ru + n_cu]
-    int chunks, bands;
-    size_t bytes;
+struct ScoreJob {
+    const void* W;
+    const float* norms;    // or nullptr: norm = 1
+    double* row_partial;   // [chunks, rows]
+    double* col_partial;   // [bands, cols]
+    float* row_out;        // [rows / row_group] or nullptr
+    float* col_out;        // [cols / col_group] or nullptr
+    int64_t rows, cols, ldw, row_group, col_group;
+    int64_t unit0;         // first global unit (row units, then column units)
+    int tile0, chunks, bands, accumulate;
+};
+template <int NJ>
+struct ScoreJobList {
+    int n;
+    ScoreJob job[NJ];
+};
+struct RankJob {
+    const float* scores;
+    int32_t* keep_out;
+    int64_t n_units, keep;
+};
+template <int NJ>
+struct RankJobList {
+    int n;
+    RankJob job[NJ];
+};
+struct AddJob {
+    float* dst;
+    const float* a;
+    const float* b;
+    int64_t n, item0;
+};
+template <int NJ>
+struct AddJobList {
+    int n;
+    AddJob job[NJ];
+};
+struct CompactJob {
+    const void* W_in;
+    void* W_out;
+    const int32_t* row_keep;
+    const int32_t* col_keep;
+    int64_t cols, ldw, n_ru, row_group, n_cu, col_group, out_rows, out_cols, out_row0;
+};
+template <int NJ>
+struct CompactJobList {
+    int n;
+    CompactJob job[NJ];
 };
 
-static StructWs struct_ws(void* base, int64_t rows, int64_t cols) {
-    StructWs w;
-    char* p = static_cast<char*>(base);
-    size_t off = 0;
-    w.chunks = (int)((cols + kSTileCols - 1) / kSTileCols);
-    w.bands = (int)((rows + kSTileRows - 1) / kSTileRows);
-    w.row_partial = reinterpret_cast<double*>(p + off);
-    off += align_up(sizeof(double) * (size_t)w.chunks * (size_t)rows, 256);
-    w.col_partial = reinterpret_cast<double*>(p + off);
-    off += align_up(sizeof(double) * (size_t)w.bands * (size_t)cols, 256);
-    w.scores = reinterpret_cast<float*>(p + off);
-    off += align_up(sizeof(float) * (size_t)(rows + cols), 256);
-    w.bytes = off;
-    return w;
+static void score_shape(int64_t rows, int64_t cols, int* chunks, int* bands) {
+    *chunks = (int)((cols + kSTileCols - 1) / kSTileCols);
+    *bands = (int)((rows + kSTileRows - 1) / kSTileRows);
+}
+// Scratch of one matrix: row partials [chunks, rows], column partials [bands, cols], 256-byte aligned.
+static size_t score_ws_bytes(int64_t rows, int64_t cols) {
+    int chunks, bands;
+    score_shape(rows, cols, &chunks, &bands);
+    return align_up(sizeof(double) * (size_t)chunks * (size_t)rows, 256) + align_up(sizeof(double) * (size_t)bands * (size_t)cols, 256);
 }
 
-// One tile per CTA (blockIdx.x = column chunk of 256, blockIdx.y = row band of 256).  Every warp
-// covers the chunk's 256 columns (a lane owns 8 adjacent ones) and takes every fourth row of the
-// band: the row's partial sum over the chunk is one butterfly away, and the lane's column
-// accumulators are combined over the four warps in warp order at the end.  All sums in fp64.
-template <int DT>
-__global__ void __launch_bounds__(kSThreads) unit_partial_kernel(const void* __restrict__ W, int64_t rows, int64_t cols,
-                                                                  int64_t ldw, const float* __restrict__ norms,
-                                                                  double* __restrict__ row_partial,
-                                                                  double* __restrict__ col_partial) {
+// Index of the job whose [first, next first) range holds x: first(i) is ascending.
+template <class F>
+__device__ __forceinline__ int find_job(int n, int64_t x, F first) {
+    int lo = 0, hi = n - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (first(mid) <= x) lo = mid;
+        else hi = mid - 1;
+    }
+    return lo;
+}
+
+// One tile per CTA.  All sums in fp64.
+template <int DT, int NJ>
+__global__ void __launch_bounds__(kSThreads) unit_partial_kernel(const __grid_constant__ ScoreJobList<NJ> jobs) {
     __shared__ double cp[kSWarps][kSTileCols + 2];
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    const int64_t c0 = (int64_t)blockIdx.x * kSTileCols + lane * kVec;
-    const int64_t r0 = (int64_t)blockIdx.y * kSTileRows;
+    const int tile = blockIdx.x;
+    const ScoreJob& J = jobs.job[find_job(jobs.n, tile, [&](int i) { return (int64_t)jobs.job[i].tile0; })];
+    const int local = tile - J.tile0;
+    const int chunk = local % J.chunks, band = local / J.chunks;
+    const int64_t rows = J.rows, cols = J.cols, ldw = J.ldw;
+    const int64_t c0 = (int64_t)chunk * kSTileCols + lane * kVec, c1 = c0 + 32 * kVec;
+    const int64_t r0 = (int64_t)band * kSTileRows;
     const int64_t r1 = (r0 + kSTileRows < rows) ? r0 + kSTileRows : rows;
-    float nrm[kVec];
-    double acc[kVec];
+    float nrm[2][kVec];
+    double acc[2][kVec];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) {
-        acc[e] = 0.0;
-        nrm[e] = (c0 + e < cols) ? (norms ? norms[c0 + e] : 1.0f) : 0.0f;
+        acc[0][e] = acc[1][e] = 0.0;
+        nrm[0][e] = (c0 + e < cols) ? (J.norms ? J.norms[c0 + e] : 1.0f) : 0.0f;
+        nrm[1][e] = (c1 + e < cols) ? (J.norms ? J.norms[c1 + e] : 1.0f) : 0.0f;
     }
-    constexpr int U = 4;   // rows in flight per warp
+    constexpr int U = 2;   // rows in flight per warp
     for (int64_t r = r0 + wid; r < r1; r += U * kSWarps) {
-        Raw8<DT> v[U];
+        Raw8<DT> v[U][2];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t rr = r + u * kSWarps;
-            if (rr < r1 && c0 < cols) load_vec<DT, true>(v[u], W, rr * ldw, c0, cols);
-            else v[u].clear();
+            if (rr < r1 && c0 < cols) load_vec<DT, true>(v[u][0], J.W, rr * ldw, c0, cols);
+            else v[u][0].clear();
+            if (rr < r1 && c1 < cols) load_vec<DT, true>(v[u][1], J.W, rr * ldw, c1, cols);
+            else v[u][1].clear();
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const int64_t rr = r + u * kSWarps;
             double p = 0.0;
 #pragma unroll
-            for (int e = 0; e < kVec; ++e) {
-                const double s = (double)__fmul_rn(nrm[e], v[u].abs_f32(e));
-                acc[e] += s;
-                p += s;
-            }
+            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) {
+                    const double s = (double)__fmul_rn(nrm[h][e], v[u][h].abs_f32(e));
+                    acc[h][e] += s;
+                    p += s;
+                }
             p = warp_sum(p);
-            if (lane == 0 && rr < r1) row_partial[(int64_t)blockIdx.x * rows + rr] = p;
+            if (lane == 0 && rr < r1) J.row_partial[(int64_t)chunk * rows + rr] = p;
         }
     }
 #pragma unroll
-    for (int e = 0; e < kVec; ++e) cp[wid][lane * kVec + e] = acc[e];
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) cp[wid][h * 256 + lane * kVec + e] = acc[h][e];
     __syncthreads();
     for (int i = threadIdx.x; i < kSTileCols; i += kSThreads) {
-        const int64_t c = (int64_t)blockIdx.x * kSTileCols + i;
+        const int64_t c = (int64_t)chunk * kSTileCols + i;
         if (c < cols) {
             double s = 0.0;
 #pragma unroll
             for (int w = 0; w < kSWarps; ++w) s += cp[w][i];
-            col_partial[(int64_t)blockIdx.y * cols + c] = s;
+            J.col_partial[(int64_t)band * cols + c] = s;
         }
     }
 }
 
-// Unit score = fp64 sum over the unit's rows (chunk partials in chunk order) or columns (band
-// partials in band order), in index order, rounded once to fp32.
-__global__ void unit_score_kernel(const double* __restrict__ row_partial, int chunks, int64_t rows, int64_t n_ru,
-                                  int64_t row_group, const double* __restrict__ col_partial, int bands, int64_t cols,
-                                  int64_t n_cu, int64_t col_group, float* __restrict__ out, int accumulate) {
-    const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (u >= n_ru + n_cu) return;
+// Unit score = fp64 sum over the unit's rows (tile partials in column order) or columns (band
+// partials in band order), in index order, rounded once to fp32.  One thread per unit of the list.
+template <int NJ>
+__global__ void unit_score_kernel(const __grid_constant__ ScoreJobList<NJ> jobs, int64_t total_units) {
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total_units) return;
+    const ScoreJob& J = jobs.job[find_job(jobs.n, g, [&](int i) { return jobs.job[i].unit0; })];
+    const int64_t u = g - J.unit0, n_ru = J.rows / J.row_group;
     double s = 0.0;
+    float* out;
     if (u < n_ru) {
-        for (int64_t i = u * row_group; i < (u + 1) * row_group; ++i) {
+        if (J.row_out == nullptr) return;
+        for (int64_t i = u * J.row_group; i < (u + 1) * J.row_group; ++i) {
             double rs = 0.0;
 #pragma unroll 8
-            for (int p = 0; p < chunks; ++p) rs += row_partial[(int64_t)p * rows + i];
+            for (int p = 0; p < J.chunks; ++p) rs += J.row_partial[(int64_t)p * J.rows + i];
             s += rs;
         }
+        out = J.row_out + u;
     } else {
+        if (J.col_out == nullptr) return;
         const int64_t v = u - n_ru;
-        for (int64_t c = v * col_group; c < (v + 1) * col_group; ++c) {
+        for (int64_t c = v * J.col_group; c < (v + 1) * J.col_group; ++c) {
             double cs = 0.0;
 #pragma unroll 16
-            for (int p = 0; p < bands; ++p) cs += col_partial[(int64_t)p * cols + c];   // loads batched, adds in order
+            for (int p = 0; p < J.bands; ++p) cs += J.col_partial[(int64_t)p * J.cols + c];   // loads batched, adds in order
             s += cs;
         }
+        out = J.col_out + v;
     }
     const float f = (float)s;
-    out[u] = accumulate ? __fadd_rn(out[u], f) : f;
+    *out = J.accumulate ? __fadd_rn(*out, f) : f;
 }
 
-__global__ void sum_scores_kernel(float* __restrict__ dst, const float* __restrict__ src, int64_t n) {
-    const int64_t u = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (u < n) dst[u] = __fadd_rn(dst[u], src[u]);
+// dst[u] = fl32(a[u] + b[u]) for every item of the list (items must not write what another reads).
+template <int NJ>
+__global__ void add_scores_kernel(const __grid_constant__ AddJobList<NJ> jobs, int64_t total) {
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total) return;
+    const AddJob& J = jobs.job[find_job(jobs.n, g, [&](int i) { return jobs.job[i].item0; })];
+    const int64_t u = g - J.item0;
+    J.dst[u] = __fadd_rn(J.a[u], J.b[u]);
 }
 
 __device__ __forceinline__ uint32_t unit_key(float s) { return (s != s) ? 0xFFFFFFFFu : __float_as_uint(s); }
@@ -147,11 +219,11 @@ __device__ __forceinline__ uint32_t unit_key(float s) { return (s != s) ? 0xFFFF
 __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, int64_t keep, int32_t* __restrict__ keep_out) {
     __shared__ uint32_t hist[256];
     __shared__ uint32_t warp_tot[2][32];
-    __shared__ uint32_t sel_bin, sel_rank, sel_cnt;
+    __shared__ uint32_t sel_bin, sel_rank;
     const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const int64_t remove = n - keep;
     uint32_t T = 0u;
-    int64_t q = 0, n_eq = 0;  // q of the n_eq units with key == T are removed
+    int64_t q = 0;   // q of the units with key == T are removed
     if (remove > 0) {
         uint32_t prefix = 0u, pmask = 0u;
         int64_t rank = remove;
@@ -173,8 +245,8 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
                 uint32_t incl = sum;
 #pragma unroll
                 for (int o = 1; o < 32; o <<= 1) {
-                    const uint32_t n = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (lane >= o) incl += n;
+                    const uint32_t nn = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += nn;
                 }
                 int64_t cum = (int64_t)(incl - sum);
                 if (cum < rank && rank <= cum + (int64_t)sum) {
@@ -183,7 +255,6 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
                         if (cum < rank && rank <= cum + (int64_t)c[i]) {
                             sel_bin = (uint32_t)(lane * 8 + i);
                             sel_rank = (uint32_t)(rank - cum);
-                            sel_cnt = c[i];
                         }
                         cum += c[i];
                     }
@@ -193,7 +264,6 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
             prefix |= sel_bin << shift;
             pmask |= 0xFFu << shift;
             rank = sel_rank;
-            n_eq = sel_cnt;
             __syncthreads();
         }
         T = prefix;
@@ -208,8 +278,7 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
             key = unit_key(scores[u]);
             is_eq = (remove > 0 && key == T) ? 1u : 0u;
         }
-        // scan of the tie indicator
-        uint32_t incl = is_eq;
+        uint32_t incl = is_eq;   // scan of the tie indicator
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t v = __shfl_up_sync(0xFFFFFFFFu, incl, o);
@@ -251,97 +320,344 @@ __device__ void rank_units_block(const float* __restrict__ scores, int64_t n, in
         kept_before += k_total;
         __syncthreads();
     }
-    (void)n_eq;
 }
 
-// blockIdx.x == 0 ranks the row units, 1 the column units (either may be skipped).
-__global__ void __launch_bounds__(kRankThreads) rank_kernel(const float* row_scores, int64_t n_ru, int64_t row_keep,
-                                                             int32_t* row_out, const float* col_scores, int64_t n_cu,
-                                                             int64_t col_keep, int32_t* col_out) {
-    if (blockIdx.x == 0) {
-        if (row_out) rank_units_block(row_scores, n_ru, row_keep, row_out);
-    } else {
-        if (col_out) rank_units_block(col_scores, n_cu, col_keep, col_out);
-    }
+// One CTA per list.
+template <int NJ>
+__global__ void __launch_bounds__(kRankThreads) rank_kernel(const __grid_constant__ RankJobList<NJ> jobs) {
+    const RankJob& J = jobs.job[blockIdx.x];
+    if (J.keep_out != nullptr && J.keep > 0) rank_units_block(J.scores, J.n_units, J.keep, J.keep_out);
 }
 
-// Dense gather.  grid.x = output rows.  The source row is staged in shared memory (dynamic,
-// cols elements) with 16-byte loads; threads then walk output vectors of 8 elements.
-template <int DT>
-__global__ void __launch_bounds__(256) compact_kernel(const void* __restrict__ W, int64_t cols, int64_t ldw,
-                                                       const int32_t* __restrict__ row_keep, int64_t n_ru, int64_t row_group,
-                                                       const int32_t* __restrict__ col_keep, int64_t n_cu, int64_t col_group,
-                                                       int64_t out_cols, void* __restrict__ out) {
+__device__ __forceinline__ int64_t clamp_unit(int64_t u, int64_t n) { return u < 0 ? 0 : (u >= n ? n - 1 : u); }
+
+// Dense gather.  CTAs walk the output rows of all jobs (grid-stride).  Dynamic shared memory: one
+// source row of the widest job that needs staging (0 if none does).
+template <int DT, int NJ>
+__global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ CompactJobList<NJ> jobs, int64_t total_out_rows) {
     extern __shared__ __align__(16) unsigned char srow[];
     constexpr int esz = (DT == MOSAIC_F32) ? 4 : 2;
-    const int64_t a = blockIdx.x;
-    int64_t ru = row_keep[a / row_group];
-    ru = ru < 0 ? 0 : (ru >= n_ru ? n_ru - 1 : ru);
-    const int64_t src_row = ru * row_group + a % row_group;
-    const int64_t in_vec = (cols + kVec - 1) / kVec;
-    for (int64_t v = threadIdx.x; v < in_vec; v += blockDim.x) {
-        Raw8<DT> r;
-        load_vec<DT, true>(r, W, src_row * ldw, v * kVec, cols);
-        uint4* dst = reinterpret_cast<uint4*>(srow + v * kVec * esz);
-        dst[0] = make_uint4(r.w[0], r.w[1], r.w[2], r.w[3]);
-        if (DT == MOSAIC_F32) dst[1] = make_uint4(r.w[4 % (Raw8<DT>::kBytes / 4)], r.w[5 % (Raw8<DT>::kBytes / 4)],
-                                                  r.w[6 % (Raw8<DT>::kBytes / 4)], r.w[7 % (Raw8<DT>::kBytes / 4)]);
-    }
-    __syncthreads();
-    const int64_t nvec = (out_cols + kVec - 1) / kVec;
-    const bool vec_ok = (out_cols % kVec) == 0;   // every output row then starts 16-byte aligned
-    for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
-        Raw8<DT> r;
-        r.clear();
-        const int64_t b0 = v * kVec;
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) {
-            const int64_t b = b0 + e;
-            if (b < out_cols) {
-                int64_t cu = (col_group == 1) ? (int64_t)col_keep[b] : (int64_t)col_keep[b / col_group];
-                cu = cu < 0 ? 0 : (cu >= n_cu ? n_cu - 1 : cu);
-                const int64_t j = (col_group == 1) ? cu : cu * col_group + b % col_group;
-                r.set_scalar(e, srow, j);
+    for (int64_t g = blockIdx.x; g < total_out_rows; g += gridDim.x) {
+        const CompactJob& J = jobs.job[find_job(jobs.n, g, [&](int i) { return jobs.job[i].out_row0; })];
+        const int64_t a = g - J.out_row0;
+        const int64_t src_row = clamp_unit(J.row_keep[a / J.row_group], J.n_ru) * J.row_group + a % J.row_group;
+        const int64_t cols = J.cols, out_cols = J.out_cols, col_group = J.col_group;
+        const char* src = static_cast<const char*>(J.W_in) + (size_t)src_row * (size_t)J.ldw * esz;
+        char* dst = static_cast<char*>(J.W_out) + (size_t)a * (size_t)out_cols * esz;
+        const bool vec_units = (col_group % kVec) == 0 || (J.out_cols == cols && col_group == 1);   // (block-uniform)
+        if (vec_units) {
+            // every output vector of 8 elements is 8 adjacent source columns inside one kept unit
+            // (all columns kept: the keep list is 0, 1, 2, ... and the row is copied as it is)
+            const int64_t nvec = out_cols / kVec;
+            const bool dst_aligned = (out_cols % kVec) == 0;   // else only a whole-row copy with a ragged width gets here
+            if (dst_aligned) {
+                for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
+                    const int64_t b0 = v * kVec;
+                    const int64_t j0 = (col_group == 1) ? b0 : clamp_unit(J.col_keep[b0 / col_group], J.n_cu) * col_group + b0 % col_group;
+                    Raw8<DT> r;
+                    r.template load<true>(src + j0 * esz);
+                    r.store(dst + b0 * esz);
+                }
+            } else {
+                for (int64_t b = threadIdx.x; b < out_cols; b += blockDim.x) {
+                    Raw8<DT> r;
+                    r.set_scalar(0, src, b);
+                    r.put_scalar(0, dst, b);
+                }
             }
+            continue;
         }
-        if (vec_ok) {
-            r.store((char*)out + (a * out_cols + b0) * esz);
-        } else {
+        __syncthreads();   // the previous row's gather is done with the staging buffer
+        const int64_t in_vec = (cols + kVec - 1) / kVec;
+        for (int64_t v = threadIdx.x; v < in_vec; v += blockDim.x) {
+            Raw8<DT> r;
+            load_vec<DT, true>(r, src, 0, v * kVec, cols);
+            uint4* d = reinterpret_cast<uint4*>(srow + v * kVec * esz);
+            d[0] = make_uint4(r.w[0], r.w[1], r.w[2], r.w[3]);
+            if (DT == MOSAIC_F32) d[1] = make_uint4(r.w[4 % (Raw8<DT>::kBytes / 4)], r.w[5 % (Raw8<DT>::kBytes / 4)],
+                                                    r.w[6 % (Raw8<DT>::kBytes / 4)], r.w[7 % (Raw8<DT>::kBytes / 4)]);
+        }
+        __syncthreads();
+        // The output matrix is dense, so its rows follow one another in memory: this row's elements
+        // [head, head + 8*body) start on a 16-byte boundary whatever out_cols is and go out as whole
+        // vectors; the up to 7 elements before and after them are stored one by one.
+        const int n_out = (int)out_cols, ng = (int)col_group;
+        const int head_full = (int)((kVec - (a * out_cols) % kVec) % kVec);
+        const int head = head_full < n_out ? head_full : n_out;
+        const int body = (n_out - head) / kVec;
+        auto source_col = [&](int b) -> int {   // column of the staged row that output column b takes
+            const int64_t cu = clamp_unit((ng == 1) ? (int64_t)J.col_keep[b] : (int64_t)J.col_keep[b / ng], J.n_cu);
+            return (ng == 1) ? (int)cu : (int)cu * ng + b % ng;
+        };
+        for (int v = threadIdx.x; v < body; v += blockDim.x) {
+            Raw8<DT> r;
+            const int b0 = head + v * kVec;
+            if (ng == 1) {
+                int j[kVec];
 #pragma unroll
-            for (int e = 0; e < kVec; ++e)
-                if (b0 + e < out_cols) r.put_scalar(e, out, a * out_cols + b0 + e);
+                for (int e = 0; e < kVec; ++e) j[e] = (int)clamp_unit((int64_t)J.col_keep[b0 + e], J.n_cu);
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) r.set_scalar(e, srow, j[e]);
+            } else {
+#pragma unroll
+                for (int e = 0; e < kVec; ++e) r.set_scalar(e, srow, source_col(b0 + e));
+            }
+            r.store(dst + (size_t)b0 * esz);
+        }
+        const int tail0 = head + body * kVec;
+        for (int t = threadIdx.x; t < head + (n_out - tail0); t += blockDim.x) {
+            const int bb = t < head ? t : tail0 + (t - head);
+            Raw8<DT> r;
+            r.set_scalar(0, srow, source_col(bb));
+            r.put_scalar(0, dst, bb);
         }
     }
+}
+
+// ---------------------------------------------------------------- host side: argument checks and launches
+static int check_score_job(const void* W, int64_t rows, int64_t cols, int64_t ldw, int dtype, const float* norms,
+                           int64_t row_group, int64_t col_group) {
+    const int rc = check_matrix(W, rows, cols, ldw, dtype);
+    if (rc != MOSAIC_OK) return rc;
+    if (rows == 0 || row_group <= 0 || col_group <= 0 || rows % row_group || cols % col_group) return MOSAIC_ERR_INVALID_ARG;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(norms) & 3u) return MOSAIC_ERR_MISALIGNED;
+    return MOSAIC_OK;
+}
+
+template <int NJ>
+static int launch_scores(const ScoreJobList<NJ>& list, int64_t tiles, int64_t units, int dtype, cudaStream_t st) {
+    if (dtype == MOSAIC_BF16) unit_partial_kernel<MOSAIC_BF16, NJ><<<(unsigned)tiles, kSThreads, 0, st>>>(list);
+    else unit_partial_kernel<MOSAIC_F32, NJ><<<(unsigned)tiles, kSThreads, 0, st>>>(list);
+    MOSAIC_LAUNCH_CHECK();
+    unit_score_kernel<NJ><<<(unsigned)((units + 127) / 128), 128, 0, st>>>(list, units);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
+// True iff the kept columns come in whole 16-byte vectors (no staging of the source row needed).
+static bool compact_by_vectors(int64_t cols, int64_t col_group, int64_t col_units_keep) {
+    return (col_group % kVec) == 0 || (col_group == 1 && col_units_keep == cols);
+}
+
+static int check_compact_job(const void* W_in, int64_t rows, int64_t cols, int64_t ldw, int dtype, const int32_t* row_keep,
+                             int64_t row_units_keep, int64_t row_group, const int32_t* col_keep, int64_t col_units_keep,
+                             int64_t col_group, const void* W_out) {
+    const int rc = check_matrix(W_in, rows, cols, ldw, dtype);
+    if (rc != MOSAIC_OK) return rc;
+    if (rows == 0 || row_group <= 0 || col_group <= 0 || rows % row_group || cols % col_group) return MOSAIC_ERR_INVALID_ARG;
+    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    const int64_t n_ru = rows / row_group, n_cu = cols / col_group;
+    if (row_units_keep < 1 || row_units_keep > n_ru || col_units_keep < 1 || col_units_keep > n_cu) return MOSAIC_ERR_INVALID_ARG;
+    if (!row_keep || !col_keep || !W_out) return MOSAIC_ERR_NULL_PTR;
+    if ((reinterpret_cast<uintptr_t>(row_keep) & 3u) || (reinterpret_cast<uintptr_t>(col_keep) & 3u) ||
+        (reinterpret_cast<uintptr_t>(W_out) & 15u))
+        return MOSAIC_ERR_MISALIGNED;
+    const size_t in_span = ((size_t)(rows - 1) * (size_t)ldw + (size_t)cols) * elem_size(dtype);
+    const size_t out_span = (size_t)(row_units_keep * row_group) * (size_t)(col_units_keep * col_group) * elem_size(dtype);
+    const char *a = static_cast<const char*>(W_in), *b = static_cast<const char*>(W_out);
+    if (a < b + out_span && b < a + in_span) return MOSAIC_ERR_ALIASING;
+    // a source row that has to be staged must fit in shared memory (cols <= 51200 fp32)
+    if (!compact_by_vectors(cols, col_group, col_units_keep) &&
+        align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16) > 200 * 1024)
+        return MOSAIC_ERR_INVALID_ARG;
+    return MOSAIC_OK;
+}
+
+static CompactJob make_compact_job(const void* W_in, int64_t rows, int64_t cols, int64_t ldw, const int32_t* row_keep,
+                                   int64_t row_units_keep, int64_t row_group, const int32_t* col_keep, int64_t col_units_keep,
+                                   int64_t col_group, void* W_out, int64_t out_row0) {
+    return CompactJob{W_in, W_out, row_keep, col_keep, cols, ldw, rows / row_group, row_group, cols / col_group, col_group,
+                      row_units_keep * row_group, col_units_keep * col_group, out_row0};
+}
+
+template <int NJ>
+static int launch_compact(const CompactJobList<NJ>& list, int64_t total_out_rows, int dtype, cudaStream_t st) {
+    size_t smem = 0;
+    for (int i = 0; i < list.n; ++i) {
+        const CompactJob& J = list.job[i];
+        if (!compact_by_vectors(J.cols, J.col_group, J.out_cols / J.col_group)) {
+            const size_t need = align_up((size_t)((J.cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
+            if (need > smem) smem = need;
+        }
+    }
+    static DeviceCache attr_set[2];   // the opt-in belongs to one device's copy of the kernel
+    const int opted = attr_set[dtype == MOSAIC_BF16].get([&]() -> int {
+        const cudaError_t e = (dtype == MOSAIC_BF16)
+            ? cudaFuncSetAttribute(compact_kernel<MOSAIC_BF16, NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
+            : cudaFuncSetAttribute(compact_kernel<MOSAIC_F32, NJ>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e != cudaSuccess) (void)cudaGetLastError();
+        return e == cudaSuccess ? 1 : -1;
+    });
+    if (opted < 0) return MOSAIC_ERR_CUDA;
+    // resident CTAs: bounded by the staging buffer (and by 2048 threads per SM)
+    int per_sm = smem == 0 ? 8 : (int)((200 * 1024) / (smem + 1024));
+    per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+    int64_t grid = (int64_t)sm_count() * per_sm;
+    if (grid > total_out_rows) grid = total_out_rows;
+    if (dtype == MOSAIC_BF16) compact_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, 256, smem, st>>>(list, total_out_rows);
+    else compact_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, 256, smem, st>>>(list, total_out_rows);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
 }
 
 }  // namespace mosaic
 
 using namespace mosaic;
 
+// ---------------------------------------------------------------- batched calls
+extern "C" size_t mosaic_unit_scores_batch_workspace_bytes(const mosaic_unit_score_job* jobs, int64_t n_jobs) {
+    size_t total = 256;
+    if (jobs == nullptr) return total;
+    for (int64_t i = 0; i < n_jobs; ++i)
+        if (jobs[i].rows > 0 && jobs[i].cols > 0) total += score_ws_bytes(jobs[i].rows, jobs[i].cols);
+    return total;
+}
+
+extern "C" int mosaic_unit_scores_batch(const mosaic_unit_score_job* jobs, int64_t n_jobs, int dtype, void* ws, size_t ws_bytes,
+                                        void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr || ws == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_unit_score_job& j = jobs[i];
+        const int rc = check_score_job(j.W, j.rows, j.cols, j.ldw, dtype, j.norms, j.row_group, j.col_group);
+        if (rc != MOSAIC_OK) return rc;
+        if ((reinterpret_cast<uintptr_t>(j.row_scores_out) & 3u) || (reinterpret_cast<uintptr_t>(j.col_scores_out) & 3u))
+            return MOSAIC_ERR_MISALIGNED;
+    }
+    if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
+    if (ws_bytes < mosaic_unit_scores_batch_workspace_bytes(jobs, n_jobs)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::unique_ptr<ScoreJobList<kStructBatch>> mem(new (std::nothrow) ScoreJobList<kStructBatch>);
+    if (!mem) return MOSAIC_ERR_INVALID_ARG;
+    ScoreJobList<kStructBatch>& list = *mem;
+    char* wsp = static_cast<char*>(ws);
+    int64_t i = 0;
+    while (i < n_jobs) {
+        list.n = 0;
+        int64_t tiles = 0, units = 0;
+        while (i < n_jobs && list.n < kStructBatch) {
+            const mosaic_unit_score_job& j = jobs[i];
+            int chunks, bands;
+            score_shape(j.rows, j.cols, &chunks, &bands);
+            if (tiles + (int64_t)chunks * bands > 0x3FFFFFFF) break;
+            double* rp = reinterpret_cast<double*>(wsp);
+            double* cpart = reinterpret_cast<double*>(wsp + align_up(sizeof(double) * (size_t)chunks * (size_t)j.rows, 256));
+            list.job[list.n++] = ScoreJob{j.W, j.norms, rp, cpart, j.row_scores_out, j.col_scores_out, j.rows, j.cols, j.ldw,
+                                          j.row_group, j.col_group, units, (int)tiles, chunks, bands, 0};
+            wsp += score_ws_bytes(j.rows, j.cols);
+            tiles += (int64_t)chunks * bands;
+            units += j.rows / j.row_group + j.cols / j.col_group;
+            ++i;
+        }
+        if (list.n == 0) return MOSAIC_ERR_INVALID_ARG;
+        const int rc = launch_scores<kStructBatch>(list, tiles, units, dtype, st);
+        if (rc != MOSAIC_OK) return rc;
+    }
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_rank_units_batch(const mosaic_rank_job* jobs, int64_t n_jobs, void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_rank_job& j = jobs[i];
+        if (!j.scores || (!j.keep_out && j.keep > 0)) return MOSAIC_ERR_NULL_PTR;
+        if (j.n_units <= 0 || j.keep < 0 || j.keep > j.n_units || j.n_units > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(j.scores) & 3u) || (reinterpret_cast<uintptr_t>(j.keep_out) & 3u)) return MOSAIC_ERR_MISALIGNED;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    constexpr int NJ = 4 * kStructBatch;
+    std::unique_ptr<RankJobList<NJ>> mem(new (std::nothrow) RankJobList<NJ>);
+    if (!mem) return MOSAIC_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n_jobs; i += NJ) {
+        mem->n = (int)(n_jobs - i < NJ ? n_jobs - i : NJ);
+        for (int m = 0; m < mem->n; ++m) mem->job[m] = RankJob{jobs[i + m].scores, jobs[i + m].keep_out, jobs[i + m].n_units, jobs[i + m].keep};
+        rank_kernel<NJ><<<(unsigned)mem->n, kRankThreads, 0, st>>>(*mem);
+        MOSAIC_LAUNCH_CHECK();
+    }
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_add_unit_scores_batch(const mosaic_add_job* jobs, int64_t n_jobs, void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_add_job& j = jobs[i];
+        if (j.n < 0) return MOSAIC_ERR_INVALID_ARG;
+        if (j.n > 0 && (!j.dst || !j.a || !j.b)) return MOSAIC_ERR_NULL_PTR;
+        if ((reinterpret_cast<uintptr_t>(j.dst) & 3u) || (reinterpret_cast<uintptr_t>(j.a) & 3u) || (reinterpret_cast<uintptr_t>(j.b) & 3u))
+            return MOSAIC_ERR_MISALIGNED;
+        // dst may be a or b exactly; any partial overlap is refused
+        for (const float* s : {j.a, j.b})
+            if (j.n > 0 && j.dst != s && j.dst < s + j.n && s < j.dst + j.n) return MOSAIC_ERR_ALIASING;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    constexpr int NJ = 4 * kStructBatch;
+    std::unique_ptr<AddJobList<NJ>> mem(new (std::nothrow) AddJobList<NJ>);
+    if (!mem) return MOSAIC_ERR_INVALID_ARG;
+    int64_t i = 0;
+    while (i < n_jobs) {
+        mem->n = 0;
+        int64_t total = 0;
+        for (; i < n_jobs && mem->n < NJ; ++i) {
+            if (jobs[i].n == 0) continue;
+            mem->job[mem->n++] = AddJob{jobs[i].dst, jobs[i].a, jobs[i].b, jobs[i].n, total};
+            total += jobs[i].n;
+        }
+        if (mem->n == 0) break;
+        add_scores_kernel<NJ><<<(unsigned)((total + 255) / 256), 256, 0, st>>>(*mem, total);
+        MOSAIC_LAUNCH_CHECK();
+    }
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_compact_batch(const mosaic_compact_job* jobs, int64_t n_jobs, int dtype, void* stream) {
+    if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
+    if (n_jobs == 0) return MOSAIC_OK;
+    if (jobs == nullptr) return MOSAIC_ERR_NULL_PTR;
+    for (int64_t i = 0; i < n_jobs; ++i) {
+        const mosaic_compact_job& j = jobs[i];
+        const int rc = check_compact_job(j.W_in, j.rows, j.cols, j.ldw, dtype, j.row_keep_units, j.row_units_keep, j.row_group,
+                                         j.col_keep_units, j.col_units_keep, j.col_group, j.W_out);
+        if (rc != MOSAIC_OK) return rc;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::unique_ptr<CompactJobList<kStructBatch>> mem(new (std::nothrow) CompactJobList<kStructBatch>);
+    if (!mem) return MOSAIC_ERR_INVALID_ARG;
+    for (int64_t i = 0; i < n_jobs; i += kStructBatch) {
+        mem->n = (int)(n_jobs - i < kStructBatch ? n_jobs - i : kStructBatch);
+        int64_t total = 0;
+        for (int m = 0; m < mem->n; ++m) {
+            const mosaic_compact_job& j = jobs[i + m];
+            mem->job[m] = make_compact_job(j.W_in, j.rows, j.cols, j.ldw, j.row_keep_units, j.row_units_keep, j.row_group,
+                                           j.col_keep_units, j.col_units_keep, j.col_group, j.W_out, total);
+            total += j.row_units_keep * j.row_group;
+        }
+        const int rc = launch_compact<kStructBatch>(*mem, total, dtype, st);
+        if (rc != MOSAIC_OK) return rc;
+    }
+    return MOSAIC_OK;
+}
+
+// ---------------------------------------------------------------- single calls
 extern "C" size_t mosaic_prune_structured_compact_workspace_bytes(int64_t rows, int64_t cols) {
     if (rows <= 0 || cols <= 0) return 256;
-    return struct_ws(nullptr, rows, cols).bytes;
+    return score_ws_bytes(rows, cols) + align_up(sizeof(float) * (size_t)(rows + cols), 256);
 }
 
 extern "C" int mosaic_rank_units(const float* scores, int64_t n_units, int64_t keep, int32_t* keep_out, void* stream) {
-    if (!scores || (!keep_out && keep > 0)) return MOSAIC_ERR_NULL_PTR;
-    if (n_units <= 0 || keep < 0 || keep > n_units || n_units > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
-    if (keep == 0) return MOSAIC_OK;
-    rank_kernel<<<1, kRankThreads, 0, static_cast<cudaStream_t>(stream)>>>(scores, n_units, keep, keep_out, nullptr, 0, 0,
-                                                                          nullptr);
-    MOSAIC_LAUNCH_CHECK();
-    return MOSAIC_OK;
+    const mosaic_rank_job one{scores, n_units, keep, keep_out};
+    return mosaic_rank_units_batch(&one, 1, stream);
 }
 
 extern "C" int mosaic_sum_unit_scores(float* dst, const float* src, int64_t n_units, void* stream) {
     if (!dst || !src) return MOSAIC_ERR_NULL_PTR;
-    if (n_units < 0) return MOSAIC_ERR_INVALID_ARG;
-    if ((reinterpret_cast<uintptr_t>(dst) & 3u) || (reinterpret_cast<uintptr_t>(src) & 3u)) return MOSAIC_ERR_MISALIGNED;
-    if (dst != src && dst < src + n_units && src < dst + n_units) return MOSAIC_ERR_ALIASING;
-    if (n_units == 0) return MOSAIC_OK;
-    sum_scores_kernel<<<(unsigned)((n_units + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(dst, src, n_units);
-    MOSAIC_LAUNCH_CHECK();
-    return MOSAIC_OK;
+    const mosaic_add_job one{dst, dst, src, n_units};
+    return mosaic_add_unit_scores_batch(&one, 1, stream);
 }
 
 extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, int64_t cols, int64_t ldw, int dtype,
@@ -349,88 +665,69 @@ extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, i
                                                int64_t row_units_keep, int64_t col_units_keep, int32_t* row_keep_units,
                                                int32_t* col_keep_units, int flags, void* W_out, float* unit_scores_out,
                                                void* ws, size_t ws_bytes, void* stream) {
-    int rc = check_matrix(W_in, rows, cols, ldw, dtype);
+    int rc = check_score_job(W_in, rows, cols, ldw, dtype, norms, row_group, col_group);
     if (rc != MOSAIC_OK) return rc;
     const int known = MOSAIC_ROWS_GIVEN | MOSAIC_COLS_GIVEN | MOSAIC_RANK_ONLY | MOSAIC_SCORES_ONLY | MOSAIC_SCORES_ACCUM;
-    if (rows == 0 || (flags & ~known) || row_group <= 0 || col_group <= 0 || rows % row_group || cols % col_group)
-        return MOSAIC_ERR_INVALID_ARG;
-    if (rows > 0x7FFFFFFF || cols > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    if (flags & ~known) return MOSAIC_ERR_INVALID_ARG;
     const int64_t n_ru = rows / row_group, n_cu = cols / col_group;
     const bool scores_only = flags & MOSAIC_SCORES_ONLY;
     const bool rank_only = flags & MOSAIC_RANK_ONLY;
     const bool rows_given = flags & MOSAIC_ROWS_GIVEN, cols_given = flags & MOSAIC_COLS_GIVEN;
     if ((flags & MOSAIC_SCORES_ACCUM) && !unit_scores_out) return MOSAIC_ERR_NULL_PTR;
     if (scores_only && !unit_scores_out) return MOSAIC_ERR_NULL_PTR;
+    if (reinterpret_cast<uintptr_t>(unit_scores_out) & 3u) return MOSAIC_ERR_MISALIGNED;
     if (!scores_only) {
         if (row_units_keep < 1 || row_units_keep > n_ru || col_units_keep < 1 || col_units_keep > n_cu)
             return MOSAIC_ERR_INVALID_ARG;
         if (!row_keep_units || !col_keep_units) return MOSAIC_ERR_NULL_PTR;
         if ((reinterpret_cast<uintptr_t>(row_keep_units) & 3u) || (reinterpret_cast<uintptr_t>(col_keep_units) & 3u))
             return MOSAIC_ERR_MISALIGNED;
+        if (!rank_only) {
+            rc = check_compact_job(W_in, rows, cols, ldw, dtype, row_keep_units, row_units_keep, row_group, col_keep_units,
+                                   col_units_keep, col_group, W_out);
+            if (rc != MOSAIC_OK) return rc;
+        }
     }
     const bool need_scores = scores_only || unit_scores_out || !(rows_given && cols_given);
-    const int64_t out_rows = row_units_keep * row_group, out_cols = col_units_keep * col_group;
-    if (!scores_only && !rank_only) {
-        if (!W_out) return MOSAIC_ERR_NULL_PTR;
-        if (reinterpret_cast<uintptr_t>(W_out) & 15u) return MOSAIC_ERR_MISALIGNED;
-        const size_t in_span = ((size_t)(rows - 1) * (size_t)ldw + (size_t)cols) * elem_size(dtype);
-        const size_t out_span = (size_t)out_rows * (size_t)out_cols * elem_size(dtype);
-        const char *a = static_cast<const char*>(W_in), *b = static_cast<const char*>(W_out);
-        if (a < b + out_span && b < a + in_span) return MOSAIC_ERR_ALIASING;
-    }
-    if ((reinterpret_cast<uintptr_t>(norms) & 3u) || (reinterpret_cast<uintptr_t>(unit_scores_out) & 3u))
-        return MOSAIC_ERR_MISALIGNED;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    StructWs w{};
+    float* scores = nullptr;   // [row units, column units]
     if (need_scores) {
         if (!ws) return MOSAIC_ERR_NULL_PTR;
         if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
         if (ws_bytes < mosaic_prune_structured_compact_workspace_bytes(rows, cols)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
-        w = struct_ws(ws, rows, cols);
-        dim3 grid((unsigned)w.chunks, (unsigned)w.bands);
-        if (dtype == MOSAIC_BF16)
-            unit_partial_kernel<MOSAIC_BF16><<<grid, kSThreads, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_partial, w.col_partial);
-        else
-            unit_partial_kernel<MOSAIC_F32><<<grid, kSThreads, 0, st>>>(W_in, rows, cols, ldw, norms, w.row_partial, w.col_partial);
-        MOSAIC_LAUNCH_CHECK();
+        int chunks, bands;
+        score_shape(rows, cols, &chunks, &bands);
+        char* wsp = static_cast<char*>(ws);
+        double* rp = reinterpret_cast<double*>(wsp);
+        double* cpart = reinterpret_cast<double*>(wsp + align_up(sizeof(double) * (size_t)chunks * (size_t)rows, 256));
+        float* ws_scores = reinterpret_cast<float*>(wsp + score_ws_bytes(rows, cols));
         // with SCORES_ACCUM the running totals live in the caller's array; ranking then uses those
-        float* dst = (flags & MOSAIC_SCORES_ACCUM) ? unit_scores_out : w.scores;
-        const int64_t nu = n_ru + n_cu;
-        unit_score_kernel<<<(unsigned)((nu + 127) / 128), 128, 0, st>>>(w.row_partial, w.chunks, rows, n_ru, row_group,
-                                                                       w.col_partial, w.bands, cols, n_cu, col_group, dst,
-                                                                       (flags & MOSAIC_SCORES_ACCUM) ? 1 : 0);
-        MOSAIC_LAUNCH_CHECK();
-        if (unit_scores_out && dst != unit_scores_out)
-            MOSAIC_CUDA_TRY(cudaMemcpyAsync(unit_scores_out, dst, sizeof(float) * (size_t)nu, cudaMemcpyDeviceToDevice, st));
-        w.scores = dst;
+        scores = (flags & MOSAIC_SCORES_ACCUM) ? unit_scores_out : ws_scores;
+        ScoreJobList<1> one;
+        one.n = 1;
+        one.job[0] = ScoreJob{W_in, norms, rp, cpart, scores, scores + n_ru, rows, cols, ldw, row_group, col_group, 0, 0,
+                              chunks, bands, (flags & MOSAIC_SCORES_ACCUM) ? 1 : 0};
+        rc = launch_scores<1>(one, (int64_t)chunks * bands, n_ru + n_cu, dtype, st);
+        if (rc != MOSAIC_OK) return rc;
+        if (unit_scores_out && scores != unit_scores_out)
+            MOSAIC_CUDA_TRY(cudaMemcpyAsync(unit_scores_out, scores, sizeof(float) * (size_t)(n_ru + n_cu), cudaMemcpyDeviceToDevice, st));
     }
     if (scores_only) return MOSAIC_OK;
 
     if (!(rows_given && cols_given)) {
-        rank_kernel<<<2, kRankThreads, 0, st>>>(w.scores, n_ru, row_units_keep, rows_given ? nullptr : row_keep_units,
-                                                w.scores + n_ru, n_cu, col_units_keep, cols_given ? nullptr : col_keep_units);
+        RankJobList<2> two;
+        two.n = 2;
+        two.job[0] = RankJob{scores, rows_given ? nullptr : row_keep_units, n_ru, rows_given ? 0 : row_units_keep};
+        two.job[1] = RankJob{scores + n_ru, cols_given ? nullptr : col_keep_units, n_cu, cols_given ? 0 : col_units_keep};
+        rank_kernel<2><<<2, kRankThreads, 0, st>>>(two);
         MOSAIC_LAUNCH_CHECK();
     }
     if (rank_only) return MOSAIC_OK;
 
-    const size_t row_smem = align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
-    if (row_smem > 200 * 1024) return MOSAIC_ERR_INVALID_ARG;   // a source row must fit in shared memory (cols <= 51200 fp32)
-    static DeviceCache attr_set[2];   // the opt-in belongs to one device's copy of the kernel
-    const int opted = attr_set[dtype == MOSAIC_BF16].get([&]() -> int {
-        const cudaError_t e = (dtype == MOSAIC_BF16)
-            ? cudaFuncSetAttribute(compact_kernel<MOSAIC_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)
-            : cudaFuncSetAttribute(compact_kernel<MOSAIC_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        if (e != cudaSuccess) (void)cudaGetLastError();
-        return e == cudaSuccess ? 1 : -1;
-    });
-    if (opted < 0) return MOSAIC_ERR_CUDA;
-    if (dtype == MOSAIC_BF16)
-        compact_kernel<MOSAIC_BF16><<<(unsigned)out_rows, 256, row_smem, st>>>(W_in, cols, ldw, row_keep_units, n_ru, row_group,
-                                                                              col_keep_units, n_cu, col_group, out_cols, W_out);
-    else
-        compact_kernel<MOSAIC_F32><<<(unsigned)out_rows, 256, row_smem, st>>>(W_in, cols, ldw, row_keep_units, n_ru, row_group,
-                                                                             col_keep_units, n_cu, col_group, out_cols, W_out);
-    MOSAIC_LAUNCH_CHECK();
-    return MOSAIC_OK;
+    CompactJobList<1> one;
+    one.n = 1;
+    one.job[0] = make_compact_job(W_in, rows, cols, ldw, row_keep_units, row_units_keep, row_group, col_keep_units,
+                                  col_units_keep, col_group, W_out, 0);
+    return launch_compact<1>(one, row_units_keep * row_group, dtype, st);
 }

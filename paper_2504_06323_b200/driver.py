@@ -323,39 +323,102 @@ def prune_structured_independent(st: ModelState, layer: int, proj: str, frac: fl
     return out, rk, ck
 
 
-def prune_structured_model(st: ModelState, frac: float, coupled: bool = True, sources: dict | None = None,
-                           use_norms: bool = True, n_streams: int = 4) -> dict:
-    """The structured stage over every owned layer.  Layers (coupled) or projections (independent)
-    do not depend on one another, so they go round-robin to `n_streams` side streams, each with its
-    own workspace: the ranking kernels - one or two CTAs each - then run beside the score and
-    compaction kernels of other matrices instead of holding the GPU alone.  `sources[layer]`, if
-    given, holds the matrices to read (the masked weights in composite mode).  Returns
-    {layer: result of prune_structured_coupled_layer} or {(layer, proj): (W_compact, row_keep,
-    col_keep)}; the current stream has waited for all of it."""
-    side = _side_streams(st, n_streams)
-    cur = torch.cuda.current_stream(st.device)
-    fork = torch.cuda.Event()
-    fork.record(cur)
-    for s, _ in side:
-        s.wait_event(fork)
-    out: dict = {}
-    i = 0
-    for layer in st.layers:
-        if coupled:
-            s, ws = side[i % n_streams]
-            i += 1
-            with torch.cuda.stream(s):      # buffers made here belong to s: freed ones are reused in s's order
-                out[layer] = prune_structured_coupled_layer(st, layer, frac, None if sources is None else sources[layer],
-                                                            use_norms, ws)
+class _StructuredPlan:
+    """Buffers and marshalled job lists of the structured stage over every owned layer, built once
+    per (fraction, coupling, source matrices) and reused: the stage is then a handful of library
+    calls (scores, sums of coupled scores, ranking, compaction - each one launch or two over all
+    matrices) with no per-projection host work."""
+
+    def __init__(self, st: ModelState, frac: float, coupled: bool, sources: dict | None, use_norms: bool):
+        cfg, dev = st.cfg, st.device
+        f32, i32 = torch.float32, torch.int32
+        self.steps: list = []          # objects with run(...), in order
+        self.out: dict = {}
+        self.ws = api.Workspace(dev)
+        src = {(layer, pr): (sources[layer][pr] if sources is not None else st.W[layer, pr])
+               for layer in st.layers for pr in PROJECTIONS}
+        nrm = {(layer, pr): (st.norms[layer, cfg.x_key(pr)] if use_norms else None) for layer in st.layers for pr in PROJECTIONS}
+        self.keepalive = (src, nrm)
+        score_jobs, rank_jobs, compact_jobs = [], [], []
+        add_steps: list[list] = [[], [], []]
+        if not coupled:
+            for layer in st.layers:
+                for pr in PROJECTIONS:
+                    W = src[layer, pr]
+                    rows, cols = W.shape
+                    kr, kc = rows - int(frac * rows), cols - int(frac * cols)
+                    rs, cs = torch.empty(rows, dtype=f32, device=dev), torch.empty(cols, dtype=f32, device=dev)
+                    rk, ck = torch.empty(kr, dtype=i32, device=dev), torch.empty(kc, dtype=i32, device=dev)
+                    out = torch.empty(kr, kc, dtype=cfg.torch_dtype, device=dev)
+                    score_jobs.append((W, nrm[layer, pr], 1, 1, rs, cs))
+                    rank_jobs += [(rs, kr, rk), (cs, kc, ck)]
+                    compact_jobs.append((W, rk, kr, 1, ck, kc, 1, out))
+                    self.out[layer, pr] = (out, rk, ck)
         else:
-            for pr in PROJECTIONS:
-                s, ws = side[i % n_streams]
-                i += 1
-                with torch.cuda.stream(s):
-                    out[layer, pr] = prune_structured_independent(st, layer, pr, frac, use_norms, ws)
-    join_side(st)
-    for res in out.values():               # the results are used on the current stream from here on
-        tensors = list(res["W"].values()) + [res["mlp_keep"], res["attn_keep"]] if coupled else list(res)
-        for t in tensors:
-            t.record_stream(cur)
-    return out
+            hd, n_kv = cfg.head_dim, cfg.n_kv_heads
+            gq = (cfg.n_heads // n_kv) * hd
+            h, it = cfg.hidden, cfg.intermediate
+            keep_n, keep_a = it - int(frac * it), n_kv - int(frac * n_kv)
+            all_h = torch.arange(h, dtype=i32, device=dev)
+            for layer in st.layers:
+                def vec(n):
+                    return torch.empty(n, dtype=f32, device=dev)
+                g_r, u_r, d_c, q_r, k_r, v_r, o_c = vec(it), vec(it), vec(it), vec(n_kv), vec(n_kv), vec(n_kv), vec(n_kv)
+                S = {pr: src[layer, pr] for pr in PROJECTIONS}
+                N = {pr: nrm[layer, pr] for pr in PROJECTIONS}
+                score_jobs += [(S["gate"], N["gate"], 1, 1, g_r, None), (S["up"], N["up"], 1, 1, u_r, None),
+                               (S["down"], N["down"], 1, 1, None, d_c), (S["q"], N["q"], gq, 1, q_r, None),
+                               (S["k"], N["k"], hd, 1, k_r, None), (S["v"], N["v"], hd, 1, v_r, None),
+                               (S["o"], N["o"], 1, gq, None, o_c)]
+                # (gate + up) + down  and  (q + (k + v)) + o, in fp32, in this order
+                add_steps[0] += [(g_r, g_r, u_r), (k_r, k_r, v_r)]
+                add_steps[1] += [(g_r, g_r, d_c), (q_r, q_r, k_r)]
+                add_steps[2] += [(q_r, q_r, o_c)]
+                ch, grp = torch.empty(keep_n, dtype=i32, device=dev), torch.empty(keep_a, dtype=i32, device=dev)
+                rank_jobs += [(g_r, keep_n, ch), (q_r, keep_a, grp)]
+                Wc = {}
+                for pr in ("gate", "up"):
+                    Wc[pr] = torch.empty(keep_n, h, dtype=cfg.torch_dtype, device=dev)
+                    compact_jobs.append((S[pr], ch, keep_n, 1, all_h, h, 1, Wc[pr]))
+                Wc["down"] = torch.empty(h, keep_n, dtype=cfg.torch_dtype, device=dev)
+                compact_jobs.append((S["down"], all_h, h, 1, ch, keep_n, 1, Wc["down"]))
+                for pr, g in (("q", gq), ("k", hd), ("v", hd)):
+                    Wc[pr] = torch.empty(keep_a * g, h, dtype=cfg.torch_dtype, device=dev)
+                    compact_jobs.append((S[pr], grp, keep_a, g, all_h, h, 1, Wc[pr]))
+                Wc["o"] = torch.empty(h, keep_a * gq, dtype=cfg.torch_dtype, device=dev)
+                compact_jobs.append((S["o"], all_h, h, 1, grp, keep_a, gq, Wc["o"]))
+                self.out[layer] = {"W": Wc, "mlp_keep": ch, "attn_keep": grp}
+        self.score = api.UnitScoreBatch(score_jobs)
+        self.adds = [api.AddBatch(a) for a in add_steps if a]
+        self.rank = api.RankBatch(rank_jobs)
+        self.compact = api.CompactBatch(compact_jobs)
+        self.launches = 2 * ((len(score_jobs) + 127) // 128) + len(self.adds) + (len(rank_jobs) + 511) // 512 + \
+            (len(compact_jobs) + 127) // 128
+
+    def run(self) -> dict:
+        self.score.run(self.ws)
+        for a in self.adds:
+            a.run()
+        self.rank.run()
+        self.compact.run()
+        return self.out
+
+
+def prune_structured_model(st: ModelState, frac: float, coupled: bool = True, sources: dict | None = None,
+                           use_norms: bool = True) -> dict:
+    """The structured stage over every owned layer through the batched calls: unit scores of all
+    matrices, (coupled) the sums of the coupled units' scores, all rankings, all compactions - a
+    launch or two per step for the whole model.  `sources[layer]`, if given, holds the matrices to
+    read (the masked weights in composite mode).  Returns {layer: {"W": {proj: compacted},
+    "mlp_keep", "attn_keep"}} (coupled, as prune_structured_coupled_layer) or {(layer, proj):
+    (W_compact, row_keep, col_keep)}.  Buffers and job lists are built on the first call with a
+    given (frac, coupled, sources) and reused by later ones: the returned tensors are overwritten
+    by the next call with the same arguments."""
+    ident = (float(frac), bool(coupled), bool(use_norms),
+             None if sources is None else tuple(id(sources[layer][pr]) for layer in st.layers for pr in PROJECTIONS),
+             tuple(id(st.W[layer, pr]) for layer in st.layers for pr in PROJECTIONS))
+    hit = st.batches.get("structured")
+    if hit is None or hit[0] != ident:
+        hit = (ident, _StructuredPlan(st, frac, coupled, sources, use_norms))
+        st.batches["structured"] = hit
+    return hit[1].run()

@@ -144,6 +144,12 @@ def test_llama3_8b_layer_composite():
     assert bits_equal(got["attn_keep"].cpu().numpy(), ref["attn_keep"])
     for pr in PROJECTIONS:
         assert bits_equal(wl.to_numpy(got["W"][pr]), ref["W"][pr]), pr
+    # the batched calls (scores, sums, ranking and compaction of all matrices in a launch or two each) give the same bits
+    got_b = driver.prune_structured_model(st, frac, coupled=True, sources={LAYER: masked})[LAYER]
+    torch.cuda.synchronize()
+    assert bits_equal(got_b["mlp_keep"].cpu().numpy(), ref["mlp_keep"]) and bits_equal(got_b["attn_keep"].cpu().numpy(), ref["attn_keep"])
+    for pr in PROJECTIONS:
+        assert bits_equal(wl.to_numpy(got_b["W"][pr]), ref["W"][pr]), pr
     # zeros inside the compacted matrices are the mask's zeros restricted to the kept rows / columns
     ch = ref["mlp_keep"]
     assert bits_equal(wl.to_numpy(got["W"]["gate"]), src["gate"][ch])
@@ -169,3 +175,10 @@ def test_llama7b_structured_layer_rows_and_columns():
             if prev_r is not None:                                                  # nested keep sets
                 assert set(prev_r.tolist()) <= set(rk_ref.tolist()) and set(prev_c.tolist()) <= set(ck_ref.tolist())
             prev_r, prev_c = rk_ref, ck_ref
+    # all seven projections at once through the batched calls
+    got = driver.prune_structured_model(st, 0.3, coupled=False)
+    torch.cuda.synchronize()
+    for pr in PROJECTIONS:
+        out, rk, ck = driver.prune_structured_independent(st, LAYER, pr, 0.3)
+        assert torch.equal(got[LAYER, pr][1], rk) and torch.equal(got[LAYER, pr][2], ck), pr
+        assert bits_equal(wl.to_numpy(got[LAYER, pr][0]), wl.to_numpy(out)), pr

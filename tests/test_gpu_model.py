@@ -205,12 +205,12 @@ def test_norm_calls_on_side_streams_match_the_serial_order():
         assert bits_equal(results[1][key], ref) and bits_equal(results[2][key], ref), key
 
 
-def test_structured_model_over_side_streams_matches_layer_by_layer():
+def test_structured_model_through_batched_calls_matches_layer_by_layer():
     cfg = small("llama3_8b", hidden=640, n_heads=10, n_kv_heads=5, head_dim=64, intermediate=1728, n_layers=5, tokens=1500)
     st = driver.alloc_model(cfg, DEV, outputs=False, masks=False)
     for layer in st.layers:
         driver.accumulate_norms(st, layer, driver.make_activations(cfg, layer, DEV))
-    for rep in range(2):   # the second pass reuses streams, workspaces and freed buffers
+    for rep in range(2):   # the second pass rebuilds the plan over the same matrices
         got = driver.prune_structured_model(st, 0.2, coupled=True)
         torch.cuda.current_stream().synchronize()
         for layer in st.layers:

@@ -570,6 +570,58 @@ def test_structured_given_lists_and_score_accumulation():
     del tot, s_up
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_structured_batched_calls_match_the_oracle(dtype):
+    # several matrices of different shapes and unit sizes through each batched step, against the oracle step by step
+    shapes = [(256, 688, 1, 1), (512, 1024, 64, 1), (96, 4096, 1, 128), (1000, 520, 1, 1), (300, 1000, 1, 8), (64, 64, 1, 1)]
+    Ws, norms, refs = [], [], []
+    for i, (rows, cols, rg, cg) in enumerate(shapes):
+        ld = cols if cols % 8 == 0 else (cols + 7) // 8 * 8
+        W = make(rows, cols, dtype, seed=700 + i, ld=ld, heavy=True)
+        n = norms_for(cols, 90 + i) if i % 2 == 0 else None
+        Ws.append(W)
+        norms.append(n)
+    rs = [torch.full((r // rg,), -1.0, dtype=torch.float32, device=DEV) for r, c, rg, cg in shapes]
+    cs = [torch.full((c // cg,), -1.0, dtype=torch.float32, device=DEV) for r, c, rg, cg in shapes]
+    jobs = [(W, n, rg, cg, rs[i] if i != 4 else None, cs[i]) for i, (W, n, (r, c, rg, cg)) in enumerate(zip(Ws, norms, shapes))]
+    api.mosaic_unit_scores_batch(jobs)
+    agreed = []
+    for i, (W, n, (rows, cols, rg, cg)) in enumerate(zip(Ws, norms, shapes)):
+        nh = None if n is None else n.cpu().numpy()
+        r_ref, c_ref = oracle.unit_scores(host(W), nh, rg, cg, dtype)
+        r_ok, c_ok = oracle.unit_scores_certify(host(W), nh, rg, cg, dtype)
+        c_ag = op.reconcile_fp32(c_ref, cs[i].cpu().numpy(), c_ok)
+        if i != 4:
+            r_ag = op.reconcile_fp32(r_ref, rs[i].cpu().numpy(), r_ok)
+        else:
+            assert (rs[i] == -1.0).all()                         # a NULL output is left alone
+            r_ag = r_ref
+        agreed.append((r_ag, c_ag))
+    # sums of coupled scores: dst = a + b in fp32, dst may be a
+    tot = rs[0].clone()
+    api.mosaic_add_unit_scores_batch([(tot, tot, rs[0]), (cs[5], cs[5], rs[5])])
+    assert_bits_equal(tot.cpu().numpy(), agreed[0][0] + agreed[0][0])
+    assert_bits_equal(cs[5].cpu().numpy(), agreed[5][1] + agreed[5][0])
+    # ranking of every list in one launch
+    fr = [0.3, 0.25, 0.1, 0.5, 0.2, 0.0]
+    keep_r = [len(a[0]) - int(f * len(a[0])) for a, f in zip(agreed, fr)]
+    keep_c = [len(a[1]) - int(f * len(a[1])) for a, f in zip(agreed, fr)]
+    sc_r = [torch.from_numpy(a[0]).to(DEV) for a in agreed]
+    sc_c = [torch.from_numpy(a[1]).to(DEV) for a in agreed]
+    rk = [torch.full((k,), -1, dtype=torch.int32, device=DEV) for k in keep_r]
+    ck = [torch.full((k,), -1, dtype=torch.int32, device=DEV) for k in keep_c]
+    api.mosaic_rank_units_batch([(s, k, o) for s, k, o in zip(sc_r + sc_c, keep_r + keep_c, rk + ck)])
+    for i, a in enumerate(agreed):
+        assert_bits_equal(rk[i].cpu().numpy(), oracle.rank_units(a[0], keep_r[i]))
+        assert_bits_equal(ck[i].cpu().numpy(), oracle.rank_units(a[1], keep_c[i]))
+    # compaction of every matrix in one launch (staged gather, whole vectors of a column unit, whole rows)
+    outs = [torch.full((keep_r[i] * rg, keep_c[i] * cg), 7.0, dtype=Ws[i].dtype, device=DEV) for i, (r, c, rg, cg) in enumerate(shapes)]
+    api.mosaic_compact_batch([(Ws[i], rk[i], keep_r[i], rg, ck[i], keep_c[i], cg, outs[i]) for i, (r, c, rg, cg) in enumerate(shapes)])
+    for i, (rows, cols, rg, cg) in enumerate(shapes):
+        ref = oracle.compact(host(Ws[i]), rk[i].cpu().numpy(), ck[i].cpu().numpy(), rg, cg, dtype)
+        assert_bits_equal(host(outs[i]), ref)
+
+
 def test_rank_units_ties_and_sizes():
     for n, keep in [(8, 7), (50, 20), (1024, 1000), (14336, 11469), (5000, 1), (3000, 3000)]:
         g = torch.Generator(device="cpu").manual_seed(n)
