@@ -23,6 +23,7 @@ _SO = os.path.join(_HERE, "libmosaic_oracle.so")
 F32, BF16 = 0, 1
 MODE_GLOBAL_NORM, MODE_PER_CATEGORY_NORM = 0, 1
 MODE_WEIGHTED_MEAN = 2      # flag, or-ed into the mode
+MODE_REDISTRIBUTE = 4       # flag, or-ed into the mode: clamp and redistribute
 
 
 def build(force: bool = False) -> str:
@@ -131,6 +132,26 @@ def outlier_ratio(W: np.ndarray, norms: np.ndarray, alpha: float = 5.0, dtype=No
                                C.c_float(alpha), C.byref(O), C.byref(s), C.byref(r), C.byref(cert))
     return {"count": int(O.value), "sum": float(s.value), "ratio": float(r.value),
             "certified": bool(cert.value), "numel": rows * cols}
+
+
+def outlier_ratio_group(Ws, norms, alpha: float = 5.0, dtype=None) -> dict:
+    """Eq. 3-4 (layer outlier distribution): one threshold alpha * mean over all matrices of the
+    group; per-matrix counts, their total, the fp64 score sum and R = 100*O/C of the group."""
+    n = len(Ws)
+    code = _code(Ws[0], dtype)
+    for W in Ws:
+        assert _code(W, dtype) == code
+    norms = [np.ascontiguousarray(x, np.float32) for x in norms]
+    PW = (C.c_void_p * n)(*[W.ctypes.data for W in Ws])
+    PN = (C.c_void_p * n)(*[x.ctypes.data for x in norms])
+    I64 = C.c_int64 * n
+    rows, cols, lds = I64(*[W.shape[0] for W in Ws]), I64(*[W.shape[1] for W in Ws]), I64(*[_ld(W) for W in Ws])
+    counts = I64()
+    s, r, cert = C.c_double(0.0), C.c_double(0.0), C.c_int(0)
+    lib().oracle_outlier_ratio_group(PW, rows, cols, lds, code, PN, C.c_int(n), C.c_float(alpha), counts, C.byref(s),
+                                     C.byref(r), C.byref(cert))
+    return {"counts": [int(v) for v in counts], "count": int(sum(counts)), "sum": float(s.value), "ratio": float(r.value),
+            "certified": bool(cert.value), "numel": int(sum(W.size for W in Ws))}
 
 
 def allocate_sparsity(outlier_counts, numels, cols, n_layers: int, n_proj: int, p: float,

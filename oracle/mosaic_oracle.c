@@ -193,6 +193,52 @@ void oracle_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw
     if (certified) *certified = (O == O_lo && O == O_hi);
 }
 
+/*
+ * Layer outlier distribution (Eq. 3-4, the layer-pruning baseline of Section 4.1.3): the same
+ * predicate with ONE threshold for a whole group of matrices (the projections of a layer):
+ *   sum   = sum over the matrices, in list order, of their row-major fp64 score sums
+ *   tau   = (double)alpha * (sum / C),   C = total number of elements of the group
+ *   O_g   = #{ (double) w_ij > tau } in matrix g
+ * counts[g] receives O_g (their total is the layer's O).  certified = 1 iff the total count is
+ * unchanged when tau is moved by +-C*2^-52 relative.
+ */
+void oracle_outlier_ratio_group(const void *const *Ws, const int64_t *rows, const int64_t *cols,
+                                const int64_t *ldws, int dtype, const float *const *norms, int n_mat,
+                                float alpha, int64_t *counts, double *score_sum, double *ratio_percent,
+                                int *certified)
+{
+    double sum = 0.0, C = 0.0;
+    for (int g = 0; g < n_mat; ++g) {
+        for (int64_t i = 0; i < rows[g]; ++i)
+            for (int64_t j = 0; j < cols[g]; ++j)
+                sum = sum + (double)weight_metric(norms[g][j], load_elem(Ws[g], i * ldws[g] + j, dtype));
+        C += (double)(rows[g] * cols[g]);
+    }
+    double mean = sum / C;
+    double tau = (double)alpha * mean;
+    double eps = C * ldexp(1.0, -52);
+    double tau_lo = tau * (1.0 - eps), tau_hi = tau * (1.0 + eps);
+    int64_t total = 0, total_lo = 0, total_hi = 0;
+    for (int g = 0; g < n_mat; ++g) {
+        int64_t O = 0, O_lo = 0, O_hi = 0;
+#pragma omp parallel for schedule(static) reduction(+ : O, O_lo, O_hi)
+        for (int64_t i = 0; i < rows[g]; ++i)
+            for (int64_t j = 0; j < cols[g]; ++j) {
+                double s = (double)weight_metric(norms[g][j], load_elem(Ws[g], i * ldws[g] + j, dtype));
+                O += (s > tau);
+                O_lo += (s > tau_lo);
+                O_hi += (s > tau_hi);
+            }
+        if (counts) counts[g] = O;
+        total += O;
+        total_lo += O_lo;
+        total_hi += O_hi;
+    }
+    if (score_sum) *score_sum = sum;
+    if (ratio_percent) *ratio_percent = 100.0 * (double)total / C;
+    if (certified) *certified = (total == total_lo && total == total_hi);
+}
+
 /* ------------------------------------------------------------------ */
 /* normalize(R_LLM) + Projection Planner (Algorithm 1; Section 3.3      */
 /* component 8; Eq. 1-2).                                              */
@@ -211,6 +257,13 @@ void oracle_outlier_ratio(const void *W, int64_t rows, int64_t cols, int64_t ldw
  * Eq. 1-2.
  * s is clamped to [0, 1 - 1/cols_q]; k_q = floor(s_q * cols_q) weights are
  * removed from every row.  Returns 0, or 1 if any clamp was applied.
+ * mode bit 2 (clamp and redistribute): where a clamp fires, the mean of the
+ * targets would leave p; the clamped targets then stay on their bounds and all
+ * others are shifted by one common amount t that brings the (plain or
+ * weighted) mean of each group back to p - repeated while the shift pushes
+ * further targets over a bound (at most one round per target).  With b_q the
+ * unclamped target:  t = (p*W - sum_clamped w_q s_q - sum_free w_q b_q) / sum_free w_q.
+ * Returns 1 only if p cannot be reached at all (every target of a group on a bound).
  */
 int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numels,
                              const int64_t *cols, int n_layers, int n_proj, double p,
@@ -222,7 +275,7 @@ int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numel
     for (int q = 0; q < total; ++q)
         R[q] = 100.0 * (double)outlier_counts[q] / (double)numels[q];
 
-    int per_category = mode & 1, weighted = (mode >> 1) & 1;
+    int per_category = mode & 1, weighted = (mode >> 1) & 1, redistribute = (mode >> 2) & 1;
     int n_groups = per_category ? n_proj : 1;
     for (int g = 0; g < n_groups; ++g) {
         /* members of this normalisation group, in q order */
@@ -254,6 +307,50 @@ int oracle_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numel
             double d = 2.0 * lambda * r;
             sparsity[q] = (p + dbar) - d;
         }
+    }
+    if (redistribute) {
+        uint8_t *fixed = (uint8_t *)malloc((size_t)total);
+        double *base = (double *)malloc(sizeof(double) * (size_t)total);
+        for (int g = 0; g < n_groups; ++g) {
+            int first = per_category ? g : 0;
+            int step = per_category ? n_proj : 1;
+            int count = per_category ? n_layers : total;
+            int any = 0;
+            for (int c = 0, q = first; c < count; ++c, q += step) {
+                double smax = 1.0 - 1.0 / (double)cols[q];
+                base[q] = sparsity[q];
+                fixed[q] = 0;
+                if (sparsity[q] < 0.0 || sparsity[q] > smax) any = 1;
+            }
+            if (!any) continue;                       /* nothing to clamp: the targets stand as they are */
+            for (int round = 0; round < count; ++round) {
+                double wtot = 0.0, wfree = 0.0, sfixed = 0.0, sfree = 0.0;
+                for (int c = 0, q = first; c < count; ++c, q += step) {
+                    double w = weighted ? (double)numels[q] : 1.0;
+                    wtot = wtot + w;
+                    if (fixed[q]) sfixed = sfixed + w * sparsity[q];
+                    else { wfree = wfree + w; sfree = sfree + w * base[q]; }
+                }
+                if (wfree == 0.0) { clamped = 1; break; }   /* every target on a bound: p is out of reach */
+                double t = (p * wtot - sfixed - sfree) / wfree;
+                int newly = 0;
+                for (int c = 0, q = first; c < count; ++c, q += step) {
+                    if (fixed[q]) continue;
+                    double smax = 1.0 - 1.0 / (double)cols[q];
+                    double v = base[q] + t;
+                    if (v < 0.0) { sparsity[q] = 0.0; fixed[q] = 1; newly = 1; }
+                    else if (v > smax) { sparsity[q] = smax; fixed[q] = 1; newly = 1; }
+                    else sparsity[q] = v;
+                }
+                if (!newly) break;
+            }
+        }
+        free(fixed);
+        free(base);
+        for (int q = 0; q < total; ++q)
+            k_out[q] = (int64_t)floor(sparsity[q] * (double)cols[q]);
+        free(R);
+        return clamped;
     }
     for (int q = 0; q < total; ++q) {
         double smax = 1.0 - 1.0 / (double)cols[q];

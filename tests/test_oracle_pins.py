@@ -491,3 +491,102 @@ def test_allocation_weighted_mean_prunes_exactly_p_of_the_parameters(base):
     a, _, _ = oracle.allocate_sparsity(O % (1 << 20), same, cols, N, M, p, lam, base | oracle.MODE_WEIGHTED_MEAN)
     b, _, _ = oracle.allocate_sparsity(O % (1 << 20), same, cols, N, M, p, lam, base)
     np.testing.assert_allclose(a, b, rtol=0, atol=1e-15)
+
+
+# ----------------------------------------------------------------- layer outlier distribution (Eq. 3-4)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_group_outlier_count_vs_exact_enumeration(dtype):
+    # three matrices of different shapes under ONE threshold alpha * mean over all their scores
+    rng = np.random.default_rng(14)
+    shapes = [(6, 16), (3, 40), (9, 8)]
+    Ws, Wv, norms = [], [], []
+    for rows, cols in shapes:
+        W = rand_matrix(rng, rows, cols, dtype)
+        W_f = as_f32(W, dtype).copy()
+        W_f[rng.random((rows, cols)) < 0.08] *= 30
+        Ws.append(bf16_bits(W_f) if dtype == "bf16" else W_f)
+        Wv.append(as_f32(Ws[-1], dtype))
+        norms.append((rng.random(cols).astype(np.float32) + np.float32(0.1)) * np.float32(10 ** rng.integers(0, 3)))
+    for alpha in (1.0, 3.0, 5.0):
+        sc = [[[Fraction(float(exact_score(n[j], W[i, j]))) for j in range(W.shape[1])] for i in range(W.shape[0])]
+              for W, n in zip(Wv, norms)]
+        C = sum(W.size for W in Wv)
+        total = sum(s for m in sc for r in m for s in r)
+        tau = Fraction(float(np.float32(alpha))) * total / C
+        want = [sum(1 for r in m for s in r if s > tau) for m in sc]
+        got = oracle.outlier_ratio_group(Ws, norms, alpha, dtype)
+        assert got["counts"] == want and got["count"] == sum(want) and got["numel"] == C
+        assert abs(Fraction(got["sum"]) - total) <= total * Fraction(C, 2 ** 52)
+        assert got["ratio"] == 100.0 * sum(want) / C
+
+
+def test_group_of_one_is_the_projection_statistic_and_groups_differ_from_projections():
+    rng = np.random.default_rng(15)
+    W = rand_matrix(rng, 12, 24, "f32")
+    n = rng.random(24).astype(np.float32) + np.float32(0.5)
+    one = oracle.outlier_ratio_group([W], [n], 4.0)
+    ref = oracle.outlier_ratio(W, n, 4.0)
+    assert one["counts"] == [ref["count"]] and one["sum"] == ref["sum"] and one["ratio"] == ref["ratio"]
+    # hand case: A = all ones (4 entries), B = all 100s (4 entries), alpha = 1.5.  Per projection nothing exceeds
+    # 1.5 x its own mean; in the group the mean is 50.5, tau = 75.75: every entry of B is an outlier, none of A.
+    A, B = np.ones((2, 2), np.float32), np.full((2, 2), 100.0, np.float32)
+    ones = np.ones(2, np.float32)
+    assert oracle.outlier_ratio(A, ones, 1.5)["count"] == 0 and oracle.outlier_ratio(B, ones, 1.5)["count"] == 0
+    g = oracle.outlier_ratio_group([A, B], [ones, ones], 1.5)
+    assert g["counts"] == [0, 4] and g["sum"] == 404.0 and g["ratio"] == 50.0 and g["certified"]
+    # a score exactly on the group threshold: not an outlier, and not certified
+    g = oracle.outlier_ratio_group([np.array([[1, 1]], np.float32), np.array([[1, 3]], np.float32)], [ones, ones], 2.0)
+    assert g["counts"] == [0, 0] and not g["certified"]
+
+
+# ----------------------------------------------------------------- clamp and redistribute
+def _wmean(s, w):
+    return float(np.dot(s, w) / np.sum(w))
+
+
+@pytest.mark.parametrize("weighted", [False, True])
+def test_redistribution_keeps_the_mean_at_p_after_clamping(weighted):
+    # ranks spread so widely (lambda = 0.6) that several targets fall below 0 or above 1 - 1/cols
+    counts = [0, 5, 10, 200, 400, 0, 900, 20]
+    numels = [1000, 4000, 1000, 2000, 1000, 8000, 1000, 3000]
+    cols = [10, 40, 10, 20, 10, 80, 10, 30]
+    mode = oracle.MODE_REDISTRIBUTE | (oracle.MODE_WEIGHTED_MEAN if weighted else 0)
+    w = np.array(numels, np.float64) if weighted else np.ones(8)
+    for p in (0.3, 0.5, 0.7):
+        s0, _, clamped0 = oracle.allocate_sparsity(counts, numels, cols, 4, 2, p, 0.6, mode & ~oracle.MODE_REDISTRIBUTE)
+        assert clamped0 and abs(_wmean(s0, w) - p) > 1e-3            # plain clamping leaves the mean off p
+        s, k, infeasible = oracle.allocate_sparsity(counts, numels, cols, 4, 2, p, 0.6, mode)
+        assert not infeasible
+        assert abs(_wmean(s, w) - p) < 1e-14                          # the (weighted) mean is p again
+        smax = 1.0 - 1.0 / np.array(cols)
+        assert (s >= 0).all() and (s <= smax).all()
+        on_bound = (s == 0) | (s == smax)
+        assert on_bound.any() and not on_bound.all()
+        free = ~on_bound                                              # the free targets keep their mutual distances
+        np.testing.assert_allclose(np.diff(s[free]), np.diff(s0_unclamped(counts, numels, cols, p, 0.6, weighted)[free]), atol=1e-15)
+        assert list(k) == [math.floor(a * c) for a, c in zip(s, cols)]
+
+
+def s0_unclamped(counts, numels, cols, p, lam, weighted):
+    R = 100.0 * np.array(counts, np.float64) / np.array(numels, np.float64)
+    r = (R - R.min()) / (R.max() - R.min())
+    d = 2 * lam * r
+    w = np.array(numels, np.float64) if weighted else np.ones(len(counts))
+    return p + np.dot(w, d) / w.sum() - d
+
+
+def test_redistribution_changes_nothing_without_a_clamp_and_flags_the_impossible():
+    counts, numels, cols = [10, 30, 20, 25], [1000] * 4, [100] * 4
+    a = oracle.allocate_sparsity(counts, numels, cols, 2, 2, 0.5, 0.08, 0)
+    b = oracle.allocate_sparsity(counts, numels, cols, 2, 2, 0.5, 0.08, oracle.MODE_REDISTRIBUTE)
+    assert np.array_equal(a[0].view(np.uint64), b[0].view(np.uint64)) and list(a[1]) == list(b[1]) and not b[2]
+    # hand case, two projections, p = 0.5, lambda = 0.8: targets 1.3 and -0.3 -> both on their bounds (0.9 and 0): the
+    # mean 0.45 cannot be brought to 0.5, which is reported
+    s, k, infeasible = oracle.allocate_sparsity([0, 10], [100, 100], [10, 10], 1, 2, 0.5, 0.8, oracle.MODE_REDISTRIBUTE)
+    np.testing.assert_allclose(s, [0.9, 0.0], atol=1e-15)
+    assert infeasible
+    # three projections, R = 0, 50, 100 %, p = 0.5, lambda = 0.5: b = (1.0, 0.5, 0.0) with bounds [0, 0.9]:
+    # the first clamps to 0.9, the others shift by t = (1.5 - 0.9 - 0.5) / 2 = 0.05
+    s, k, infeasible = oracle.allocate_sparsity([0, 50, 100], [100] * 3, [10] * 3, 1, 3, 0.5, 0.5, oracle.MODE_REDISTRIBUTE)
+    np.testing.assert_allclose(s, [0.9, 0.55, 0.05], atol=1e-15)
+    assert not infeasible and list(k) == [9, 5, 0]
