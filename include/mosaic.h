@@ -65,6 +65,10 @@ typedef enum mosaic_dtype { MOSAIC_F32 = 0, MOSAIC_BF16 = 1 } mosaic_dtype;
 #define MOSAIC_WEIGHTED_MEAN 2     /* flag, or-ed in: the targets average to p weighted by
                                       each projection's parameter count, so the pruned share
                                       of all parameters is p (Eq. 1-2 use the plain mean)   */
+#define MOSAIC_REDISTRIBUTE 4      /* flag, or-ed in: clamp and redistribute - a target that
+                                      leaves [0, 1 - 1/cols] stays on the bound and the others
+                                      of its group shift by one common amount so that the mean
+                                      stays p (without it a clamp moves the mean off p)      */
 
 /* flags of mosaic_prune_structured_compact */
 #define MOSAIC_ROWS_GIVEN 1    /* row_keep_units is an input (ascending unit indices)      */
@@ -145,6 +149,21 @@ int mosaic_outlier_ratio_batch(const mosaic_outlier_job *jobs, int64_t n_jobs, i
                                void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * mosaic_outlier_ratio_grouped - the layer outlier distribution (Eq. 3-4, the
+ * layer-pruning baseline of Section 4.1.3): as mosaic_outlier_ratio_batch, but
+ * the matrices of a group (the projections of a layer) are counted against ONE
+ * threshold,  tau_g = (double)alpha * (S_g / C_g),  S_g the sum over the group's
+ * matrices (in list order) of their fp64 score sums, C_g their number of
+ * elements.  Every job's outlier_count_out receives that matrix's count against
+ * its group's tau (their sum is the layer's O); score_sum_out, if given, the
+ * matrix's own S.
+ *   group_of   HOST array, n_jobs entries: jobs of one group are adjacent and
+ *              carry the same value; a group has at most 256 jobs
+ * ------------------------------------------------------------------------- */
+int mosaic_outlier_ratio_grouped(const mosaic_outlier_job *jobs, const int32_t *group_of, int64_t n_jobs,
+                                 int dtype, float alpha, void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
  * mosaic_outlier_ratio_static - mosaic_outlier_ratio without a workspace
  * argument.  (The paper has no counterpart: this is a packaging variant of the
  * call above, not another operation.)
@@ -194,7 +213,15 @@ int mosaic_outlier_ratio_static(const void *W, int64_t rows, int64_t cols, int64
  *     k_q = floor(s_q * cols_q)       (weights removed from every row)
  * MOSAIC_PER_CATEGORY_NORM applies the same over the n_layers entries of each
  * projection index m separately.  Returns MOSAIC_ERR_INFEASIBLE if a clamp
- * fired (outputs are still complete).
+ * fired (outputs are still complete).  With MOSAIC_REDISTRIBUTE, b_q being the
+ * unclamped target: clamped targets keep their bound and every other target of
+ * the group becomes b_q + t,  t = (p*W - sum_clamped w_q s_q - sum_free w_q b_q)
+ * / sum_free w_q, repeated while t pushes further targets over a bound;
+ * MOSAIC_ERR_INFEASIBLE is then returned only if every target of a group sits
+ * on a bound (p out of reach).
+ * For the layer-pruning baseline (Eq. 3-4, one target per layer) pass the
+ * layers' outlier counts with n_proj = 1 and give every projection of layer n
+ * k = floor(s_n * cols).
  * ------------------------------------------------------------------------- */
 int mosaic_allocate_sparsity(const int64_t *outlier_counts, const int64_t *numels,
                              const int64_t *cols, int n_layers, int n_proj, double p,

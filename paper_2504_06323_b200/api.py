@@ -21,6 +21,7 @@ F32, BF16 = 0, 1
 RESET_ACCUM = 1
 GLOBAL_NORM, PER_CATEGORY_NORM = 0, 1
 WEIGHTED_MEAN = 2        # flag, or-ed into the mode
+REDISTRIBUTE = 4         # flag, or-ed into the mode: clamp and redistribute
 ROWS_GIVEN, COLS_GIVEN, RANK_ONLY, SCORES_ONLY, SCORES_ACCUM = 1, 2, 4, 8, 16
 OK, ERR_INFEASIBLE = 0, -9
 
@@ -31,7 +32,7 @@ SYMBOLS = (
     "mosaic_score",
     "mosaic_outlier_ratio_workspace_bytes", "mosaic_outlier_ratio", "mosaic_ratio_from_count",
     "mosaic_outlier_ratio_static_max_workspace_bytes", "mosaic_outlier_ratio_static",
-    "mosaic_outlier_ratio_batch_workspace_bytes", "mosaic_outlier_ratio_batch",
+    "mosaic_outlier_ratio_batch_workspace_bytes", "mosaic_outlier_ratio_batch", "mosaic_outlier_ratio_grouped",
     "mosaic_allocate_sparsity",
     "mosaic_prune_unstructured_workspace_bytes", "mosaic_prune_unstructured",
     "mosaic_prune_unstructured_batch_workspace_bytes", "mosaic_prune_unstructured_batch",
@@ -82,6 +83,8 @@ def lib() -> C.CDLL:
         L.mosaic_outlier_ratio_batch_workspace_bytes.argtypes = [vp, i64]
         L.mosaic_outlier_ratio_batch.restype = ci
         L.mosaic_outlier_ratio_batch.argtypes = [vp, i64, ci, flt, vp, sz, vp]
+        L.mosaic_outlier_ratio_grouped.restype = ci
+        L.mosaic_outlier_ratio_grouped.argtypes = [vp, vp, i64, ci, flt, vp, sz, vp]
         L.mosaic_ratio_from_count.restype = dbl
         L.mosaic_ratio_from_count.argtypes = [i64, i64]
         L.mosaic_allocate_sparsity.restype = ci
@@ -288,10 +291,19 @@ class OutlierBatch:
         self.device = self.jobs[0][0].device
         self.ws_bytes = lib().mosaic_outlier_ratio_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs))
 
-    def run(self, alpha: float, ws: Workspace | None = None, stream=None) -> None:
+    def run(self, alpha: float, ws: Workspace | None = None, stream=None, group_of=None) -> None:
+        """group_of: None (every matrix against its own mean, Eq. 6) or one group id per job - adjacent jobs
+        with equal ids are counted against the mean over the whole group (Eq. 3-4, layer outlier distribution)."""
         wp, wn = _ws(ws, self.device).get(self.ws_bytes)
-        _check(lib().mosaic_outlier_ratio_batch(C.addressof(self.arr), len(self.jobs), self.code, float(alpha), wp, wn,
-                                                _stream(stream)), "mosaic_outlier_ratio_batch")
+        if group_of is None:
+            _check(lib().mosaic_outlier_ratio_batch(C.addressof(self.arr), len(self.jobs), self.code, float(alpha), wp, wn,
+                                                    _stream(stream)), "mosaic_outlier_ratio_batch")
+            return
+        if len(group_of) != len(self.jobs):
+            raise ValueError("one group id per job")
+        g = (C.c_int32 * len(self.jobs))(*[int(v) for v in group_of])
+        _check(lib().mosaic_outlier_ratio_grouped(C.addressof(self.arr), C.addressof(g), len(self.jobs), self.code, float(alpha),
+                                                  wp, wn, _stream(stream)), "mosaic_outlier_ratio_grouped")
 
 
 def mosaic_outlier_ratio_batch(jobs, alpha: float, ws: Workspace | None = None, stream=None) -> None:
@@ -299,6 +311,12 @@ def mosaic_outlier_ratio_batch(jobs, alpha: float, ws: Workspace | None = None, 
     in two launches; the count tensors may be one-element views of a larger int64 tensor."""
     if jobs:
         OutlierBatch(jobs).run(alpha, ws, stream)
+
+
+def mosaic_outlier_ratio_grouped(jobs, group_of, alpha: float, ws: Workspace | None = None, stream=None) -> None:
+    """Eq. 3-4: as mosaic_outlier_ratio_batch, with adjacent jobs of equal group id sharing one threshold."""
+    if jobs:
+        OutlierBatch(jobs).run(alpha, ws, stream, group_of=group_of)
 
 
 def mosaic_ratio_from_count(outlier_count: int, numel: int) -> float:

@@ -1,6 +1,8 @@
 // Host-only entry points and argument validation shared by the device calls.
 #include <math.h>
 
+#include <vector>
+
 #include "common.cuh"
 
 namespace mosaic {
@@ -70,8 +72,9 @@ int mosaic_allocate_sparsity(const int64_t* outlier_counts, const int64_t* numel
                              double* sparsity_out, int64_t* k_out) {
     if (!outlier_counts || !numels || !cols || !sparsity_out || !k_out) return MOSAIC_ERR_NULL_PTR;
     if (n_layers <= 0 || n_proj <= 0 || !(p >= 0.0 && p < 1.0) || !(lambda >= 0.0)) return MOSAIC_ERR_INVALID_ARG;
-    if (mode & ~(MOSAIC_PER_CATEGORY_NORM | MOSAIC_WEIGHTED_MEAN)) return MOSAIC_ERR_INVALID_ARG;
+    if (mode & ~(MOSAIC_PER_CATEGORY_NORM | MOSAIC_WEIGHTED_MEAN | MOSAIC_REDISTRIBUTE)) return MOSAIC_ERR_INVALID_ARG;
     const bool per_category = (mode & MOSAIC_PER_CATEGORY_NORM) != 0, weighted = (mode & MOSAIC_WEIGHTED_MEAN) != 0;
+    const bool redistribute = (mode & MOSAIC_REDISTRIBUTE) != 0;
     const int total = n_layers * n_proj;
     for (int q = 0; q < total; ++q)
         if (numels[q] <= 0 || cols[q] <= 0 || outlier_counts[q] < 0 || outlier_counts[q] > numels[q])
@@ -111,6 +114,47 @@ int mosaic_allocate_sparsity(const int64_t* outlier_counts, const int64_t* numel
         }
     }
     int status = MOSAIC_OK;
+    if (redistribute) {
+        // Targets that leave [0, 1 - 1/cols] stay on the bound; the others of the group move by one
+        // common amount t that brings the (plain or weighted) mean back to p, for as long as the move
+        // pushes further targets over a bound.  sparsity_out holds the unclamped targets b_q on entry.
+        std::vector<char> fixed((size_t)total, 0);
+        std::vector<double> base(sparsity_out, sparsity_out + total);
+        for (int g = 0; g < n_groups; ++g) {
+            bool any = false;
+            for (int c = 0; c < members; ++c) {
+                const int q = g + c * stride;
+                const double smax = 1.0 - 1.0 / (double)cols[q];
+                if (sparsity_out[q] < 0.0 || sparsity_out[q] > smax) any = true;
+            }
+            if (!any) continue;   // nothing to clamp: the targets stand as they are
+            for (int round = 0; round < members; ++round) {
+                double wtot = 0.0, wfree = 0.0, sfixed = 0.0, sfree = 0.0;
+                for (int c = 0; c < members; ++c) {
+                    const int q = g + c * stride;
+                    const double w = weighted ? (double)numels[q] : 1.0;
+                    wtot = wtot + w;
+                    if (fixed[(size_t)q]) sfixed = sfixed + w * sparsity_out[q];
+                    else { wfree = wfree + w; sfree = sfree + w * base[(size_t)q]; }
+                }
+                if (wfree == 0.0) { status = MOSAIC_ERR_INFEASIBLE; break; }   // every target on a bound: p is out of reach
+                const double t = (p * wtot - sfixed - sfree) / wfree;
+                bool newly = false;
+                for (int c = 0; c < members; ++c) {
+                    const int q = g + c * stride;
+                    if (fixed[(size_t)q]) continue;
+                    const double smax = 1.0 - 1.0 / (double)cols[q];
+                    const double v = base[(size_t)q] + t;
+                    if (v < 0.0) { sparsity_out[q] = 0.0; fixed[(size_t)q] = 1; newly = true; }
+                    else if (v > smax) { sparsity_out[q] = smax; fixed[(size_t)q] = 1; newly = true; }
+                    else sparsity_out[q] = v;
+                }
+                if (!newly) break;
+            }
+        }
+        for (int q = 0; q < total; ++q) k_out[q] = (int64_t)floor(sparsity_out[q] * (double)cols[q]);
+        return status;
+    }
     for (int q = 0; q < total; ++q) {
         const double smax = 1.0 - 1.0 / (double)cols[q];
         if (sparsity_out[q] < 0.0) { sparsity_out[q] = 0.0; status = MOSAIC_ERR_INFEASIBLE; }

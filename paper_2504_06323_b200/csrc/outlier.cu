@@ -48,6 +48,7 @@ struct OutlierJob {
     int tile0;             // first global tile
     int chunks;            // tiles per row band
     int ctile0;            // first global tile of the bf16 count sweep (taller tiles)
+    int g_first, g_last;   // jobs of the launch that share this job's threshold (itself alone: Eq. 6; a layer: Eq. 3-4)
 };
 template <int NJ>
 struct OutlierJobList {
@@ -116,6 +117,32 @@ __global__ void __launch_bounds__(kOutThreads) score_sum_kernel(const __grid_con
     }
 }
 
+
+// tau of job j, rounded toward -inf for the fp32 comparison: alpha * (S / C) over the jobs g_first..g_last
+// that share it - each job's partial sums in tile order (thread-strided, then a fixed tree), the jobs in
+// list order.  Block-wide; also writes the job's own sum if asked to.
+template <int NJ>
+__device__ float group_threshold(const OutlierJobList<NJ>& jobs, int j, bool write_sum, double* red, float* tau_sh) {
+    const OutlierJob& J = jobs.job[j];
+    double total = 0.0, numel = 0.0;
+    for (int g = J.g_first; g <= J.g_last; ++g) {
+        const OutlierJob& G = jobs.job[g];
+        const int nt_g = (int)outlier_tiles(G.rows, G.cols);
+        double s = 0.0;
+        for (int i = threadIdx.x; i < nt_g; i += kOutThreads) s += __ldcg(&G.partial[i]);
+        const double sg = block_sum(s, red);   // valid in thread 0
+        total = total + sg;
+        numel = numel + (double)(G.rows * G.cols);
+        if (g == j && write_sum && threadIdx.x == 0 && J.sum_out) *J.sum_out = sg;
+    }
+    if (threadIdx.x == 0) {
+        const double mean = total / numel;
+        *tau_sh = __double2float_rd((double)jobs.alpha * mean);
+    }
+    __syncthreads();
+    return *tau_sh;
+}
+
 template <int DT, int NJ>
 __global__ void __launch_bounds__(kOutThreads) outlier_count_kernel(const __grid_constant__ OutlierJobList<NJ> jobs, int n_tiles) {
     __shared__ double red[32];
@@ -146,19 +173,8 @@ __global__ void __launch_bounds__(kOutThreads) outlier_count_kernel(const __grid
         const int64_t rows = J.rows, cols = J.cols, ldw = J.ldw;
         if (j != j_tau) {
             if (j_tau >= 0) flush(j_tau);
-            // this matrix's partials in tile order: thread-strided, then a fixed tree
             const int nt_j = (int)outlier_tiles(rows, cols);
-            double s = 0.0;
-            for (int i = threadIdx.x; i < nt_j; i += kOutThreads) s += __ldcg(&J.partial[i]);
-            const double total = block_sum(s, red);
-            if (threadIdx.x == 0) {
-                const double mean = total / (double)(rows * cols);
-                const double tau_d = (double)jobs.alpha * mean;
-                tau_sh = __double2float_rd(tau_d);
-                if (tile == J.tile0 + nt_j - 1 && J.sum_out) *J.sum_out = total;   // once: by the CTA that owns the last tile
-            }
-            __syncthreads();
-            tau = tau_sh;
+            tau = group_threshold<NJ>(jobs, j, tile == J.tile0 + nt_j - 1, red, &tau_sh);   // the sum: once, by the CTA that owns the last tile
             j_tau = j;
         }
         const int local = tile - J.tile0;
@@ -312,20 +328,8 @@ __global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(cons
         const OutlierJob& J = jobs.job[j];
         if (j != j_tau) {
             if (j_tau >= 0) flush(j_tau);
-            // this matrix's partials in tile order: thread-strided, then a fixed tree (as in the general kernel)
-            const int nt_j = (int)outlier_tiles(J.rows, J.cols);
-            double s = 0.0;
-            for (int i = threadIdx.x; i < nt_j; i += kOutThreads) s += __ldcg(&J.partial[i]);
-            const double total = block_sum(s, red);
-            if (threadIdx.x == 0) {
-                const double mean = total / (double)(J.rows * J.cols);
-                const double tau_d = (double)jobs.alpha * mean;
-                tau_sh = __double2float_rd(tau_d);
-                const int last = J.ctile0 + (int)outlier_count_tiles(J.rows, J.cols) - 1;
-                if (tile == last && J.sum_out) *J.sum_out = total;   // once: by the CTA that owns the matrix's last tile
-            }
-            __syncthreads();
-            tau = tau_sh;
+            const int last = J.ctile0 + (int)outlier_count_tiles(J.rows, J.cols) - 1;
+            tau = group_threshold<NJ>(jobs, j, tile == last, red, &tau_sh);   // the sum: once, by the CTA that owns the matrix's last tile
             j_tau = j;
         }
         const int local = tile - J.ctile0;
@@ -472,7 +476,7 @@ extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, i
     one.n = 1;
     one.alpha = alpha;
     one.job[0] = OutlierJob{W, norms, reinterpret_cast<unsigned long long*>(outlier_count_out), score_sum_out,
-                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk), 0};
+                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk), 0, 0, 0};
     return launch_outlier<1>(one, outlier_tiles(rows, cols), outlier_count_tiles(rows, cols), dtype,
                              dtype == MOSAIC_BF16 && cols % kVec == 0, static_cast<cudaStream_t>(stream));
 }
@@ -484,8 +488,10 @@ extern "C" size_t mosaic_outlier_ratio_batch_workspace_bytes(const mosaic_outlie
     return total;
 }
 
-extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_t n_jobs, int dtype, float alpha, void* ws,
-                                          size_t ws_bytes, void* stream) {
+// The batched sweeps.  group_of == nullptr: every job has its own threshold (Eq. 6).  Otherwise adjacent
+// jobs with equal group_of share one threshold (Eq. 3-4); a group never straddles two launches.
+static int outlier_batch(const mosaic_outlier_job* jobs, const int32_t* group_of, int64_t n_jobs, int dtype, float alpha,
+                         void* ws, size_t ws_bytes, void* stream) {
     if (n_jobs < 0) return MOSAIC_ERR_INVALID_ARG;
     if (n_jobs == 0) return MOSAIC_OK;
     if (jobs == nullptr || ws == nullptr) return MOSAIC_ERR_NULL_PTR;
@@ -496,6 +502,15 @@ extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_
     }
     if (reinterpret_cast<uintptr_t>(ws) & 255u) return MOSAIC_ERR_MISALIGNED;
     if (ws_bytes < mosaic_outlier_ratio_batch_workspace_bytes(jobs, n_jobs)) return MOSAIC_ERR_WORKSPACE_TOO_SMALL;
+    auto group_end = [&](int64_t i) -> int64_t {   // one past the last job of the group that starts at i
+        int64_t e = i + 1;
+        if (group_of != nullptr)
+            while (e < n_jobs && group_of[e] == group_of[i]) ++e;
+        return e;
+    };
+    if (group_of != nullptr)
+        for (int64_t i = 0; i < n_jobs; i = group_end(i))
+            if (group_end(i) - i > kOutBatch) return MOSAIC_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // host staging of the kernel parameter (on the heap, one per call, so concurrent callers do not meet)
     std::unique_ptr<OutlierJobList<kOutBatch>> list_mem(new (std::nothrow) OutlierJobList<kOutBatch>);
@@ -509,22 +524,40 @@ extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_
         list.n = 0;
         list.alpha = alpha;
         int64_t tiles = 0, ctiles = 0;
-        while (i < n_jobs && list.n < kOutBatch) {
-            const mosaic_outlier_job& j = jobs[i];
-            const int64_t nt = outlier_tiles(j.rows, j.cols);
-            if (tiles + nt > 0x3FFFFFFF) break;
-            list.job[list.n++] = OutlierJob{j.W, j.norms, reinterpret_cast<unsigned long long*>(j.outlier_count_out),
-                                            j.score_sum_out, reinterpret_cast<double*>(wsp), j.rows, j.cols, j.ldw,
-                                            (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk), (int)ctiles};
-            wsp += mosaic_outlier_ratio_workspace_bytes(j.rows, j.cols);
-            tiles += nt;
-            ctiles += outlier_count_tiles(j.rows, j.cols);
-            ++i;
+        while (i < n_jobs) {
+            const int64_t e = group_end(i);
+            int64_t g_tiles = 0;
+            for (int64_t m = i; m < e; ++m) g_tiles += outlier_tiles(jobs[m].rows, jobs[m].cols);
+            if (list.n + (e - i) > kOutBatch || tiles + g_tiles > 0x3FFFFFFF) break;
+            const int g_first = list.n, g_last = list.n + (int)(e - i) - 1;
+            for (int64_t m = i; m < e; ++m) {
+                const mosaic_outlier_job& j = jobs[m];
+                list.job[list.n++] = OutlierJob{j.W, j.norms, reinterpret_cast<unsigned long long*>(j.outlier_count_out),
+                                                j.score_sum_out, reinterpret_cast<double*>(wsp), j.rows, j.cols, j.ldw,
+                                                (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk), (int)ctiles,
+                                                g_first, g_last};
+                wsp += mosaic_outlier_ratio_workspace_bytes(j.rows, j.cols);
+                tiles += outlier_tiles(j.rows, j.cols);
+                ctiles += outlier_count_tiles(j.rows, j.cols);
+            }
+            i = e;
         }
+        if (list.n == 0) return MOSAIC_ERR_INVALID_ARG;   // a single group too large for one launch
         const int rc = launch_outlier<kOutBatch>(list, tiles, ctiles, dtype, lean, st);
         if (rc != MOSAIC_OK) return rc;
     }
     return MOSAIC_OK;
+}
+
+extern "C" int mosaic_outlier_ratio_batch(const mosaic_outlier_job* jobs, int64_t n_jobs, int dtype, float alpha, void* ws,
+                                          size_t ws_bytes, void* stream) {
+    return outlier_batch(jobs, nullptr, n_jobs, dtype, alpha, ws, ws_bytes, stream);
+}
+
+extern "C" int mosaic_outlier_ratio_grouped(const mosaic_outlier_job* jobs, const int32_t* group_of, int64_t n_jobs, int dtype,
+                                            float alpha, void* ws, size_t ws_bytes, void* stream) {
+    if (n_jobs > 0 && group_of == nullptr) return MOSAIC_ERR_NULL_PTR;
+    return outlier_batch(jobs, group_of, n_jobs, dtype, alpha, ws, ws_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -207,6 +207,42 @@ def count_outliers_all(st: ModelState, alpha: float | None = None) -> int:
     return len(jobs)
 
 
+def count_outliers_by_layer(st: ModelState, alpha: float | None = None) -> int:
+    """Layer outlier distribution (Eq. 3-4, the layer-pruning baseline): every projection of a layer
+    is counted against alpha times the mean score of the WHOLE layer.  st.counts receives the
+    per-projection counts (their sum over a layer is the layer's outlier count)."""
+    cfg = st.cfg
+    a = cfg.alpha if alpha is None else alpha
+    if "count_views" not in st.batches or st.batches["count_views"][0] is not st.counts:
+        st.batches["count_views"] = (st.counts, [st.counts[q:q + 1] for q in range(st.counts.numel())])
+    views = st.batches["count_views"][1]
+    jobs = [(st.W[layer, pr], st.norms[layer, cfg.x_key(pr)], views[st.q_local(layer, pr)], None)
+            for layer in st.layers for pr in PROJECTIONS]
+    groups = [i for i, _ in enumerate(st.layers) for _ in PROJECTIONS]
+    if st.ws_batch is None:
+        st.ws_batch = api.Workspace(st.device)
+    _cached_batch(st, "outlier", jobs, api.OutlierBatch).run(a, st.ws_batch, group_of=groups)
+    return len(jobs)
+
+
+def plan_sparsity_by_layer(cfg: ModelConfig, counts: list[int], p: float | None = None, lam: float | None = None,
+                           mode: int = api.GLOBAL_NORM, n_layers: int | None = None):
+    """One target per layer from the layers' outlier counts (normalize + planner over N entries, one
+    "projection" per layer); every projection of layer n gets k = floor(s_n * cols).  Returns
+    (s per layer, k per (layer, projection), infeasible)."""
+    import math
+    n_layers = cfg.n_layers if n_layers is None else n_layers
+    M = len(PROJECTIONS)
+    per_layer = sum(r * c for r, c in (cfg.shape(pr) for pr in PROJECTIONS))
+    layer_counts = [sum(counts[n * M:(n + 1) * M]) for n in range(n_layers)]
+    # the clamp bound needs a column count: the shortest row of the layer is the binding one
+    min_cols = min(cfg.shape(pr)[1] for pr in PROJECTIONS)
+    s, _, infeasible = api.mosaic_allocate_sparsity(layer_counts, [per_layer] * n_layers, [min_cols] * n_layers, n_layers, 1,
+                                                    cfg.p if p is None else p, cfg.lam if lam is None else lam, mode)
+    k = [int(math.floor(s[n] * cfg.shape(pr)[1])) for n in range(n_layers) for pr in PROJECTIONS]
+    return s, k, infeasible
+
+
 # ------------------------------------------------------------------ phase B
 def prune_unstructured_layer(st: ModelState, layer: int, k_global: list[int], in_place: bool = False) -> int:
     cfg = st.cfg

@@ -226,3 +226,32 @@ def test_structured_model_through_batched_calls_matches_layer_by_layer():
                 g = got[layer, pr]
                 assert torch.equal(g[1], rk) and torch.equal(g[2], ck)
                 assert bits_equal(wl.to_numpy(g[0]), wl.to_numpy(out)), (rep, layer, pr)
+
+
+def test_layer_pruning_baseline_model():
+    # Eq. 3-4 / the layer method of Section 4.1.3: one outlier statistic and one target per layer
+    cfg = small("llama7b", n_layers=3)
+    st, Wh, Xh, norms_ref, _ = run_phase_a(cfg)
+    driver.count_outliers_by_layer(st)
+    counts = driver.exchange_counts(st.counts, cfg.n_layers, 0, 1)
+    M = len(PROJECTIONS)
+    layer_counts = []
+    for layer in st.layers:
+        ref = oracle.outlier_ratio_group([Wh[layer, pr] for pr in PROJECTIONS], [norms_ref[layer, cfg.x_key(pr)] for pr in PROJECTIONS],
+                                         cfg.alpha, cfg.dtype)
+        assert ref["certified"] and counts[layer * M:(layer + 1) * M] == ref["counts"]
+        layer_counts.append(ref["count"])
+    s, k, infeasible = driver.plan_sparsity_by_layer(cfg, counts, lam=0.15)
+    per_layer = sum(r * c for r, c in (cfg.shape(pr) for pr in PROJECTIONS))
+    min_cols = min(cfg.shape(pr)[1] for pr in PROJECTIONS)
+    s_ref, _, inf_ref = oracle.allocate_sparsity(layer_counts, [per_layer] * cfg.n_layers, [min_cols] * cfg.n_layers, cfg.n_layers, 1,
+                                                 cfg.p, 0.15)
+    assert np.array_equal(np.array(s).view(np.uint64), s_ref.view(np.uint64)) and infeasible == inf_ref
+    assert abs(np.mean(s) - cfg.p) < 1e-12 and len(set(s)) == cfg.n_layers          # one target per layer, mean p
+    assert k == [int(np.floor(s_ref[n] * cfg.shape(pr)[1])) for n in range(cfg.n_layers) for pr in PROJECTIONS]
+    driver.prune_unstructured_all(st, k)
+    for layer in st.layers:
+        ref = op.unstructured(cfg, Wh, norms_ref, layer, k)
+        for pr in PROJECTIONS:
+            assert bits_equal(wl.to_numpy(st.W_out[layer, pr]), ref[pr][0]), (layer, pr)
+            assert bits_equal(st.mask[layer, pr].cpu().numpy().view(np.uint32), ref[pr][1]), (layer, pr)

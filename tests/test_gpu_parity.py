@@ -183,6 +183,36 @@ def test_outlier_ratio_uneven_rows_and_dense_threshold(dtype):
     assert ref["certified"] and cnt.item() == ref["count"] and 0 < ref["count"] < 600 * 2048
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_outlier_ratio_grouped_matches_oracle(dtype):
+    # Eq. 3-4: the matrices of a group are counted against ONE threshold; three groups of different sizes
+    shapes = [(256, 256), (688, 256), (256, 688), (300, 1000), (1100, 4096), (64, 11008), (65, 1024), (1, 8), (40, 2048)]
+    groups = [0, 0, 0, 1, 1, 2, 2, 2, 2]
+    Ws, norms = [], []
+    for i, (rows, cols) in enumerate(shapes):
+        W = make(rows, cols, dtype, seed=1300 + i, heavy=(i % 2 == 1), scale=0.02 * (1 + 3 * (i % 3)))
+        Ws.append(W)
+        norms.append(norms_for(cols, 110 + i))
+    counts = torch.full((len(shapes),), -5, dtype=torch.int64, device=DEV)
+    sums = torch.full((len(shapes),), -1.0, dtype=torch.float64, device=DEV)
+    jobs = [(W, n, counts[i:i + 1], sums[i:i + 1]) for i, (W, n) in enumerate(zip(Ws, norms))]
+    api.mosaic_outlier_ratio_grouped(jobs, groups, 4.0)
+    got = counts.cpu().tolist()
+    for g in sorted(set(groups)):
+        idx = [i for i, x in enumerate(groups) if x == g]
+        ref = oracle.outlier_ratio_group([host(Ws[i]) for i in idx], [norms[i].cpu().numpy() for i in idx], 4.0, dtype)
+        assert ref["certified"] and ref["count"] > 0
+        assert [got[i] for i in idx] == ref["counts"], g
+        np.testing.assert_allclose(sum(sums[i].item() for i in idx), ref["sum"], rtol=1e-12)
+    # the grouped count differs from the per-matrix one somewhere (else the test shows nothing)
+    api.mosaic_outlier_ratio_batch(jobs, 4.0)
+    assert counts.cpu().tolist() != got
+    # groups of one matrix each are the per-matrix statistic
+    per_matrix = counts.cpu().tolist()
+    api.mosaic_outlier_ratio_grouped(jobs, list(range(len(shapes))), 4.0)
+    assert counts.cpu().tolist() == per_matrix
+
+
 def test_outlier_planted_and_constant():
     rows, cols = 64, 1024
     W = torch.ones(rows, cols, dtype=torch.bfloat16, device=DEV)

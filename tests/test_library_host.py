@@ -63,8 +63,10 @@ def test_argument_validation_needs_no_device(lib):
 
 
 @pytest.mark.parametrize("mode", [api.GLOBAL_NORM, api.PER_CATEGORY_NORM, api.GLOBAL_NORM | api.WEIGHTED_MEAN,
-                                  api.PER_CATEGORY_NORM | api.WEIGHTED_MEAN])
-@pytest.mark.parametrize("p,lam", [(0.5, 0.08), (0.8, 0.15), (0.1, 0.0), (0.7, 0.3)])
+                                  api.PER_CATEGORY_NORM | api.WEIGHTED_MEAN, api.REDISTRIBUTE,
+                                  api.REDISTRIBUTE | api.WEIGHTED_MEAN, api.REDISTRIBUTE | api.PER_CATEGORY_NORM,
+                                  api.REDISTRIBUTE | api.PER_CATEGORY_NORM | api.WEIGHTED_MEAN])
+@pytest.mark.parametrize("p,lam", [(0.5, 0.08), (0.8, 0.15), (0.1, 0.0), (0.7, 0.3), (0.9, 0.6), (0.05, 0.5)])
 def test_allocate_sparsity_bit_exact_vs_oracle(lib, mode, p, lam):
     rng = np.random.default_rng(42)
     for N, M in [(1, 7), (32, 7), (40, 7), (3, 2)]:
