@@ -8,9 +8,9 @@
 //            columns (a lane owns two vectors of 8 adjacent columns) and takes every fourth row:
 //            every score goes to the lane's column accumulators and to the row's partial sum
 //            (fp64); a row's partial over the tile is combined by a fixed butterfly, the tiles of
-//            a row in column order, the warps' and the row bands' column partials in index order.
-//            One fp64 sum per unit over its rows / columns in index order follows, rounded once
-//            to fp32.  Nothing depends on the launch shape.
+//            a row in column order, the warps' and the row bands' column partials in index order
+//            (one thread per row / column).  One fp64 sum per unit over its rows / columns in
+//            index order follows, rounded once to fp32.  Nothing depends on the launch shape.
 //   rank   : one CTA per list of units; 4 x 8-bit radix select on the fp32 score bits finds the
 //            threshold key and tie quota; an ordered block scan then emits the ascending keep
 //            list (ties: lowest index removed first).
@@ -41,6 +41,7 @@ struct ScoreJob {
     float* col_out;        // [cols / col_group] or nullptr
     int64_t rows, cols, ldw, row_group, col_group;
     int64_t unit0;         // first global unit (row units, then column units)
+    int64_t line0;         // first global line (rows, then columns)
     int tile0, chunks, bands, accumulate;
 };
 template <int NJ>
@@ -169,8 +170,33 @@ __global__ void __launch_bounds__(kSThreads) unit_partial_kernel(const __grid_co
     }
 }
 
-// Unit score = fp64 sum over the unit's rows (tile partials in column order) or columns (band
-// partials in band order), in index order, rounded once to fp32.  One thread per unit of the list.
+// Line sums: for every row the fp64 sum of its tile partials in column order, for every column
+// the sum of its band partials in band order, written over the first partial of the line.  One
+// thread per line (row lines first, then column lines) of the list.
+template <int NJ>
+__global__ void line_sum_kernel(const __grid_constant__ ScoreJobList<NJ> jobs, int64_t total_lines) {
+    const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= total_lines) return;
+    const ScoreJob& J = jobs.job[find_job(jobs.n, g, [&](int i) { return jobs.job[i].line0; })];
+    const int64_t l = g - J.line0;
+    if (l < J.rows) {
+        if (J.row_out == nullptr) return;
+        double rs = 0.0;
+#pragma unroll 8
+        for (int p = 0; p < J.chunks; ++p) rs += J.row_partial[(int64_t)p * J.rows + l];
+        J.row_partial[l] = rs;
+    } else {
+        if (J.col_out == nullptr) return;
+        const int64_t c = l - J.rows;
+        double cs = 0.0;
+#pragma unroll 16
+        for (int p = 0; p < J.bands; ++p) cs += J.col_partial[(int64_t)p * J.cols + c];   // loads batched, adds in order
+        J.col_partial[c] = cs;
+    }
+}
+
+// Unit score = fp64 sum of the unit's line sums in index order, rounded once to fp32.  One thread
+// per unit of the list.
 template <int NJ>
 __global__ void unit_score_kernel(const __grid_constant__ ScoreJobList<NJ> jobs, int64_t total_units) {
     const int64_t g = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -181,22 +207,14 @@ __global__ void unit_score_kernel(const __grid_constant__ ScoreJobList<NJ> jobs,
     float* out;
     if (u < n_ru) {
         if (J.row_out == nullptr) return;
-        for (int64_t i = u * J.row_group; i < (u + 1) * J.row_group; ++i) {
-            double rs = 0.0;
 #pragma unroll 8
-            for (int p = 0; p < J.chunks; ++p) rs += J.row_partial[(int64_t)p * J.rows + i];
-            s += rs;
-        }
+        for (int64_t i = u * J.row_group; i < (u + 1) * J.row_group; ++i) s += J.row_partial[i];
         out = J.row_out + u;
     } else {
         if (J.col_out == nullptr) return;
         const int64_t v = u - n_ru;
-        for (int64_t c = v * J.col_group; c < (v + 1) * J.col_group; ++c) {
-            double cs = 0.0;
-#pragma unroll 16
-            for (int p = 0; p < J.bands; ++p) cs += J.col_partial[(int64_t)p * J.cols + c];   // loads batched, adds in order
-            s += cs;
-        }
+#pragma unroll 8
+        for (int64_t c = v * J.col_group; c < (v + 1) * J.col_group; ++c) s += J.col_partial[c];
         out = J.col_out + v;
     }
     const float f = (float)s;
@@ -426,9 +444,11 @@ static int check_score_job(const void* W, int64_t rows, int64_t cols, int64_t ld
 }
 
 template <int NJ>
-static int launch_scores(const ScoreJobList<NJ>& list, int64_t tiles, int64_t units, int dtype, cudaStream_t st) {
+static int launch_scores(const ScoreJobList<NJ>& list, int64_t tiles, int64_t units, int64_t lines, int dtype, cudaStream_t st) {
     if (dtype == MOSAIC_BF16) unit_partial_kernel<MOSAIC_BF16, NJ><<<(unsigned)tiles, kSThreads, 0, st>>>(list);
     else unit_partial_kernel<MOSAIC_F32, NJ><<<(unsigned)tiles, kSThreads, 0, st>>>(list);
+    MOSAIC_LAUNCH_CHECK();
+    line_sum_kernel<NJ><<<(unsigned)((lines + 127) / 128), 128, 0, st>>>(list, lines);
     MOSAIC_LAUNCH_CHECK();
     unit_score_kernel<NJ><<<(unsigned)((units + 127) / 128), 128, 0, st>>>(list, units);
     MOSAIC_LAUNCH_CHECK();
@@ -536,7 +556,7 @@ extern "C" int mosaic_unit_scores_batch(const mosaic_unit_score_job* jobs, int64
     int64_t i = 0;
     while (i < n_jobs) {
         list.n = 0;
-        int64_t tiles = 0, units = 0;
+        int64_t tiles = 0, units = 0, lines = 0;
         while (i < n_jobs && list.n < kStructBatch) {
             const mosaic_unit_score_job& j = jobs[i];
             int chunks, bands;
@@ -545,14 +565,15 @@ extern "C" int mosaic_unit_scores_batch(const mosaic_unit_score_job* jobs, int64
             double* rp = reinterpret_cast<double*>(wsp);
             double* cpart = reinterpret_cast<double*>(wsp + align_up(sizeof(double) * (size_t)chunks * (size_t)j.rows, 256));
             list.job[list.n++] = ScoreJob{j.W, j.norms, rp, cpart, j.row_scores_out, j.col_scores_out, j.rows, j.cols, j.ldw,
-                                          j.row_group, j.col_group, units, (int)tiles, chunks, bands, 0};
+                                          j.row_group, j.col_group, units, lines, (int)tiles, chunks, bands, 0};
             wsp += score_ws_bytes(j.rows, j.cols);
             tiles += (int64_t)chunks * bands;
             units += j.rows / j.row_group + j.cols / j.col_group;
+            lines += j.rows + j.cols;
             ++i;
         }
         if (list.n == 0) return MOSAIC_ERR_INVALID_ARG;
-        const int rc = launch_scores<kStructBatch>(list, tiles, units, dtype, st);
+        const int rc = launch_scores<kStructBatch>(list, tiles, units, lines, dtype, st);
         if (rc != MOSAIC_OK) return rc;
     }
     return MOSAIC_OK;
@@ -706,9 +727,9 @@ extern "C" int mosaic_prune_structured_compact(const void* W_in, int64_t rows, i
         scores = (flags & MOSAIC_SCORES_ACCUM) ? unit_scores_out : ws_scores;
         ScoreJobList<1> one;
         one.n = 1;
-        one.job[0] = ScoreJob{W_in, norms, rp, cpart, scores, scores + n_ru, rows, cols, ldw, row_group, col_group, 0, 0,
+        one.job[0] = ScoreJob{W_in, norms, rp, cpart, scores, scores + n_ru, rows, cols, ldw, row_group, col_group, 0, 0, 0,
                               chunks, bands, (flags & MOSAIC_SCORES_ACCUM) ? 1 : 0};
-        rc = launch_scores<1>(one, (int64_t)chunks * bands, n_ru + n_cu, dtype, st);
+        rc = launch_scores<1>(one, (int64_t)chunks * bands, n_ru + n_cu, rows + cols, dtype, st);
         if (rc != MOSAIC_OK) return rc;
         if (unit_scores_out && scores != unit_scores_out)
             MOSAIC_CUDA_TRY(cudaMemcpyAsync(unit_scores_out, scores, sizeof(float) * (size_t)(n_ru + n_cu), cudaMemcpyDeviceToDevice, st));

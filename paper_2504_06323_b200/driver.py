@@ -428,7 +428,7 @@ class _StructuredPlan:
         self.adds = [api.AddBatch(a) for a in add_steps if a]
         self.rank = api.RankBatch(rank_jobs)
         self.compact = api.CompactBatch(compact_jobs)
-        self.launches = 2 * ((len(score_jobs) + 127) // 128) + len(self.adds) + (len(rank_jobs) + 511) // 512 + \
+        self.launches = 3 * ((len(score_jobs) + 127) // 128) + len(self.adds) + (len(rank_jobs) + 511) // 512 + \
             (len(compact_jobs) + 127) // 128
 
     def run(self) -> dict:
