@@ -4,11 +4,11 @@
 // matrices and do each step for all of them in one launch (a model has N*M projections; one
 // launch chain per projection is bound by launch latency and by the host).
 //
-//   scores : one sweep over W in tiles of 512 columns x 256 rows.  A warp covers the tile's 512
-//            columns (a lane owns two vectors of 8 adjacent columns) and takes every fourth row:
-//            every score goes to the lane's column accumulators and to the row's partial sum
-//            (fp64); a row's partial over the tile is combined by a fixed butterfly, the tiles of
-//            a row in column order, the warps' and the row bands' column partials in index order
+//   scores : one sweep over W in tiles of 256 columns x 256 rows.  A warp covers the tile's 256
+//            columns (a lane owns 8 adjacent ones) and takes every fourth row: every score goes to
+//            the lane's column accumulators and to the row's partial sum (fp64); a row's partial
+//            over the tile is the lanes' sums added in lane order (through shared memory), the tiles
+//            of a row in column order, the warps' and the row bands' column partials in index order
 //            (one thread per row / column).  One fp64 sum per unit over its rows / columns in
 //            index order follows, rounded once to fp32.  Nothing depends on the launch shape.
 //   rank   : one CTA per list of units; 4 x 8-bit radix select on the fp32 score bits finds the
@@ -26,8 +26,9 @@
 namespace mosaic {
 
 constexpr int kRankThreads = 1024;
-constexpr int kSTileCols = 512;    // columns per tile: a warp row of 32 lanes x 2 vectors of 8 columns
+constexpr int kSTileCols = 256;    // columns per tile: a warp row of 32 lanes x 8 columns
 constexpr int kSTileRows = 256;    // rows per tile, dealt round-robin to the CTA's warps
+constexpr int kSSubRows = 64;      // rows whose lane sums wait in shared memory for the per-row addition
 constexpr int kSThreads = 128;
 constexpr int kSWarps = kSThreads / 32;
 constexpr int kStructBatch = 128;  // matrices per launch (the list travels as a kernel parameter)
@@ -106,58 +107,63 @@ __device__ __forceinline__ int find_job(int n, int64_t x, F first) {
     return lo;
 }
 
-// One tile per CTA.  All sums in fp64.
+// One tile per CTA.  All sums in fp64.  The tile's rows are worked through in sub-tiles of 64: a
+// lane adds the 8 scores of its vector of a row into its column accumulators and leaves their sum
+// in shared memory; after the sub-tile one thread per row adds the 32 lane sums in lane order.
 template <int DT, int NJ>
-__global__ void __launch_bounds__(kSThreads) unit_partial_kernel(const __grid_constant__ ScoreJobList<NJ> jobs) {
+__global__ void __launch_bounds__(kSThreads, 6) unit_partial_kernel(const __grid_constant__ ScoreJobList<NJ> jobs) {
     __shared__ double cp[kSWarps][kSTileCols + 2];
+    __shared__ double rowbuf[32][kSSubRows + 1];   // [lane][row of the sub-tile]
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const int tile = blockIdx.x;
     const ScoreJob& J = jobs.job[find_job(jobs.n, tile, [&](int i) { return (int64_t)jobs.job[i].tile0; })];
     const int local = tile - J.tile0;
     const int chunk = local % J.chunks, band = local / J.chunks;
     const int64_t rows = J.rows, cols = J.cols, ldw = J.ldw;
-    const int64_t c0 = (int64_t)chunk * kSTileCols + lane * kVec, c1 = c0 + 32 * kVec;
+    const int64_t c0 = (int64_t)chunk * kSTileCols + lane * kVec;
     const int64_t r0 = (int64_t)band * kSTileRows;
     const int64_t r1 = (r0 + kSTileRows < rows) ? r0 + kSTileRows : rows;
-    float nrm[2][kVec];
-    double acc[2][kVec];
+    float nrm[kVec];
+    double acc[kVec];
 #pragma unroll
     for (int e = 0; e < kVec; ++e) {
-        acc[0][e] = acc[1][e] = 0.0;
-        nrm[0][e] = (c0 + e < cols) ? (J.norms ? J.norms[c0 + e] : 1.0f) : 0.0f;
-        nrm[1][e] = (c1 + e < cols) ? (J.norms ? J.norms[c1 + e] : 1.0f) : 0.0f;
+        acc[e] = 0.0;
+        nrm[e] = (c0 + e < cols) ? (J.norms ? J.norms[c0 + e] : 1.0f) : 0.0f;
     }
-    constexpr int U = 2;   // rows in flight per warp
-    for (int64_t r = r0 + wid; r < r1; r += U * kSWarps) {
-        Raw8<DT> v[U][2];
+    constexpr int U = 4;   // rows in flight per warp
+    for (int64_t rs = r0; rs < r1; rs += kSSubRows) {
+#pragma unroll 1
+        for (int i = wid; i < kSSubRows; i += U * kSWarps) {
+            Raw8<DT> v[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t rr = r + u * kSWarps;
-            if (rr < r1 && c0 < cols) load_vec<DT, true>(v[u][0], J.W, rr * ldw, c0, cols);
-            else v[u][0].clear();
-            if (rr < r1 && c1 < cols) load_vec<DT, true>(v[u][1], J.W, rr * ldw, c1, cols);
-            else v[u][1].clear();
-        }
+            for (int u = 0; u < U; ++u) {
+                const int64_t rr = rs + i + u * kSWarps;
+                if (rr < r1 && c0 < cols) load_vec<DT, true>(v[u], J.W, rr * ldw, c0, cols);
+                else v[u].clear();
+            }
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int64_t rr = r + u * kSWarps;
-            double p = 0.0;
-#pragma unroll
-            for (int h = 0; h < 2; ++h)
+            for (int u = 0; u < U; ++u) {
+                double p = 0.0;
 #pragma unroll
                 for (int e = 0; e < kVec; ++e) {
-                    const double s = (double)__fmul_rn(nrm[h][e], v[u][h].abs_f32(e));
-                    acc[h][e] += s;
+                    const double s = (double)__fmul_rn(nrm[e], v[u].abs_f32(e));
+                    acc[e] += s;
                     p += s;
                 }
-            p = warp_sum(p);
-            if (lane == 0 && rr < r1) J.row_partial[(int64_t)chunk * rows + rr] = p;
+                rowbuf[lane][i + u * kSWarps] = p;
+            }
         }
+        __syncthreads();
+        if (threadIdx.x < kSSubRows && rs + threadIdx.x < r1) {
+            double s = 0.0;
+#pragma unroll
+            for (int l = 0; l < 32; ++l) s += rowbuf[l][threadIdx.x];
+            J.row_partial[(int64_t)chunk * rows + rs + threadIdx.x] = s;
+        }
+        __syncthreads();
     }
 #pragma unroll
-    for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int e = 0; e < kVec; ++e) cp[wid][h * 256 + lane * kVec + e] = acc[h][e];
+    for (int e = 0; e < kVec; ++e) cp[wid][lane * kVec + e] = acc[e];
     __syncthreads();
     for (int i = threadIdx.x; i < kSTileCols; i += kSThreads) {
         const int64_t c = (int64_t)chunk * kSTileCols + i;
