@@ -384,6 +384,26 @@ def test_prune_rows_of_very_different_scale(dtype):
         _check_prune(W, norms, k, dtype)
 
 
+@pytest.mark.parametrize("cols", [4096, 11008])
+def test_prune_thresholds_across_and_beyond_the_window(cols):
+    # rows of one matrix scaled by factors that rise smoothly over +-8 %: their thresholds sweep through the
+    # matrix's whole window of score keys, sit on its edges and fall just outside it (the kernel's window holds
+    # about +-3 sigma of the rank scatter of equally scaled rows, a few per cent in score)
+    rows = 640 if cols == 4096 else 320
+    W = make(rows, cols, "bf16", seed=cols + 5)
+    scale = (1.0 + 0.16 * (torch.arange(rows, device=DEV).float() / rows - 0.5))[:, None]
+    W = (W.float() * scale).to(torch.bfloat16)
+    for norms in (norms_for(cols, 51), torch.full((cols,), 37.5, dtype=torch.float32, device=DEV)):
+        for k in (cols // 2, (3 * cols) // 10):
+            _check_prune(W, norms, k, "bf16")
+            out = torch.full_like(W, 3.0)
+            mask = torch.full((rows, (cols + 31) // 32), -1, dtype=torch.int32, device=DEV)
+            api.mosaic_prune_unstructured_batch([(W, out, norms, k, mask)])
+            ref_W, ref_mask = oracle.prune_unstructured(host(W), norms.cpu().numpy(), k, "bf16")
+            assert_bits_equal(host(out), ref_W)
+            assert_bits_equal(mask.cpu().numpy().view(np.uint32), ref_mask)
+
+
 def test_prune_already_pruned_matrix():
     # half of every row is exactly zero (a matrix pruned before): thousands of tied keys at +0
     rows, cols = 1200, 4096
