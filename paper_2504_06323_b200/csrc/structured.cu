@@ -402,30 +402,46 @@ __global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ Co
                                                     r.w[6 % (Raw8<DT>::kBytes / 4)], r.w[7 % (Raw8<DT>::kBytes / 4)]);
         }
         __syncthreads();
-        // The output matrix is dense, so its rows follow one another in memory: this row's elements
+        const int n_out = (int)out_cols, ng = (int)col_group;
+        if (ng == 1) {
+            // Single columns: one 32-bit word of the output per lane, so that a warp reads 32
+            // neighbouring entries of the keep list and writes 128 adjacent bytes per step.
+            const int n_cu_m1 = (int)J.n_cu - 1;
+            auto col = [&](int b) -> int { return min(max(__ldg(J.col_keep + b), 0), n_cu_m1); };
+            if (DT == MOSAIC_F32) {
+                const uint32_t* s32 = reinterpret_cast<const uint32_t*>(srow);
+                uint32_t* d32 = reinterpret_cast<uint32_t*>(dst);
+                for (int e = threadIdx.x; e < n_out; e += blockDim.x) __stcs(d32 + e, s32[col(e)]);
+            } else {
+                // the output matrix is dense: an odd row of odd width starts on the upper half of a word
+                const uint16_t* s16 = reinterpret_cast<const uint16_t*>(srow);
+                uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
+                const int head = (int)((a * out_cols) & 1);
+                const int pairs = (n_out - head) / 2;
+                uint32_t* d32 = reinterpret_cast<uint32_t*>(d16 + head);
+                for (int q = threadIdx.x; q < pairs; q += blockDim.x) {
+                    const int j0 = col(head + 2 * q), j1 = col(head + 2 * q + 1);
+                    __stcs(d32 + q, __byte_perm((uint32_t)s16[j0], (uint32_t)s16[j1], 0x5410));
+                }
+                if (threadIdx.x == 0 && head) d16[0] = s16[col(0)];
+                if (threadIdx.x == 32 % blockDim.x && head + 2 * pairs < n_out) d16[n_out - 1] = s16[col(n_out - 1)];
+            }
+            continue;
+        }
+        // Units of several columns that are not whole vectors.  This row's elements
         // [head, head + 8*body) start on a 16-byte boundary whatever out_cols is and go out as whole
         // vectors; the up to 7 elements before and after them are stored one by one.
-        const int n_out = (int)out_cols, ng = (int)col_group;
         const int head_full = (int)((kVec - (a * out_cols) % kVec) % kVec);
         const int head = head_full < n_out ? head_full : n_out;
         const int body = (n_out - head) / kVec;
         auto source_col = [&](int b) -> int {   // column of the staged row that output column b takes
-            const int64_t cu = clamp_unit((ng == 1) ? (int64_t)J.col_keep[b] : (int64_t)J.col_keep[b / ng], J.n_cu);
-            return (ng == 1) ? (int)cu : (int)cu * ng + b % ng;
+            return (int)clamp_unit((int64_t)J.col_keep[b / ng], J.n_cu) * ng + b % ng;
         };
         for (int v = threadIdx.x; v < body; v += blockDim.x) {
             Raw8<DT> r;
             const int b0 = head + v * kVec;
-            if (ng == 1) {
-                int j[kVec];
 #pragma unroll
-                for (int e = 0; e < kVec; ++e) j[e] = (int)clamp_unit((int64_t)J.col_keep[b0 + e], J.n_cu);
-#pragma unroll
-                for (int e = 0; e < kVec; ++e) r.set_scalar(e, srow, j[e]);
-            } else {
-#pragma unroll
-                for (int e = 0; e < kVec; ++e) r.set_scalar(e, srow, source_col(b0 + e));
-            }
+            for (int e = 0; e < kVec; ++e) r.set_scalar(e, srow, source_col(b0 + e));
             r.store(dst + (size_t)b0 * esz);
         }
         const int tail0 = head + body * kVec;
@@ -466,6 +482,10 @@ static bool compact_by_vectors(int64_t cols, int64_t col_group, int64_t col_unit
     return (col_group % kVec) == 0 || (col_group == 1 && col_units_keep == cols);
 }
 
+static size_t staged_row_bytes(int64_t cols, int dtype) {
+    return align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
+}
+
 static int check_compact_job(const void* W_in, int64_t rows, int64_t cols, int64_t ldw, int dtype, const int32_t* row_keep,
                              int64_t row_units_keep, int64_t row_group, const int32_t* col_keep, int64_t col_units_keep,
                              int64_t col_group, const void* W_out) {
@@ -485,7 +505,7 @@ static int check_compact_job(const void* W_in, int64_t rows, int64_t cols, int64
     if (a < b + out_span && b < a + in_span) return MOSAIC_ERR_ALIASING;
     // a source row that has to be staged must fit in shared memory (cols <= 51200 fp32)
     if (!compact_by_vectors(cols, col_group, col_units_keep) &&
-        align_up((size_t)((cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16) > 200 * 1024)
+        staged_row_bytes(cols, dtype) > 200 * 1024)
         return MOSAIC_ERR_INVALID_ARG;
     return MOSAIC_OK;
 }
@@ -503,7 +523,7 @@ static int launch_compact(const CompactJobList<NJ>& list, int64_t total_out_rows
     for (int i = 0; i < list.n; ++i) {
         const CompactJob& J = list.job[i];
         if (!compact_by_vectors(J.cols, J.col_group, J.out_cols / J.col_group)) {
-            const size_t need = align_up((size_t)((J.cols + kVec - 1) / kVec * kVec) * elem_size(dtype), 16);
+            const size_t need = staged_row_bytes(J.cols, dtype);
             if (need > smem) smem = need;
         }
     }
@@ -516,13 +536,15 @@ static int launch_compact(const CompactJobList<NJ>& list, int64_t total_out_rows
         return e == cudaSuccess ? 1 : -1;
     });
     if (opted < 0) return MOSAIC_ERR_CUDA;
-    // resident CTAs: bounded by the staging buffer (and by 2048 threads per SM)
-    int per_sm = smem == 0 ? 8 : (int)((200 * 1024) / (smem + 1024));
-    per_sm = per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm);
+    // Resident CTAs: bounded by the staging buffer and by 2048 threads per SM.  What has to be in
+    // flight to keep HBM busy is rows, not threads: short rows get CTAs of 128 threads, 16 per SM.
+    const int by_smem = smem == 0 ? 16 : (int)((200 * 1024) / (smem + 1024));
+    const int threads = by_smem > 8 ? 128 : 256;
+    int per_sm = by_smem < 1 ? 1 : (by_smem > 2048 / threads ? 2048 / threads : by_smem);
     int64_t grid = (int64_t)sm_count() * per_sm;
     if (grid > total_out_rows) grid = total_out_rows;
-    if (dtype == MOSAIC_BF16) compact_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, 256, smem, st>>>(list, total_out_rows);
-    else compact_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, 256, smem, st>>>(list, total_out_rows);
+    if (dtype == MOSAIC_BF16) compact_kernel<MOSAIC_BF16, NJ><<<(unsigned)grid, threads, smem, st>>>(list, total_out_rows);
+    else compact_kernel<MOSAIC_F32, NJ><<<(unsigned)grid, threads, smem, st>>>(list, total_out_rows);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }
@@ -655,17 +677,32 @@ extern "C" int mosaic_compact_batch(const mosaic_compact_job* jobs, int64_t n_jo
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     std::unique_ptr<CompactJobList<kStructBatch>> mem(new (std::nothrow) CompactJobList<kStructBatch>);
     if (!mem) return MOSAIC_ERR_INVALID_ARG;
-    for (int64_t i = 0; i < n_jobs; i += kStructBatch) {
-        mem->n = (int)(n_jobs - i < kStructBatch ? n_jobs - i : kStructBatch);
-        int64_t total = 0;
-        for (int m = 0; m < mem->n; ++m) {
-            const mosaic_compact_job& j = jobs[i + m];
-            mem->job[m] = make_compact_job(j.W_in, j.rows, j.cols, j.ldw, j.row_keep_units, j.row_units_keep, j.row_group,
-                                           j.col_keep_units, j.col_units_keep, j.col_group, j.W_out, total);
-            total += j.row_units_keep * j.row_group;
+    // One launch per class of staged row length (steps of 8 KB; class 0 = no staging), so that the
+    // shared memory of a CTA, and with it the number of rows in flight per SM, fits the rows it serves.
+    auto row_class = [&](const mosaic_compact_job& j) -> int {
+        if (compact_by_vectors(j.cols, j.col_group, j.col_units_keep)) return 0;
+        return (int)((staged_row_bytes(j.cols, dtype) + 8191) / 8192);
+    };
+    constexpr int kClasses = 200 * 1024 / 8192 + 1;
+    bool present[kClasses] = {};
+    for (int64_t i = 0; i < n_jobs; ++i) present[row_class(jobs[i])] = true;
+    for (int c = 0; c < kClasses; ++c) {
+        if (!present[c]) continue;
+        int64_t i = 0;
+        while (i < n_jobs) {
+            mem->n = 0;
+            int64_t total = 0;
+            for (; i < n_jobs && mem->n < kStructBatch; ++i) {
+                const mosaic_compact_job& j = jobs[i];
+                if (row_class(j) != c) continue;
+                mem->job[mem->n++] = make_compact_job(j.W_in, j.rows, j.cols, j.ldw, j.row_keep_units, j.row_units_keep, j.row_group,
+                                                      j.col_keep_units, j.col_units_keep, j.col_group, j.W_out, total);
+                total += j.row_units_keep * j.row_group;
+            }
+            if (mem->n == 0) break;
+            const int rc = launch_compact<kStructBatch>(*mem, total, dtype, st);
+            if (rc != MOSAIC_OK) return rc;
         }
-        const int rc = launch_compact<kStructBatch>(*mem, total, dtype, st);
-        if (rc != MOSAIC_OK) return rc;
     }
     return MOSAIC_OK;
 }
