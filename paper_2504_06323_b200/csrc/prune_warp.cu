@@ -21,16 +21,16 @@
 //   1. the warp's vectors arrive in the group's row buffer by cp.async;
 //   2. classification, two weights per integer subtract: (w | 0x8000) - A has bit 15 set iff the
 //      magnitude is >= A.  Weights under A_lo are pruned for sure, weights from A_lo + D up are
-//      kept for sure, the few per cent in between are the row's candidates;
+//      kept for sure, the few per cent in between are the row's candidates; the keep bits of the
+//      sure ones (candidates counted as kept) go to the row's keep bytes;
 //   3. the warp queues its candidates (their columns), forms their exact fp32 score keys from the
-//      row buffer and the norm table (again whenever it needs them: a queue of columns alone is a
-//      third the size), and adds them to the group's histogram of the window (up to 256 bins);
-//   4. (group barrier) every warp finds the bin that holds rank k; the keys of that bin are
-//      collected (group barrier) and ranked under (key, column), which is the oracle's total
-//      order, so ties need no special case;
-//   5. the warp zeroes its candidates at or below the threshold in the row buffer.  A zeroed weight
-//      has magnitude 0 < A_lo, so the store pass - which masks everything under A_lo - writes both
-//      the sure and the selected zeros and the keep bits from one classification.
+//      row buffer and the norm table, adds them to the group's histogram of the window (up to 256
+//      bins) and notes each one's bin beside its column;
+//   4. (group barrier) every warp finds the bin that holds rank k and walks its queue once more:
+//      a candidate of a lower bin loses its keep bit, the keys of the bin itself are collected
+//      (group barrier) and ranked under (key, column), which is the oracle's total order, so ties
+//      need no special case; those at or below the rank lose their keep bits too;
+//   5. the store pass writes each vector under its keep byte; the row buffer is never modified.
 // A row whose threshold falls outside the window, whose candidates overflow a queue, or whose bin
 // holds more than 32 keys, and every row of a job whose window is unusable (norms that are not
 // finite and >= 0, a threshold at zero or at overflow) takes slow_row(): a radix select by the
@@ -50,7 +50,7 @@ constexpr uint32_t kWOverflow = 0xFFFFFFFFu;   // a warp's "my queue overflowed"
 struct WarpLayout {
     int nvec, nwords, qcap;   // qcap: candidates one warp may queue
     uint32_t off_alo, off_nrm, off_misc, off_group0, per_group;                      // bytes
-    uint32_t o_queue, per_queue, o_qcol, o_hist, o_mbytes, o_bkey, o_bcol, o_ctl;   // bytes inside a group's block
+    uint32_t o_queue, per_queue, o_qcol, o_qbin, per_qbin, o_hist, o_mbytes, o_bkey, o_bcol, o_ctl;   // bytes inside a group's block
 };
 __host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
     WarpLayout L;
@@ -68,6 +68,9 @@ __host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
     L.o_qcol = 0u;
     L.per_queue = (uint32_t)L.qcap * 2u;
     w += L.per_queue * (uint32_t)G;
+    L.o_qbin = w;                                      // per warp: the window bin of each queued candidate (1 B each)
+    L.per_qbin = (uint32_t)L.qcap;
+    w += L.per_qbin * (uint32_t)G;
     w = (w + 15u) & ~15u;
     L.o_hist = w;    w += sets * kWBins * 4u;
     L.o_mbytes = w;  w += ((uint32_t)L.nwords * 4u + 15u) & ~15u;
@@ -315,10 +318,12 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                                                                        // [17] samples taken, [32..63] samples by distance from the centre
     unsigned char* mine = smem + L.off_group0 + (size_t)gid * L.per_group;
     uint4* row = reinterpret_cast<uint4*>(mine);
-    uint16_t* row16 = reinterpret_cast<uint16_t*>(mine);
+    const uint16_t* row16 = reinterpret_cast<const uint16_t*>(mine);
     uint16_t* qcol = reinterpret_cast<uint16_t*>(mine + L.o_queue + (size_t)sub * L.per_queue);
+    uint8_t* qbin = mine + L.o_qbin + (size_t)sub * L.per_qbin;
     uint32_t* hist0 = reinterpret_cast<uint32_t*>(mine + L.o_hist);
     uint8_t* mbytes = mine + L.o_mbytes;
+    uint32_t* mwords = reinterpret_cast<uint32_t*>(mine + L.o_mbytes);
     uint32_t* bkey0 = reinterpret_cast<uint32_t*>(mine + L.o_bkey);
     uint32_t* bcol0 = reinterpret_cast<uint32_t*>(mine + L.o_bcol);
     uint32_t* ctl = reinterpret_cast<uint32_t*>(mine + L.o_ctl);
@@ -529,6 +534,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                         const uint32_t above = flags8(t0 - DD, t1 - DD, t2 - DD, t3 - DD);
                         candw[v >> 2] |= (keepf & ~above) >> (2 * (v & 3));
                         below += 8u - (uint32_t)__popc(keepf);
+                        mbytes[vec] = (uint8_t)byte_of_flags(keepf);   // candidates count as kept until the threshold says otherwise
                     }
                 }
                 // ---- queue the warp's candidates (their columns)
@@ -567,6 +573,8 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                                 const uint32_t d = key - lo;   // key < lo wraps to >= 2^31 (key, lo < 2^31)
                                 if (d < width) atomicAdd(&hist[d >> shift], 1u);
                                 else below += d >> 31;
+                                const uint32_t b = d >> shift;   // bin of the window; 255 also stands for everything above it
+                                qbin[i] = (uint8_t)((d >> 31) ? 0u : (b < 255u ? b : 255u));
                             }
                         }
                     }
@@ -590,13 +598,24 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 uint32_t bin = 0u, r_bin = 0u, n_bin = 0u;
                 if (ok) ok = warp_find_bin<G == 1>(hist, below, uk, lane, &bin, &r_bin, &n_bin) && n_bin <= (uint32_t)kWBinList;
                 if (ok) {
+                    // The queue again, by bin code: a candidate of a lower bin is pruned (its keep bit
+                    // cleared); one whose code matches the bin goes on the bin list after its exact
+                    // key confirms it (code 255 also covers keys above the window).
+                    auto prune_col = [&](uint32_t col) { atomicAnd(&mwords[col >> 5], ~(1u << (col & 31u))); };
                     uint32_t nl = 0u;
                     for (uint32_t base = 0u; base < qn; base += 32u) {
                         const uint32_t i = base + lane;
-                        const uint32_t col = i < qn ? (uint32_t)qcol[i] : (uint32_t)(gl * 8);
-                        const uint32_t key =
-                            __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
-                        const bool in = i < qn && ((key - lo) >> shift) == bin;
+                        const uint32_t code = i < qn ? (uint32_t)qbin[i] : 0xFFFFu;
+                        const uint32_t col = i < qn ? (uint32_t)qcol[i] : 0u;
+                        if (code < bin) prune_col(col);
+                        bool in = false;
+                        uint32_t key = 0u;
+                        if (code == bin) {
+                            key = __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
+                            const uint32_t d = key - lo;
+                            if (d >> 31) prune_col(col);   // below the window (cannot happen with exact thresholds)
+                            else in = d < width && (d >> shift) == bin;
+                        }
                         const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
                         if (G > 1 && m != 0u) {   // the group's list is filled by all its warps: take a range of it
                             uint32_t first = 0u;
@@ -618,34 +637,27 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                         const uint32_t ok2 = __shfl_sync(0xFFFFFFFFu, mk, (int)jj), oc = __shfl_sync(0xFFFFFFFFu, mc, (int)jj);
                         less += (ok2 < mk || (ok2 == mk && oc < mc)) ? 1u : 0u;
                     }
-                    const unsigned sel = __ballot_sync(0xFFFFFFFFu, have && less + 1u == r_bin);
-                    const int src_l = __ffs(sel) - 1;   // exactly one entry holds rank r_bin: the pairs are distinct
-                    const uint32_t T = __shfl_sync(0xFFFFFFFFu, mk, src_l), colT = __shfl_sync(0xFFFFFFFFu, mc, src_l);
                     if (G > 1 && sub == 0) {   // every warp has read this row's histogram: clean for the row after next
                         warp_clear_hist(hist, lane);
                         if (lane == 0) *fill = 0u;
                     }
-                    // ---- zero the warp's selected candidates in the row buffer
-                    for (uint32_t i = lane; i < qn; i += 32u) {
-                        const uint32_t col = (uint32_t)qcol[i];
-                        const uint32_t key =
-                            __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
-                        if (key < T || (key == T && col <= colT)) row16[col] = (uint16_t)0;
-                    }
+                    // ---- the entries of the bin at or below rank r_bin are pruned (a warp clears the bits of its own columns only:
+                    //      the other warps of the group may already be at their next row)
+                    if (have && less < r_bin && (G == 1 || (int)((mc >> 3) % (uint32_t)TG) / 32 == sub)) prune_col(mc);
                     __syncwarp();
-                    // ---- store: everything under A_lo (the sure ones and the zeroed candidates) becomes +0
+                    // ---- store: each weight under its keep bit
+                    if (out_row != nullptr) {
 #pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        const int vec = v * TG + gl;
-                        if (FULL || vec < nvec) {
-                            const uint4 rr = row[vec], a = alo[vec];
-                            const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
-                                           t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
-                            if (out_row != nullptr)
+                        for (int v = 0; v < V; ++v) {
+                            const int vec = v * TG + gl;
+                            if (FULL || vec < nvec) {
+                                const uint4 rr = row[vec];
+                                const uint32_t kb = (uint32_t)mbytes[vec];
+                                // kb * (2^(15-2i) + 2^(30-2i)) has bit 2i of kb on bit 15 and bit 2i+1 on bit 31
                                 st_stream16(out_row + (int64_t)vec * kVec,
-                                            make_uint4(rr.x & lane_mask(t0), rr.y & lane_mask(t1), rr.z & lane_mask(t2),
-                                                       rr.w & lane_mask(t3)));
-                            mbytes[vec] = (uint8_t)byte_of_flags(flags8(t0, t1, t2, t3));
+                                            make_uint4(rr.x & lane_mask(kb * 0x40008000u), rr.y & lane_mask(kb * 0x10002000u),
+                                                       rr.z & lane_mask(kb * 0x04000800u), rr.w & lane_mask(kb * 0x01000200u)));
+                            }
                         }
                     }
                     done = true;
