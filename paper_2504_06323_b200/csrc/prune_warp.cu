@@ -547,9 +547,20 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 if (fits) {
                     uint32_t off = incl - cnt;
 #pragma unroll
-                    for (int w = 0; w < NW; ++w)
-                        for (uint32_t c = candw[w]; c != 0u; c &= c - 1u)
-                            qcol[off++] = (uint16_t)(w * 32 * TG + gl * 8 + flagtab[__ffs(c) - 1]);
+                    for (int w = 0; w < NW; ++w) {
+                        const uint32_t col0 = (uint32_t)(w * 32 * TG + gl * 8);
+                        for (uint32_t c = candw[w]; c != 0u;) {   // two per turn: both table reads in flight together
+                            const int p0 = __ffs(c) - 1;
+                            c &= c - 1u;
+                            const bool two = c != 0u;
+                            const int p1 = two ? __ffs(c) - 1 : p0;
+                            c &= c - 1u;
+                            const uint32_t f0 = flagtab[p0], f1 = flagtab[p1];
+                            qcol[off] = (uint16_t)(col0 + f0);
+                            if (two) qcol[off + 1u] = (uint16_t)(col0 + f1);
+                            off += two ? 2u : 1u;
+                        }
+                    }
                     __syncwarp();
                     // ---- exact keys of the candidates, four rounds of 32 at a time
                     for (uint32_t base = lane; base < qn; base += 128u) {
@@ -603,31 +614,41 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                     // key confirms it (code 255 also covers keys above the window).
                     auto prune_col = [&](uint32_t col) { atomicAnd(&mwords[col >> 5], ~(1u << (col & 31u))); };
                     uint32_t nl = 0u;
-                    for (uint32_t base = 0u; base < qn; base += 32u) {
-                        const uint32_t i = base + lane;
-                        const uint32_t code = i < qn ? (uint32_t)qbin[i] : 0xFFFFu;
-                        const uint32_t col = i < qn ? (uint32_t)qcol[i] : 0u;
-                        if (code < bin) prune_col(col);
-                        bool in = false;
-                        uint32_t key = 0u;
-                        if (code == bin) {
-                            key = __float_as_uint(__fmul_rn(nrm[col], __uint_as_float(((uint32_t)row16[col] & 0x7FFFu) << 16)));
-                            const uint32_t d = key - lo;
-                            if (d >> 31) prune_col(col);   // below the window (cannot happen with exact thresholds)
-                            else in = d < width && (d >> shift) == bin;
+                    for (uint32_t base = 0u; base < qn; base += 128u) {   // four rounds of 32 per turn
+                        uint32_t code[4], col[4];
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const uint32_t i = base + 32u * g + lane;
+                            code[g] = i < qn ? (uint32_t)qbin[i] : 0xFFFFu;
+                            col[g] = i < qn ? (uint32_t)qcol[i] : 0u;
                         }
-                        const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
-                        if (G > 1 && m != 0u) {   // the group's list is filled by all its warps: take a range of it
-                            uint32_t first = 0u;
-                            if (lane == 0) first = atomicAdd(fill, (uint32_t)__popc(m));
-                            nl = __shfl_sync(0xFFFFFFFFu, first, 0);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g)
+                            if (code[g] < bin) prune_col(col[g]);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            bool in = false;
+                            uint32_t key = 0u;
+                            if (code[g] == bin) {
+                                key = __float_as_uint(__fmul_rn(nrm[col[g]], __uint_as_float(((uint32_t)row16[col[g]] & 0x7FFFu) << 16)));
+                                const uint32_t d = key - lo;
+                                if (d >> 31) prune_col(col[g]);   // below the window (cannot happen with exact thresholds)
+                                else in = d < width && (d >> shift) == bin;
+                            }
+                            const unsigned m = __ballot_sync(0xFFFFFFFFu, in);
+                            if (m == 0u) continue;
+                            if (G > 1) {   // the group's list is filled by all its warps: take a range of it
+                                uint32_t first = 0u;
+                                if (lane == 0) first = atomicAdd(fill, (uint32_t)__popc(m));
+                                nl = __shfl_sync(0xFFFFFFFFu, first, 0);
+                            }
+                            if (in) {
+                                const uint32_t pos = nl + (uint32_t)__popc(m & ((1u << lane) - 1u));
+                                bkey[pos] = key;
+                                bcol[pos] = col[g];
+                            }
+                            if (G == 1) nl += (uint32_t)__popc(m);
                         }
-                        if (in) {
-                            const uint32_t pos = nl + (uint32_t)__popc(m & ((1u << lane) - 1u));
-                            bkey[pos] = key;
-                            bcol[pos] = col;
-                        }
-                        if (G == 1) nl += (uint32_t)__popc(m);
                     }
                     group_barrier<G>(gid);
                     const bool have = (uint32_t)lane < n_bin;
