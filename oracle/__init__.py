@@ -211,6 +211,35 @@ def unit_scores_certify(W: np.ndarray, norms, row_group: int = 1, col_group: int
     return r_ok.astype(bool), c_ok.astype(bool)
 
 
+def gram(X: np.ndarray, G: np.ndarray | None = None, dtype=None, with_abs: bool = False):
+    """G[j,l] += sum_t X[t,j] X[t,l] in fp64, t in order (second moments of a projection's input;
+    the back-end's layer Hessian is 2/T times it).  with_abs: also sum_t |X[t,j]| |X[t,l]|."""
+    code = _code(X, dtype)
+    tokens, cols = X.shape
+    G = np.zeros((cols, cols), dtype=np.float64) if G is None else G
+    assert G.dtype == np.float64 and G.shape == (cols, cols) and G.flags.c_contiguous
+    Ga = np.zeros((cols, cols), dtype=np.float64) if with_abs else None
+    lib().oracle_gram(_p(X), _i64(tokens), _i64(cols), _i64(_ld(X)), code, _p(G), _p(Ga) if with_abs else None)
+    return (G, Ga) if with_abs else G
+
+
+def gram_pairs(X: np.ndarray, js, ls, dtype=None):
+    """(sum_t X[t,j] X[t,l], sum_t |X[t,j]| |X[t,l]|) for the listed (j, l) pairs, fp64."""
+    code = _code(X, dtype)
+    js = np.ascontiguousarray(js, dtype=np.int64)
+    ls = np.ascontiguousarray(ls, dtype=np.int64)
+    assert js.shape == ls.shape and js.ndim == 1
+    out = np.zeros(js.shape[0], dtype=np.float64)
+    out_abs = np.zeros(js.shape[0], dtype=np.float64)
+    lib().oracle_gram_pairs(_p(X), _i64(X.shape[0]), _i64(_ld(X)), code, _i64(js.shape[0]), _p(js), _p(ls), _p(out), _p(out_abs))
+    return out, out_abs
+
+
+def hessian(X: np.ndarray, dtype=None) -> np.ndarray:
+    """Layer Hessian of the inverse-Hessian back-end: (2 / T) * sum_t x_t x_t^T, fp64."""
+    return gram(X, None, dtype) * (2.0 / X.shape[0])
+
+
 def rank_units(scores: np.ndarray, keep: int) -> np.ndarray:
     """Ascending list of the `keep` units that survive removal of the lowest-scored ones."""
     scores = np.ascontiguousarray(scores, np.float32)

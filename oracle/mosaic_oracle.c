@@ -562,6 +562,55 @@ void oracle_compact(const void *W, int64_t ldw, int dtype, const int32_t *row_ke
     }
 }
 
+/*
+ * Calibration-side companion of the path (Section 4.1.3, "Calibration"; Section 4.1.2: the
+ * pruning back-end ranks weights with the inverse Hessian): the second-moment matrix of a
+ * projection's input activations,
+ *     G[j][l] += sum_t X[t][j] * X[t][l],
+ * every product and sum in fp64, t in order.  The layer Hessian of that back-end is
+ * H = (2 / T) * G over all T calibration tokens (the published definition 2 X X^T averaged over
+ * the samples); its diagonal G[j][j] is the squared norm of Eq. 5.  G_abs (optional) receives
+ * sum_t |X[t][j]| * |X[t][l]|, the scale an fp32 accumulation's error is bounded against.
+ */
+void oracle_gram(const void *X, int64_t tokens, int64_t cols, int64_t ldx, int dtype,
+                 double *G, double *G_abs)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t j = 0; j < cols; ++j) {
+        for (int64_t l = 0; l < cols; ++l) {
+            double s = 0.0, a = 0.0;
+            for (int64_t t = 0; t < tokens; ++t) {
+                const double xj = (double)load_elem(X, t * ldx + j, dtype);
+                const double xl = (double)load_elem(X, t * ldx + l, dtype);
+                s += xj * xl;
+                a += fabs(xj) * fabs(xl);
+            }
+            G[j * cols + l] += s;
+            if (G_abs)
+                G_abs[j * cols + l] += a;
+        }
+    }
+}
+
+/* The same sums for a list of (j, l) pairs only: out[q] = sum_t X[t][js[q]] * X[t][ls[q]]. */
+void oracle_gram_pairs(const void *X, int64_t tokens, int64_t ldx, int dtype, int64_t n_pairs,
+                       const int64_t *js, const int64_t *ls, double *out, double *out_abs)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t q = 0; q < n_pairs; ++q) {
+        double s = 0.0, a = 0.0;
+        for (int64_t t = 0; t < tokens; ++t) {
+            const double xj = (double)load_elem(X, t * ldx + js[q], dtype);
+            const double xl = (double)load_elem(X, t * ldx + ls[q], dtype);
+            s += xj * xl;
+            a += fabs(xj) * fabs(xl);
+        }
+        out[q] = s;
+        if (out_abs)
+            out_abs[q] = a;
+    }
+}
+
 /* Thread count of the parallel loops above (timing only: no result depends on it). */
 void oracle_set_num_threads(int n)
 {

@@ -590,3 +590,88 @@ def test_redistribution_changes_nothing_without_a_clamp_and_flags_the_impossible
     s, k, infeasible = oracle.allocate_sparsity([0, 50, 100], [100] * 3, [10] * 3, 1, 3, 0.5, 0.5, oracle.MODE_REDISTRIBUTE)
     np.testing.assert_allclose(s, [0.9, 0.55, 0.05], atol=1e-15)
     assert not infeasible and list(k) == [9, 5, 0]
+
+
+# ----------------------------------------------------------------- second moments / Hessian (calibration side, Section 4.1.3)
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_gram_exact_rational_brute_force(dtype):
+    """Every entry against sum_t x_tj x_tl in exact rational arithmetic (the fp64 sums are exact
+    here: a handful of products of 8- or 24-bit mantissas with close exponents)."""
+    rng = np.random.default_rng(11)
+    X = (rng.integers(-8, 9, size=(7, 5)) * 0.25).astype(np.float32)
+    Xd = bf16_bits(X) if dtype == "bf16" else X
+    G, Ga = oracle.gram(Xd, None, dtype, with_abs=True)
+    Xv = as_f32(Xd, dtype)
+    for j in range(5):
+        for l in range(5):
+            exact = sum(Fraction(float(Xv[t, j])) * Fraction(float(Xv[t, l])) for t in range(7))
+            exact_abs = sum(abs(Fraction(float(Xv[t, j])) * Fraction(float(Xv[t, l]))) for t in range(7))
+            assert Fraction(float(G[j, l])) == exact, (j, l)
+            assert Fraction(float(Ga[j, l])) == exact_abs, (j, l)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_gram_closed_forms(dtype):
+    # constant columns c_j: G[j,l] = T c_j c_l (all values powers of two: exact)
+    T, c = 64, np.array([1.0, -2.0, 0.5, 4.0, 0.0, -0.25], np.float32)
+    X = np.tile(c, (T, 1))
+    Xd = bf16_bits(X) if dtype == "bf16" else X
+    G = oracle.gram(Xd, None, dtype)
+    assert np.array_equal(G, T * np.outer(c, c).astype(np.float64))
+    # one non-zero per token (token t excites channel t mod cols with value v_t): G is diagonal
+    cols = 5
+    v = (np.arange(1, 21) * 0.5).astype(np.float32)
+    X = np.zeros((20, cols), np.float32)
+    X[np.arange(20), np.arange(20) % cols] = v
+    Xd = bf16_bits(X) if dtype == "bf16" else X
+    G = oracle.gram(Xd, None, dtype)
+    expect = np.zeros((cols, cols))
+    for t in range(20):
+        expect[t % cols, t % cols] += float(v[t]) ** 2
+    assert np.array_equal(G, expect)
+    # the back-end's Hessian is 2/T times it
+    assert np.array_equal(oracle.hessian(Xd, dtype), expect * (2.0 / 20))
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_gram_against_library_matmul_and_invariants(dtype):
+    rng = np.random.default_rng(12)
+    T, cols = 300, 24
+    X = rng.standard_normal((T, cols)).astype(np.float32)
+    X[:, 3] *= 50.0                                   # an outlier channel
+    Xd = bf16_bits(X) if dtype == "bf16" else X
+    Xv = as_f32(Xd, dtype).astype(np.float64)
+    G, Ga = oracle.gram(Xd, None, dtype, with_abs=True)
+    ref = Xv.T @ Xv                                    # the textbook definition through BLAS (another summation order)
+    assert np.allclose(G, ref, rtol=0, atol=1e-12 * np.abs(Xv).T @ np.abs(Xv))
+    assert np.array_equal(G, G.T)                      # symmetric, bit for bit (products commute)
+    assert np.linalg.eigvalsh(G).min() > -1e-9 * np.trace(G)          # positive semi-definite
+    assert (Ga >= np.abs(G)).all() and np.allclose(Ga, np.abs(Xv).T @ np.abs(Xv), rtol=1e-12)
+    # the diagonal is the squared norm of Eq. 5
+    assert np.allclose(np.diag(G), oracle.act_sumsq(Xd, None, dtype), rtol=1e-14)
+    # scaling the activations by 2 scales every second moment by exactly 4
+    X2 = (2.0 * as_f32(Xd, dtype)).astype(np.float32)
+    X2d = bf16_bits(X2) if dtype == "bf16" else X2
+    assert np.array_equal(oracle.gram(X2d, None, dtype), 4.0 * G)
+    # a transposed or mis-strided read shows on a view with a leading dimension larger than cols
+    wide = np.zeros((T, cols + 8), Xd.dtype)
+    wide[:, :cols] = Xd
+    wide[:, cols:] = Xd[:, :8]                         # junk beyond the columns
+    assert np.array_equal(oracle.gram(wide[:, :cols], None, dtype), G)
+
+
+@pytest.mark.parametrize("dtype", DTYPES)
+def test_gram_accumulates_over_token_chunks_and_pairs_agree(dtype):
+    rng = np.random.default_rng(13)
+    T, cols = 257, 16
+    X = rng.standard_normal((T, cols)).astype(np.float32)
+    Xd = bf16_bits(X) if dtype == "bf16" else X
+    G = oracle.gram(Xd, None, dtype)
+    acc = np.zeros((cols, cols))
+    for a, b in [(0, 100), (100, 101), (101, 257)]:
+        oracle.gram(np.ascontiguousarray(Xd[a:b]), acc, dtype)
+    assert np.allclose(acc, G, rtol=0, atol=1e-13 * np.abs(G).max())
+    js, ls = np.array([0, 3, 15, 7, 7]), np.array([0, 9, 2, 7, 8])
+    out, out_abs = oracle.gram_pairs(Xd, js, ls, dtype)
+    assert np.array_equal(out, G[js, ls])
+    assert (out_abs >= np.abs(out)).all()
