@@ -51,7 +51,7 @@ typedef enum mosaic_status {
     MOSAIC_ERR_CUDA = -7,
     MOSAIC_ERR_NONFINITE = -8,   /* reserved */
     MOSAIC_ERR_INFEASIBLE = -9,  /* allocation had to clamp a target; outputs are still written */
-    MOSAIC_ERR_TIMEOUT = -10     /* reserved */
+    MOSAIC_ERR_TIMEOUT = -10     /* a bounded device-side wait ran out (reported through a status word) */
 } mosaic_status;
 
 typedef enum mosaic_dtype { MOSAIC_F32 = 0, MOSAIC_BF16 = 1 } mosaic_dtype;
@@ -387,6 +387,34 @@ typedef struct mosaic_compact_job {
     void *W_out;
 } mosaic_compact_job;
 int mosaic_compact_batch(const mosaic_compact_job *jobs, int64_t n_jobs, int dtype, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * mosaic_gram_accumulate - second moments of a projection's input activations,
+ * the calibration-side companion of mosaic_act_norms (Section 4.1.3: the same
+ * calibration samples also give the pruning back-end its Hessian; Section 4.1.2:
+ * that back-end ranks and updates weights with the inverse Hessian):
+ *     G[j,l] += sum_t X[t,j] * X[t,l]        for all 0 <= j, l < cols.
+ * The layer Hessian of the back-end is H = (2/T) * G over all T calibration
+ * tokens; diag(G) is the squared norm of Eq. 5.  Call once per chunk of tokens.
+ *
+ *   X          device, [tokens, cols] row-major, ld = ldx, MOSAIC_BF16 only
+ *              (bf16 products are exact in fp32; MOSAIC_F32 -> MOSAIC_ERR_BAD_DTYPE).
+ *              cols % 8 == 0, tokens < 2^31 - 64.  tokens = 0 is legal.
+ *   G          device, fp32 [cols, cols] row-major, ld = ldg (ldg % 4 == 0,
+ *              16-byte aligned), in-out, caller-owned; both triangles are written.
+ *              Must not overlap X (MOSAIC_ERR_ALIASING).
+ *   flags      0 or MOSAIC_RESET_ACCUM (treat G as zero on entry)
+ *   status_dev device, one int, or NULL.  Set to 0 when the call is enqueued and to
+ *              1 by the kernel if one of its bounded waits ran out (G is then
+ *              undefined); read it after synchronising the stream.
+ *
+ * Arithmetic: products exact, sums in fp32 on the tensor cores in token order
+ * within a chunk, one fp32 add per chunk into G.  The result is deterministic
+ * (independent of the grid) and differs from the exact sum by at most
+ * (tokens/16 + 2) * 2^-24 * sum_t |X[t,j]| |X[t,l]| per call.
+ * ------------------------------------------------------------------------- */
+int mosaic_gram_accumulate(const void *X, int64_t tokens, int64_t cols, int64_t ldx, int dtype, float *G,
+                           int64_t ldg, int flags, int *status_dev, void *stream);
 
 #ifdef __cplusplus
 }

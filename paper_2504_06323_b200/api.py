@@ -40,6 +40,7 @@ SYMBOLS = (
     "mosaic_rank_units", "mosaic_sum_unit_scores",
     "mosaic_unit_scores_batch_workspace_bytes", "mosaic_unit_scores_batch", "mosaic_add_unit_scores_batch",
     "mosaic_rank_units_batch", "mosaic_compact_batch",
+    "mosaic_gram_accumulate",
 )
 
 
@@ -65,6 +66,8 @@ def lib() -> C.CDLL:
         L.mosaic_version.restype = ci
         L.mosaic_status_string.restype = C.c_char_p
         L.mosaic_status_string.argtypes = [ci]
+        L.mosaic_gram_accumulate.restype = ci
+        L.mosaic_gram_accumulate.argtypes = [vp, i64, i64, i64, ci, vp, i64, ci, vp, vp]
         L.mosaic_act_norms_workspace_bytes.restype = sz
         L.mosaic_act_norms_workspace_bytes.argtypes = [i64, i64]
         L.mosaic_act_norms.restype = ci
@@ -210,6 +213,21 @@ def mosaic_act_norms(X: torch.Tensor, sumsq_accum: torch.Tensor, norms_out: torc
     wp, wn = _ws(ws, X.device).get(L.mosaic_act_norms_workspace_bytes(tokens, cols))
     _check(L.mosaic_act_norms(xp, tokens, cols, ldx, _dtype_code(X), sumsq_accum.data_ptr(), _ptr(norms_out),
                               int(flags), wp, wn, _stream(stream)), "mosaic_act_norms")
+
+
+def mosaic_gram_accumulate(X: torch.Tensor, G: torch.Tensor, flags: int = 0, status: torch.Tensor | None = None,
+                           stream=None) -> None:
+    """G[j,l] += sum_t X[t,j] X[t,l] (fp32, both triangles): the second moments of a projection's
+    input, from which the inverse-Hessian back-end forms H = (2/T) G.  `status` (one int32 on the
+    device) reads 1 after synchronisation if a bounded wait of the kernel ran out."""
+    xp, tokens, cols, ldx = _mat(X, "X")
+    _dev(G, "G", torch.float32)
+    if G.dim() != 2 or tuple(G.shape) != (cols, cols) or G.stride(1) != 1:
+        raise ValueError("G must be a [cols, cols] fp32 matrix with unit column stride")
+    if status is not None:
+        _dev(status, "status", torch.int32)
+    _check(lib().mosaic_gram_accumulate(xp, tokens, cols, ldx, _dtype_code(X), G.data_ptr(), G.stride(0), int(flags),
+                                        _ptr(status), _stream(stream)), "mosaic_gram_accumulate")
 
 
 def mosaic_score(W: torch.Tensor, norms: torch.Tensor, score_out: torch.Tensor, stream=None) -> None:

@@ -1,0 +1,391 @@
+// mosaic_gram_accumulate: G += X^T X for one chunk of calibration tokens (bf16 activations, fp32
+// accumulation) - the second-moment matrix from which the inverse-Hessian back-end of Section
+// 4.1.2 forms its layer Hessian H = (2/T) G with the calibration samples of Section 4.1.3.  Its
+// diagonal is the squared norm of Eq. 5.
+//
+// A dense contraction over the token dimension, so it runs on the tensor cores:
+//   * G is cut into 256 x 256 blocks; only blocks on or above the diagonal are computed, the
+//     mirror image of an off-diagonal block is written by the same epilogue;
+//   * one persistent CTA per SM walks its blocks.  Per block the 512 columns of tensor memory
+//     hold the 256 x 256 fp32 accumulator as two 128-row halves;
+//   * both operands are column blocks of X, read straight from the row-major [tokens, cols]
+//     tensor by TMA in boxes of 64 columns x 64 tokens with the 128-byte swizzle.  In shared
+//     memory the columns of a token lie contiguous, i.e. both operands are "MN-major", which
+//     tcgen05.mma takes through its instruction descriptor - X is never transposed;
+//   * warp 0 issues the TMA loads of a 3-stage ring, one thread of warp 1 issues the MMAs (eight
+//     128 x 256 x 16 per stage) and commits each stage back to the loader, warps 2..5 drain the
+//     accumulator with tcgen05.ld once the block's last MMA has completed.  On a diagonal block the
+//     two operands are the same columns: they are loaded once.
+// A block is accumulated by one CTA in token order, so results do not depend on the grid.
+// Every wait on an mbarrier is bounded; a wait that runs out sets the kernel's error word, all
+// roles leave their loops, loads in flight are awaited (bounded), tensor memory is freed.
+#include <cuda.h>   // CUtensorMap and its enums; the encoder itself is looked up at run time
+
+#include "common.cuh"
+
+namespace mosaic {
+namespace {
+
+constexpr int kGBlk = 256;                                               // block edge
+constexpr int kGTok = 64;                                                // tokens per stage
+constexpr int kGStages = 3;
+constexpr int kGBoxCols = 64;                                            // 64 bf16 = one 128-byte swizzle row
+constexpr uint32_t kGBoxBytes = kGBoxCols * kGTok * 2;                   // 8 KB
+constexpr uint32_t kGOperandBytes = (kGBlk / kGBoxCols) * kGBoxBytes;    // 256 columns x 64 tokens = 32 KB
+constexpr uint32_t kGStageBytes = 2 * kGOperandBytes;                    // A block, then B block
+constexpr int kGThreads = 192;
+constexpr uint32_t kGTmemCols = 512;
+constexpr size_t kGSmemBytes = (size_t)kGStages * kGStageBytes + 1024 /* alignment */ + 256 /* barriers */;
+constexpr long long kGWaitCycles = 4000000000ll;                         // about two seconds
+
+// Instruction descriptor of tcgen05.mma kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16
+// (bits 7-9 and 10-12 = 1), A and B MN-major (bits 15, 16), N / 8 at bit 17, M / 16 at bit 24.
+constexpr uint32_t kGInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (1u << 16) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
+// Waits for the phase of the given parity to complete.  False if it gave up: after kGWaitCycles
+// (then it raises *err) or because another role raised *err.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err) {
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*err != 0) return false;
+        if (clock64() - t0 > kGWaitCycles) {
+            *err = 1;
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_box(void* dst, const CUtensorMap* map, uint64_t* bar, int col, int token) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+                     smem_u32(dst)),
+                 "l"(map), "r"(smem_u32(bar)), "r"(col), "r"(token)
+                 : "memory");
+}
+
+// Shared-memory operand descriptor, MN-major with the 128-byte swizzle: 64 columns of a token are
+// contiguous (one swizzle row), the rows of 8 consecutive tokens lie 128 bytes apart, groups of 8
+// tokens 1024 bytes apart (stride offset), the next 64 columns one TMA box further (leading offset).
+__device__ __forceinline__ uint64_t operand_desc(uint32_t smem_addr) {
+    uint64_t d = (uint64_t)((smem_addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((kGBoxBytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;   // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;   // 128-byte swizzle
+    return d;
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t"
+        "}"
+        :
+        : "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(kGInstrDesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+// The barrier gets one arrival when every MMA issued so far by this thread has completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 32 consecutive accumulator columns of this thread's lane of tensor memory.
+__device__ __forceinline__ void tmem_load32(uint32_t addr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(addr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Block (bi, bj), bi <= bj, number `tile` in the row-by-row list of the blocks on or above the diagonal.
+__device__ __forceinline__ void block_of_tile(int tile, int n_blk, int* bi, int* bj) {
+    int i = 0, rem = tile;
+    while (rem >= n_blk - i) {
+        rem -= n_blk - i;
+        ++i;
+    }
+    *bi = i;
+    *bj = i + rem;
+}
+
+__global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constant__ CUtensorMap x_map, float* __restrict__ G, int64_t ldg,
+                                                            int cols, int tokens, int n_blk, int n_tiles, int reset, int* status) {
+    extern __shared__ unsigned char gram_smem_raw[];
+    unsigned char* stages = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(gram_smem_raw) + 1023u) & ~(uintptr_t)1023u);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(stages + (size_t)kGStages * kGStageBytes);
+    uint64_t* full = bars;                    // [kGStages] loads of a stage have landed
+    uint64_t* empty = bars + kGStages;        // [kGStages] the MMAs reading a stage have completed
+    uint64_t* acc_full = bars + 2 * kGStages;       // the block's accumulator is complete
+    uint64_t* acc_empty = bars + 2 * kGStages + 1;  // the epilogue has read it
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kGStages + 2);
+    volatile int* err = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kGStages; ++s) {
+            mbar_init(&full[s], 1u);
+            mbar_init(&empty[s], 1u);
+        }
+        mbar_init(acc_full, 1u);
+        mbar_init(acc_empty, 4u);   // one arrival per epilogue warp
+        *err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kGTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const int nk = (tokens + kGTok - 1) / kGTok;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ loader
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                int bi, bj;
+                block_of_tile(tile, n_blk, &bi, &bj);
+                for (int k = 0; k < nk; ++k, ++it) {
+                    const uint32_t s = it % kGStages, ph = (it / kGStages) & 1u;
+                    if (!mbar_wait(&empty[s], ph ^ 1u, err)) {
+                        ok = false;
+                        break;
+                    }
+                    unsigned char* st = stages + (size_t)s * kGStageBytes;
+                    mbar_expect_tx(&full[s], bi == bj ? kGOperandBytes : kGStageBytes);
+#pragma unroll
+                    for (int b = 0; b < kGBlk / kGBoxCols; ++b)
+                        tma_load_box(st + kGOperandBytes + (size_t)b * kGBoxBytes, &x_map, &full[s], bj * kGBlk + b * kGBoxCols, k * kGTok);
+                    if (bi != bj) {
+#pragma unroll
+                        for (int b = 0; b < kGBlk / kGBoxCols; ++b)
+                            tma_load_box(st + (size_t)b * kGBoxBytes, &x_map, &full[s], bi * kGBlk + b * kGBoxCols, k * kGTok);
+                    }
+                }
+            }
+            if (!ok) {
+                // gave up: let the loads already issued land before the CTA leaves (bounded)
+                for (uint32_t back = 1; back <= (uint32_t)kGStages && back <= it; ++back) {
+                    const uint32_t j = it - back, s = j % kGStages, ph = (j / kGStages) & 1u;
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&full[s], ph) && clock64() - t0 < kGWaitCycles) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            uint32_t it = 0, n = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++n) {
+                int bi, bj;
+                block_of_tile(tile, n_blk, &bi, &bj);
+                if (!mbar_wait(acc_empty, (n & 1u) ^ 1u, err)) break;   // the epilogue has drained the previous block
+                tc_fence_after();
+                for (int k = 0; k < nk; ++k, ++it) {
+                    const uint32_t s = it % kGStages, ph = (it / kGStages) & 1u;
+                    if (!mbar_wait(&full[s], ph, err)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t st = smem_u32(stages + (size_t)s * kGStageBytes);
+                    const uint32_t b_base = st + kGOperandBytes;
+                    const uint32_t a_base = bi == bj ? b_base : st;
+#pragma unroll
+                    for (int kk = 0; kk < kGTok / 16; ++kk) {
+                        // 16 tokens further = 16 swizzle rows = 2048 bytes
+                        const uint64_t db = operand_desc(b_base + (uint32_t)kk * 2048u);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const uint64_t da = operand_desc(a_base + (uint32_t)h * 2u * kGBoxBytes + (uint32_t)kk * 2048u);
+                            umma_bf16(tmem_base + (uint32_t)h * 256u, da, db, (k > 0 || kk > 0) ? 1u : 0u);
+                        }
+                    }
+                    umma_commit(&empty[s]);
+                }
+                if (ok) umma_commit(acc_full);
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..5)
+        const int q = warp & 3;   // the quarter of the tensor-memory lanes this warp may read
+        uint32_t n = 0;
+        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++n) {
+            int bi, bj;
+            block_of_tile(tile, n_blk, &bi, &bj);
+            if (!mbar_wait(acc_full, n & 1u, err)) break;
+            tc_fence_after();
+#pragma unroll 1
+            for (int h = 0; h < 2; ++h) {
+                const int64_t row = (int64_t)bi * kGBlk + h * 128 + q * 32 + lane;   // accumulator row = lane of tensor memory
+#pragma unroll 1
+                for (int c0 = 0; c0 < kGBlk; c0 += 32) {
+                    float v[32];
+                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), v);
+                    const int64_t col0 = (int64_t)bj * kGBlk + c0;
+                    if (row < cols) {
+                        float* g = G + row * ldg + col0;
+#pragma unroll
+                        for (int e = 0; e < 32; e += 4) {
+                            if (col0 + e < cols) {   // cols % 8 == 0: a group of four is inside or outside as a whole
+                                float4 o = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                                if (!reset) {
+                                    const float4 old = *reinterpret_cast<const float4*>(g + e);
+                                    o.x = __fadd_rn(old.x, o.x);
+                                    o.y = __fadd_rn(old.y, o.y);
+                                    o.z = __fadd_rn(old.z, o.z);
+                                    o.w = __fadd_rn(old.w, o.w);
+                                }
+                                *reinterpret_cast<float4*>(g + e) = o;
+                            }
+                        }
+                        if (bi != bj) {   // the mirror image: a warp writes 32 adjacent rows of one column
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) {
+                                if (col0 + e < cols) {
+                                    float* m = G + (col0 + e) * ldg + row;
+                                    *m = reset ? v[e] : __fadd_rn(*m, v[e]);
+                                }
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kGTmemCols) : "memory");
+    }
+    if (threadIdx.x == 0 && *err != 0 && status != nullptr) atomicExch(status, 1);
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                   const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// The driver's tensor-map encoder (a host-side function of the process, not of a device).
+EncodeTiledFn encode_tiled() {
+    static std::atomic<void*> cached{nullptr};
+    void* fn = cached.load(std::memory_order_acquire);
+    if (fn == nullptr) {
+        cudaDriverEntryPointQueryResult found;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &found) != cudaSuccess ||
+            found != cudaDriverEntryPointSuccess) {
+            (void)cudaGetLastError();
+            return nullptr;
+        }
+        cached.store(fn, std::memory_order_release);
+    }
+    return reinterpret_cast<EncodeTiledFn>(fn);
+}
+
+}  // namespace
+}  // namespace mosaic
+
+using namespace mosaic;
+
+extern "C" int mosaic_gram_accumulate(const void* X, int64_t tokens, int64_t cols, int64_t ldx, int dtype, float* G, int64_t ldg,
+                                      int flags, int* status_dev, void* stream) {
+    if (dtype == MOSAIC_F32) return MOSAIC_ERR_BAD_DTYPE;   // the products must be exact in fp32: bf16 only
+    if (dtype != MOSAIC_BF16) return MOSAIC_ERR_BAD_DTYPE;
+    if (tokens < 0 || cols <= 0 || ldx < cols) return MOSAIC_ERR_INVALID_ARG;
+    if (tokens > 0) {   // without tokens X is never read and may be NULL
+        const int rc = check_matrix(X, tokens, cols, ldx, dtype);
+        if (rc != MOSAIC_OK) return rc;
+    }
+    if ((cols % 8) != 0 || tokens > 0x7FFFFFFF - kGTok || cols > 0x7FFFFFFF - kGBlk || ldg < cols) return MOSAIC_ERR_INVALID_ARG;
+    if (G == nullptr) return MOSAIC_ERR_NULL_PTR;
+    if ((reinterpret_cast<uintptr_t>(G) & 15u) != 0 || (ldg % 4) != 0 || (reinterpret_cast<uintptr_t>(status_dev) & 3u) != 0)
+        return MOSAIC_ERR_MISALIGNED;
+    {   // G must not overlap X
+        const char *a = static_cast<const char*>(X), *b = reinterpret_cast<const char*>(G);
+        const size_t xs = tokens > 0 ? ((size_t)(tokens - 1) * (size_t)ldx + (size_t)cols) * 2u : 0u;   // 0: no overlap possible
+        const size_t gs = ((size_t)(cols - 1) * (size_t)ldg + (size_t)cols) * 4u;
+        if (a < b + gs && b < a + xs) return MOSAIC_ERR_ALIASING;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool reset = (flags & MOSAIC_RESET_ACCUM) != 0;
+    if (status_dev != nullptr) MOSAIC_CUDA_TRY(cudaMemsetAsync(status_dev, 0, sizeof(int), st));
+    if (tokens == 0) {
+        if (reset) MOSAIC_CUDA_TRY(cudaMemset2DAsync(G, (size_t)ldg * 4u, 0, (size_t)cols * 4u, (size_t)cols, st));
+        return MOSAIC_OK;
+    }
+    EncodeTiledFn encode = encode_tiled();
+    if (encode == nullptr) return MOSAIC_ERR_CUDA;
+    CUtensorMap map;
+    const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)tokens};
+    const cuuint64_t gstride[1] = {(cuuint64_t)ldx * 2u};
+    const cuuint32_t box[2] = {(cuuint32_t)kGBoxCols, (cuuint32_t)kGTok};
+    const cuuint32_t estride[2] = {1u, 1u};
+    if (encode(&map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2u, const_cast<void*>(X), gdim, gstride, box, estride, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return MOSAIC_ERR_CUDA;
+    static DeviceCache opted;   // the shared-memory opt-in belongs to one device's copy of the kernel
+    const int ok = opted.get([&]() -> int {
+        if (cudaFuncSetAttribute(gram_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGSmemBytes) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return -1;
+        }
+        return 1;
+    });
+    if (ok < 0) return MOSAIC_ERR_CUDA;
+    const int n_blk = (int)((cols + kGBlk - 1) / kGBlk);
+    const int64_t n_tiles = (int64_t)n_blk * (n_blk + 1) / 2;
+    if (n_tiles > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
+    const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
+    gram_kernel<<<grid, kGThreads, kGSmemBytes, st>>>(map, G, ldg, (int)cols, (int)tokens, n_blk, (int)n_tiles, reset ? 1 : 0, status_dev);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
