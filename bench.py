@@ -21,7 +21,9 @@ After the headline region (N = 1 only) two more arms are timed and appended
 to the same JSON line: `structured` - rows and columns of every projection of
 the compaction-stress configuration ranked and compacted at f = 0.3 - and
 `composite` - one pass over the LLaMA-3-8B-shaped configuration: outlier
-sweeps, allocation, 50 % unstructured, then the coupled 20 % structured stage.
+sweeps, allocation, 50 % unstructured, then the coupled 20 % structured stage -
+and `hessian` - the second-moment matrices X^T X of one layer's projection
+inputs on the tensor cores (the calibration-side companion of the norms).
 --blocks chooses the arms (default: all).
 
 --impl reference times the CPU oracle (as it stands) on the host cores over a
@@ -62,6 +64,16 @@ def measured_peaks():
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured"
     return 6650.0, "fallback"
+
+
+def measured_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s of the library GEMM on this machine, and where they come from."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), "measured"
+    return 1590.0, 1400.0, "fallback"
 
 
 class ClockSampler:
@@ -230,6 +242,8 @@ def run_native(args, cfg):
         line = {"metric": METRIC, "n_gpus": 1, "note": "headline arm skipped (--blocks)"}
         if "structured" in blocks:
             line["structured"] = run_structured_block(args, st, peak)
+        if "hessian" in blocks:
+            line["hessian"] = run_hessian_block(args, cfg, X, dev, local)
         del st, X
         torch.cuda.empty_cache()
         if "composite" in blocks:
@@ -372,6 +386,8 @@ def run_native(args, cfg):
     if world == 1:
         if "structured" in blocks:
             line["structured"] = run_structured_block(args, st, peak)
+        if "hessian" in blocks:
+            line["hessian"] = run_hessian_block(args, cfg, X, dev, local)
         del st, X
         torch.cuda.empty_cache()
         if "composite" in blocks:
@@ -416,6 +432,52 @@ def run_structured_block(args, st, peak):
                         f"projection independently, f = {f}", "ms": t["median"], "ms_min": t["min"], "ms_max": t["max"],
             "algorithmic_bytes": nbytes, "bytes_per_weight": nbytes / w, "achieved": gbs, "unit": "GB/s", "peak": peak,
             "frac": gbs / peak, "projections": len(st.W)}
+
+
+def run_hessian_block(args, cfg, X, dev, local):
+    """Calibration-side companion: the second-moment matrix G = X^T X of every projection input of one
+    layer (the matrix the inverse-Hessian back-end is built from), on the tensor cores, over the resident
+    calibration activations in calls of 32768 tokens.  Algorithmic flops: tokens * cols * (cols + 1) per
+    input (G is symmetric: the blocks on or above the diagonal are computed, the rest mirrored)."""
+    from paper_2504_06323_b200 import driver
+    chunk = 32768
+    G = {xk: torch.empty(x.shape[1], x.shape[1], device=dev, dtype=torch.float32) for xk, x in X.items()}
+    status = torch.zeros(1, device=dev, dtype=torch.int32)
+    timed_out = []
+
+    def one_pass():
+        launches = 0
+        for xk, x in X.items():
+            launches += driver.accumulate_second_moments(G[xk], x, reset=True, status=status, chunk_tokens=chunk)
+        return launches
+
+    one_pass()
+    torch.cuda.synchronize()
+    timed_out.append(int(status.item()))
+    sampler = ClockSampler(local)
+    sampler.start()
+    t = _median_ms(one_pass, warmup=1, reps=5)
+    clocks = sampler.stop()
+    timed_out.append(int(status.item()))
+    launches = one_pass()
+    torch.cuda.synchronize()
+    alg = sum(float(x.shape[0]) * x.shape[1] * (x.shape[1] + 1) for x in X.values())
+    exe = 0.0
+    for x in X.values():
+        nb = (x.shape[1] + 255) // 256
+        exe += 2.0 * x.shape[0] * 256.0 * 256.0 * nb * (nb + 1) / 2
+    burst, sustained, kind = measured_tensor_peaks()
+    tf = alg / (t["median"] * 1e-3) / 1e12
+    return {"workload": f"{cfg.name}: G = X^T X of the {len(X)} projection inputs of one layer "
+                        f"({', '.join(str(x.shape[1]) for x in X.values())} columns, {next(iter(X.values())).shape[0]} tokens, "
+                        f"bf16 in, fp32 out, {chunk} tokens per call)",
+            "kernel": "gram_kernel (tcgen05.mma, TMA-staged MN-major tiles, 256x256 fp32 blocks in tensor memory)",
+            "bound": "tensor", "ms": t["median"], "ms_min": t["min"], "ms_max": t["max"], "gpu_launches": launches,
+            "algorithmic_flops": alg, "executed_flops": exe, "achieved": tf, "achieved_executed": exe / (t["median"] * 1e-3) / 1e12,
+            "unit": "TFLOP/s", "peak": burst, "peak_sustained": sustained, "peak_kind": f"of {kind} (library bf16 GEMM; burst / sustained)",
+            "frac": tf / burst, "frac_of_sustained": tf / sustained, "dtype": "bf16 x bf16 -> fp32", "clocks": clocks,
+            "bounded_wait_ran_out": any(timed_out),
+            "vs_full_square_gemm": "a library GEMM of X^T X computes both triangles: twice the flops counted here"}
 
 
 def run_composite_block(args, dev, peak):
@@ -584,7 +646,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--e2e-chunk", type=int, default=16384)
-    ap.add_argument("--blocks", default="headline,structured,composite",
+    ap.add_argument("--blocks", default="headline,structured,composite,hessian",
                     help="arms appended to the line at N = 1: headline, structured, composite")
     args = ap.parse_args()
     cfg = wl.CONFIGS[args.config]

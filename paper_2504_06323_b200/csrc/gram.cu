@@ -269,28 +269,41 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
                     tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), v);
                     const int64_t col0 = (int64_t)bj * kGBlk + c0;
                     if (row < cols) {
+                        // (when accumulating, all old values of a pass are read before the first store, so
+                        // that the reads are in flight together rather than one round trip each)
                         float* g = G + row * ldg + col0;
+                        float4 o[8];
 #pragma unroll
-                        for (int e = 0; e < 32; e += 4) {
-                            if (col0 + e < cols) {   // cols % 8 == 0: a group of four is inside or outside as a whole
-                                float4 o = make_float4(v[e], v[e + 1], v[e + 2], v[e + 3]);
+                        for (int e = 0; e < 8; ++e) {   // cols % 8 == 0: a group of four is inside or outside as a whole
+                            o[e] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                            if (!reset && col0 + 4 * e < cols) o[e] = *reinterpret_cast<const float4*>(g + 4 * e);
+                        }
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) {
+                            if (col0 + 4 * e < cols) {
+                                float4 w = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                                 if (!reset) {
-                                    const float4 old = *reinterpret_cast<const float4*>(g + e);
-                                    o.x = __fadd_rn(old.x, o.x);
-                                    o.y = __fadd_rn(old.y, o.y);
-                                    o.z = __fadd_rn(old.z, o.z);
-                                    o.w = __fadd_rn(old.w, o.w);
+                                    w.x = __fadd_rn(o[e].x, w.x);
+                                    w.y = __fadd_rn(o[e].y, w.y);
+                                    w.z = __fadd_rn(o[e].z, w.z);
+                                    w.w = __fadd_rn(o[e].w, w.w);
                                 }
-                                *reinterpret_cast<float4*>(g + e) = o;
+                                *reinterpret_cast<float4*>(g + 4 * e) = w;
                             }
                         }
                         if (bi != bj) {   // the mirror image: a warp writes 32 adjacent rows of one column
+                            float* m = G + col0 * ldg + row;
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) {
-                                if (col0 + e < cols) {
-                                    float* m = G + (col0 + e) * ldg + row;
-                                    *m = reset ? v[e] : __fadd_rn(*m, v[e]);
+                            for (int e0 = 0; e0 < 32; e0 += 16) {
+                                float om[16];
+#pragma unroll
+                                for (int e = 0; e < 16; ++e) {
+                                    om[e] = 0.0f;
+                                    if (!reset && col0 + e0 + e < cols) om[e] = m[(int64_t)(e0 + e) * ldg];
                                 }
+#pragma unroll
+                                for (int e = 0; e < 16; ++e)
+                                    if (col0 + e0 + e < cols) m[(int64_t)(e0 + e) * ldg] = reset ? v[e0 + e] : __fadd_rn(om[e], v[e0 + e]);
                             }
                         }
                     }

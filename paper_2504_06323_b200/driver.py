@@ -207,6 +207,22 @@ def count_outliers_all(st: ModelState, alpha: float | None = None) -> int:
     return len(jobs)
 
 
+def accumulate_second_moments(G: torch.Tensor, X: torch.Tensor, reset: bool = True, status: torch.Tensor | None = None,
+                              chunk_tokens: int = 32768) -> int:
+    """G (+)= X^T X over the tokens of X (fp32, both triangles): the second moments of a projection's
+    input, from which the inverse-Hessian back-end forms H = (2/T) G.  `chunk_tokens` tokens per call:
+    the fp32 error bound of a call grows with its tokens.  Returns the number of kernel launches.
+    `status` (one int32) is overwritten by every call: check it after the last one only if the calls
+    before cannot have failed, or pass chunk_tokens >= tokens."""
+    tokens = X.shape[0]
+    launches, first = 0, True
+    for t0 in range(0, max(tokens, 1), chunk_tokens):
+        api.mosaic_gram_accumulate(X[t0:t0 + chunk_tokens], G, api.RESET_ACCUM if (reset and first) else 0, status)
+        first = False
+        launches += 1 if tokens > 0 else 0
+    return launches
+
+
 def count_outliers_by_layer(st: ModelState, alpha: float | None = None) -> int:
     """Layer outlier distribution (Eq. 3-4, the layer-pruning baseline): every projection of a layer
     is counted against alpha times the mean score of the WHOLE layer.  st.counts receives the
