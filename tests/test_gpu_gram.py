@@ -105,7 +105,7 @@ def test_gram_many_blocks_sampled_pairs():
 def test_gram_llama_width_sampled_pairs():
     """One projection input at the LLaMA-7B width, 32768 calibration tokens in two calls."""
     cfg = wl.CONFIGS["llama7b"]
-    X = wl.gen_activation(wl.scaled(cfg, tokens=32768), 0, cfg.x_keys()[0], DEV)
+    X = wl.gen_activation(cfg, 0, cfg.x_keys()[0], DEV, tokens=32768)
     tokens, cols = X.shape
     assert cols == 4096
     G = run(X[:16384])
@@ -117,6 +117,29 @@ def test_gram_llama_width_sampled_pairs():
     ref, ref_abs = oracle.gram_pairs(wl.to_numpy(X), js, ls, "bf16")
     assert (np.abs(G[js, ls] - ref) <= bound(16384, 2, ref_abs)).all()
     assert np.array_equal(G[:512, 2048:2560], G[2048:2560, :512].T)
+
+
+def test_gram_full_size_widest_input_sampled_pairs():
+    """The widest projection input of the LLaMA-7B shape (11008 channels) at the full calibration
+    size (262144 tokens), accumulated the way the benchmark does it (calls of 32768 tokens)."""
+    from paper_2504_06323_b200 import driver
+    cfg = wl.CONFIGS["llama7b"]
+    X = wl.gen_activation(cfg, 0, "mlp_mid", DEV)
+    tokens, cols = X.shape
+    assert (tokens, cols) == (262144, 11008)
+    G = torch.empty(cols, cols, device=DEV)
+    status = torch.zeros(1, device=DEV, dtype=torch.int32)
+    n = driver.accumulate_second_moments(G, X, reset=True, status=status, chunk_tokens=32768)
+    torch.cuda.synchronize()
+    assert n == 8 and int(status.item()) == 0
+    rng = np.random.default_rng(2)
+    js = np.concatenate([np.array([0, 255, 256, 11007, 10752, 5000]), rng.integers(0, cols, 300)])
+    ls = np.concatenate([np.array([0, 256, 255, 11007, 17, 5000]), rng.integers(0, cols, 300)])
+    Gs = G[torch.from_numpy(js).to(DEV), torch.from_numpy(ls).to(DEV)].cpu().numpy()
+    Gt = G[torch.from_numpy(ls).to(DEV), torch.from_numpy(js).to(DEV)].cpu().numpy()
+    ref, ref_abs = oracle.gram_pairs(wl.to_numpy(X), js, ls, "bf16")
+    assert (np.abs(Gs - ref) <= bound(32768, 8, ref_abs)).all()
+    assert np.array_equal(Gs, Gt)
 
 
 def test_gram_argument_errors():

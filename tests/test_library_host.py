@@ -58,6 +58,15 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.mosaic_prune_structured_compact(16, 4, 8, 8, 1, None, 3, 1, 1, 1, 16, 16, 0, 4096, None, 256, 1 << 20,
                                                None) == -1                                   # rows % row_group
     assert lib.mosaic_rank_units(16, 4, 5, 16, None) == -1                                   # keep > n
+    # mosaic_gram_accumulate(X, tokens, cols, ldx, dtype, G, ldg, flags, status, stream)
+    assert lib.mosaic_gram_accumulate(16, 64, 64, 64, 0, 4096, 64, 0, None, None) == -3         # fp32 input: products not exact
+    assert lib.mosaic_gram_accumulate(None, 64, 64, 64, 1, 4096, 64, 0, None, None) == -2        # tokens but no X
+    assert lib.mosaic_gram_accumulate(16, 64, 64, 64, 1, None, 64, 0, None, None) == -2          # no G
+    assert lib.mosaic_gram_accumulate(16, 64, 60, 64, 1, 1 << 20, 64, 0, None, None) == -1       # cols % 8
+    assert lib.mosaic_gram_accumulate(16, 64, 64, 64, 1, 1 << 20, 60, 0, None, None) == -1       # ldg < cols
+    assert lib.mosaic_gram_accumulate(16, 64, 64, 64, 1, (1 << 20) + 4, 64, 0, None, None) == -4  # G not 16-byte aligned
+    assert lib.mosaic_gram_accumulate(16, 64, 64, 64, 1, 1 << 20, 64, 0, 6, None) == -4          # status word not 4-byte aligned
+    assert lib.mosaic_gram_accumulate(1 << 20, 64, 64, 64, 1, (1 << 20) + 4096, 64, 0, None, None) == -6   # G inside X
     assert lib.mosaic_ratio_from_count(3, 200) == 1.5
     assert lib.mosaic_act_norms_workspace_bytes(262144, 4096) % 256 == 0
 
