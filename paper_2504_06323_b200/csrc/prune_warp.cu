@@ -6,10 +6,11 @@
 // One persistent CTA per SM.  A CTA takes a contiguous range of the launch's rows, so it changes
 // matrix (job) only a few times; per job it keeps two tables in shared memory: the norms and, for
 // a window [lo, hi) of score keys that should contain every row's threshold, per column the bf16
-// magnitude pattern A_lo[j] such that a weight below it scores surely under lo, while a weight
-// from A_lo[j] + D up scores surely at least hi (the score norm_j * |w| is monotone in |w|; D is
-// one depth for the whole job).  Both patterns are exact: they are found by bisection on the very
-// product that defines a score.  The window is centred on the median of one estimate per warp -
+// magnitude pattern A_lo[j] such that a weight scores under lo iff its magnitude is below it, and
+// the depth D[j] = A_hi[j] - A_lo[j] to the pattern from which a weight scores at least hi (the
+// score norm_j * |w| is monotone in |w|).  Both patterns are exact: they are found by bisection on
+// the very product that defines a score, so the candidates of a row are exactly its weights
+// inside the window.  The window is centred on the median of one estimate per warp -
 // the matching quantile of the exact scores of a quarter of one row of the job (rows spread
 // evenly over the matrix), selected in registers - and made just wide enough, judged by the same
 // samples, to hold the ranks a row's threshold can scatter over.
@@ -49,7 +50,7 @@ constexpr uint32_t kWOverflow = 0xFFFFFFFFu;   // a warp's "my queue overflowed"
 // count slots from row to row, so that a warp may start the next row while another still reads.
 struct WarpLayout {
     int nvec, nwords, qcap;   // qcap: candidates one warp may queue
-    uint32_t off_alo, off_nrm, off_misc, off_group0, per_group;                      // bytes
+    uint32_t off_alo, off_dep, off_nrm, off_misc, off_group0, per_group;             // bytes
     uint32_t o_queue, per_queue, o_qcol, o_qbin, per_qbin, o_hist, o_mbytes, o_bkey, o_bcol, o_ctl;   // bytes inside a group's block
 };
 __host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
@@ -57,9 +58,10 @@ __host__ __device__ inline WarpLayout warp_layout(int cols, int G) {
     const uint32_t sets = G == 1 ? 1u : 2u;
     L.nvec = cols >> 3;
     L.nwords = (cols + 31) >> 5;
-    L.qcap = (((cols >> 3) * 3 / 2 + G - 1) / G + 31) & ~31;     // 3/16 of the warp's share of the row
+    L.qcap = (((cols >> 3) + G - 1) / G + 31) & ~31;             // 1/8 of the warp's share of the row
     uint32_t o = 0;
     L.off_alo = o;   o += (uint32_t)L.nvec * 16u;
+    L.off_dep = o;   o += (uint32_t)L.nvec * 16u;
     L.off_nrm = o;   o += (uint32_t)cols * 4u;
     L.off_misc = o;  o += 256u;
     L.off_group0 = o;
@@ -286,15 +288,15 @@ __device__ __forceinline__ uint32_t pattern_at_key(float n, uint32_t key_t) {
 
 // A_lo of one vector of 8 columns for the window [lo, hi) of keys (packed like the row's words);
 // returns the largest A_hi - A_lo of the vector.
-__device__ __forceinline__ uint32_t thresholds_of_vector(const float* nrm8, uint32_t lo, uint32_t hi, uint4* alo) {
-    uint32_t al[8], depth = 0u;
+__device__ __forceinline__ void thresholds_of_vector(const float* nrm8, uint32_t lo, uint32_t hi, uint4* alo, uint4* dep) {
+    uint32_t al[8], d[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         al[e] = pattern_at_key(nrm8[e], lo);
-        depth = max(depth, pattern_at_key(nrm8[e], hi) - al[e]);
+        d[e] = pattern_at_key(nrm8[e], hi) - al[e];   // hi > lo: never negative
     }
     *alo = make_uint4(al[0] | (al[1] << 16), al[2] | (al[3] << 16), al[4] | (al[5] << 16), al[6] | (al[7] << 16));
-    return depth;
+    *dep = make_uint4(d[0] | (d[1] << 16), d[2] | (d[3] << 16), d[4] | (d[5] << 16), d[6] | (d[7] << 16));
 }
 
 // blockDim.x = 32 * G * groups; dynamic shared memory = off_group0 + groups * per_group of warp_layout(cols, G).
@@ -313,8 +315,9 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
     const int gid = wid / G, sub = wid % G, ngroups = nwarps / G;
     const int gl = sub * 32 + lane;    // thread within the row group: owns the vectors v * TG + gl
     uint4* alo = reinterpret_cast<uint4*>(smem + L.off_alo);
+    uint4* dep = reinterpret_cast<uint4*>(smem + L.off_dep);
     float* nrm = reinterpret_cast<float*>(smem + L.off_nrm);
-    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates, [16] window depth,
+    uint32_t* misc = reinterpret_cast<uint32_t*>(smem + L.off_misc);   // [0..15] the warps' threshold estimates,
                                                                        // [17] samples taken, [32..63] samples by distance from the centre
     unsigned char* mine = smem + L.off_group0 + (size_t)gid * L.per_group;
     uint4* row = reinterpret_cast<uint4*>(mine);
@@ -363,7 +366,7 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
         }
         if (tid < 64) misc[tid] = 0u;
         bool valid = __syncthreads_and(fin ? 1 : 0) != 0;
-        uint32_t lo = 0u, width = 0u, DD = 0u;
+        uint32_t lo = 0u, width = 0u;
         int shift = 0;
         if (valid) {
             // One estimate per warp: the k-th score of row (rows-1)*wid/(nwarps-1), taken as the matching
@@ -474,24 +477,15 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 }
             }
             if (valid) {
-                uint32_t depth = 0u;
+                // A_lo + D = A_hi <= 0x7F80 for every column, which the borrow-free subtraction needs
                 for (int vec = tid; vec < nvec; vec += nthreads) {
                     const float4 n0 = reinterpret_cast<const float4*>(nrm)[vec * 2], n1 = reinterpret_cast<const float4*>(nrm)[vec * 2 + 1];
                     const float n8[8] = {n0.x, n0.y, n0.z, n0.w, n1.x, n1.y, n1.z, n1.w};
-                    depth = max(depth, thresholds_of_vector(n8, lo, lo + width, &alo[vec]));
+                    thresholds_of_vector(n8, lo, lo + width, &alo[vec], &dep[vec]);
                 }
-                depth = __reduce_max_sync(0xFFFFFFFFu, depth);
-                if (lane == 0) atomicMax(&misc[16], depth);
             }
         }
         __syncthreads();
-        if (valid) {
-            // One depth for all columns: A_hi = A_lo + D.  D <= 128 keeps A_lo + D <= 0x8000 for every
-            // column (A_lo <= 0x7F80), which the borrow-free subtraction needs.
-            const uint32_t depth = misc[16];
-            valid = depth <= 128u;
-            DD = depth | (depth << 16);
-        }
 
         // ---------------- rows of the segment, one per group at a time
         auto fetch = [&](int64_t rr) {   // this warp's vectors of global row rr into the group's buffer (one cp.async group)
@@ -527,11 +521,11 @@ __global__ void __launch_bounds__(kWMaxWarps * 32, 1) prune_rows_warp_kernel(con
                 for (int v = 0; v < V; ++v) {
                     const int vec = v * TG + gl;
                     if (FULL || vec < nvec) {
-                        const uint4 rr = row[vec], a = alo[vec];
+                        const uint4 rr = row[vec], a = alo[vec], d = dep[vec];
                         const uint32_t t0 = (rr.x | 0x80008000u) - a.x, t1 = (rr.y | 0x80008000u) - a.y,
                                        t2 = (rr.z | 0x80008000u) - a.z, t3 = (rr.w | 0x80008000u) - a.w;
                         const uint32_t keepf = flags8(t0, t1, t2, t3);
-                        const uint32_t above = flags8(t0 - DD, t1 - DD, t2 - DD, t3 - DD);
+                        const uint32_t above = flags8(t0 - d.x, t1 - d.y, t2 - d.z, t3 - d.w);
                         candw[v >> 2] |= (keepf & ~above) >> (2 * (v & 3));
                         below += 8u - (uint32_t)__popc(keepf);
                         mbytes[vec] = (uint8_t)byte_of_flags(keepf);   // candidates count as kept until the threshold says otherwise
