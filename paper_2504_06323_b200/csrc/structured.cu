@@ -131,7 +131,40 @@ __global__ void __launch_bounds__(kSThreads, 6) unit_partial_kernel(const __grid
         nrm[e] = (c0 + e < cols) ? (J.norms ? J.norms[c0 + e] : 1.0f) : 0.0f;
     }
     constexpr int U = 4;   // rows in flight per warp
+    // bf16 rows of whole vectors: the same sums in the same order with plain pointer stepping
+    const bool lean = DT == MOSAIC_BF16 && (cols % kVec) == 0;
     for (int64_t rs = r0; rs < r1; rs += kSSubRows) {
+        if (lean) {
+            const int n_sub = (int)(r1 - rs < kSSubRows ? r1 - rs : kSSubRows);
+            const bool lane_in = c0 < cols;
+            const size_t stride = (size_t)ldw * 2u;
+            const char* base = static_cast<const char*>(J.W) + ((size_t)rs * (size_t)ldw + (size_t)(lane_in ? c0 : 0)) * 2u;
+#pragma unroll 1
+            for (int i = wid; i < kSSubRows; i += U * kSWarps) {
+                uint4 v[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int r = i + u * kSWarps;
+                    v[u] = make_uint4(0u, 0u, 0u, 0u);
+                    if (lane_in && r < n_sub) v[u] = ld_stream16_ro(base + (size_t)r * stride);
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const uint32_t w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+                    double p = 0.0;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const double s0 = (double)__fmul_rn(nrm[2 * q], fabsf(__uint_as_float(w[q] << 16)));
+                        acc[2 * q] += s0;
+                        p += s0;
+                        const double s1 = (double)__fmul_rn(nrm[2 * q + 1], fabsf(__uint_as_float(w[q] & 0xFFFF0000u)));
+                        acc[2 * q + 1] += s1;
+                        p += s1;
+                    }
+                    rowbuf[lane][i + u * kSWarps] = p;
+                }
+            }
+        } else
 #pragma unroll 1
         for (int i = wid; i < kSSubRows; i += U * kSWarps) {
             Raw8<DT> v[U];
