@@ -571,7 +571,7 @@ static int launch_compact(const CompactJobList<NJ>& list, int64_t total_out_rows
     if (opted < 0) return MOSAIC_ERR_CUDA;
     // Resident CTAs: bounded by the staging buffer and by 2048 threads per SM.  What has to be in
     // flight to keep HBM busy is rows, not threads: short rows get CTAs of 128 threads, 16 per SM.
-    const int by_smem = smem == 0 ? 16 : (int)((200 * 1024) / (smem + 1024));
+    const int by_smem = smem == 0 ? 16 : (int)((216 * 1024) / (smem + 1024));
     const int threads = by_smem > 8 ? 128 : 256;
     int per_sm = by_smem < 1 ? 1 : (by_smem > 2048 / threads ? 2048 / threads : by_smem);
     int64_t grid = (int64_t)sm_count() * per_sm;
