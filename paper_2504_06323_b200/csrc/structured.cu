@@ -572,7 +572,7 @@ static int launch_compact(const CompactJobList<NJ>& list, int64_t total_out_rows
     // Resident CTAs: bounded by the staging buffer and by 2048 threads per SM.  What has to be in
     // flight to keep HBM busy is rows, not threads: short rows get CTAs of 128 threads, 16 per SM.
     const int by_smem = smem == 0 ? 16 : (int)((216 * 1024) / (smem + 1024));
-    const int threads = by_smem > 8 ? 128 : 256;
+    const int threads = by_smem >= 16 ? 128 : 256;
     int per_sm = by_smem < 1 ? 1 : (by_smem > 2048 / threads ? 2048 / threads : by_smem);
     int64_t grid = (int64_t)sm_count() * per_sm;
     if (grid > total_out_rows) grid = total_out_rows;
