@@ -13,7 +13,7 @@
 //     memory the columns of a token lie contiguous, i.e. both operands are "MN-major", which
 //     tcgen05.mma takes through its instruction descriptor - X is never transposed;
 //   * warp 0 issues the TMA loads of a 3-stage ring, one thread of warp 1 issues the MMAs (eight
-//     128 x 256 x 16 per stage) and commits each stage back to the loader, warps 2..5 drain the
+//     128 x 256 x 16 per stage) and commits each stage back to the loader, warps 2..9 drain the
 //     accumulator with tcgen05.ld once the block's last MMA has completed.  On a diagonal block the
 //     two operands are the same columns: they are loaded once.
 // A block is accumulated by one CTA in token order, so results do not depend on the grid.
@@ -33,7 +33,8 @@ constexpr int kGBoxCols = 64;                                            // 64 b
 constexpr uint32_t kGBoxBytes = kGBoxCols * kGTok * 2;                   // 8 KB
 constexpr uint32_t kGOperandBytes = (kGBlk / kGBoxCols) * kGBoxBytes;    // 256 columns x 64 tokens = 32 KB
 constexpr uint32_t kGStageBytes = 2 * kGOperandBytes;                    // A block, then B block
-constexpr int kGThreads = 192;
+constexpr int kGEpiWarps = 8;                                            // two per quarter of the tensor-memory lanes
+constexpr int kGThreads = 64 + 32 * kGEpiWarps;
 constexpr uint32_t kGTmemCols = 512;
 constexpr size_t kGSmemBytes = (size_t)kGStages * kGStageBytes + 1024 /* alignment */ + 256 /* barriers */;
 constexpr long long kGWaitCycles = 4000000000ll;                         // about two seconds
@@ -117,22 +118,19 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 32 consecutive accumulator columns of this thread's lane of tensor memory.
-__device__ __forceinline__ void tmem_load32(uint32_t addr, float (&v)[32]) {
-    uint32_t r[32];
+// 16 consecutive accumulator columns of this thread's lane of tensor memory.
+__device__ __forceinline__ void tmem_load16(uint32_t addr, float (&v)[16]) {
+    uint32_t r[16];
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
-          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
-          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
-          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
         : "r"(addr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+    for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // Block (bi, bj), bi <= bj, number `tile` in the row-by-row list of the blocks on or above the diagonal.
@@ -165,7 +163,7 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
             mbar_init(&empty[s], 1u);
         }
         mbar_init(acc_full, 1u);
-        mbar_init(acc_empty, 4u);   // one arrival per epilogue warp
+        mbar_init(acc_empty, (uint32_t)kGEpiWarps);   // one arrival per epilogue warp
         *err = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -252,8 +250,12 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
             }
         }
     } else {
-        // ------------------------------------------------------------ epilogue (warps 2..5)
-        const int q = warp & 3;   // the quarter of the tensor-memory lanes this warp may read
+        // ------------------------------------------------------------ epilogue (warps 2..9)
+        // A warp reads the quarter (warp % 4) of the tensor-memory lanes; the two warps of a quarter
+        // split the accumulator's columns.  Passes of 16 columns: all old values of a pass (direct
+        // block and mirror block) are read before its first store, one round trip per pass.
+        const int q = warp & 3;
+        const int c_begin = ((warp - 2) >> 2) * (kGBlk / 2);
         uint32_t n = 0;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++n) {
             int bi, bj;
@@ -264,22 +266,28 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
             for (int h = 0; h < 2; ++h) {
                 const int64_t row = (int64_t)bi * kGBlk + h * 128 + q * 32 + lane;   // accumulator row = lane of tensor memory
 #pragma unroll 1
-                for (int c0 = 0; c0 < kGBlk; c0 += 32) {
-                    float v[32];
-                    tmem_load32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), v);
+                for (int c0 = c_begin; c0 < c_begin + kGBlk / 2; c0 += 16) {
+                    float v[16];
+                    tmem_load16(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(h * 256 + c0), v);
                     const int64_t col0 = (int64_t)bj * kGBlk + c0;
                     if (row < cols) {
-                        // (when accumulating, all old values of a pass are read before the first store, so
-                        // that the reads are in flight together rather than one round trip each)
-                        float* g = G + row * ldg + col0;
-                        float4 o[8];
+                        float* g = G + row * ldg + col0;      // direct block: 64 bytes of the lane's own row
+                        float* m = G + col0 * ldg + row;      // mirror block: a warp covers 32 adjacent rows of a column
+                        const bool mirror = bi != bj;
+                        float4 o[4];
+                        float om[16];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {   // cols % 8 == 0: a group of four is inside or outside as a whole
+                        for (int e = 0; e < 4; ++e) {   // cols % 8 == 0: a group of four is inside or outside as a whole
                             o[e] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                             if (!reset && col0 + 4 * e < cols) o[e] = *reinterpret_cast<const float4*>(g + 4 * e);
                         }
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) {
+                        for (int e = 0; e < 16; ++e) {
+                            om[e] = 0.0f;
+                            if (!reset && mirror && col0 + e < cols) om[e] = m[(int64_t)e * ldg];
+                        }
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
                             if (col0 + 4 * e < cols) {
                                 float4 w = make_float4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
                                 if (!reset) {
@@ -291,20 +299,10 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
                                 *reinterpret_cast<float4*>(g + 4 * e) = w;
                             }
                         }
-                        if (bi != bj) {   // the mirror image: a warp writes 32 adjacent rows of one column
-                            float* m = G + col0 * ldg + row;
+                        if (mirror) {
 #pragma unroll
-                            for (int e0 = 0; e0 < 32; e0 += 16) {
-                                float om[16];
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) {
-                                    om[e] = 0.0f;
-                                    if (!reset && col0 + e0 + e < cols) om[e] = m[(int64_t)(e0 + e) * ldg];
-                                }
-#pragma unroll
-                                for (int e = 0; e < 16; ++e)
-                                    if (col0 + e0 + e < cols) m[(int64_t)(e0 + e) * ldg] = reset ? v[e0 + e] : __fadd_rn(om[e], v[e0 + e]);
-                            }
+                            for (int e = 0; e < 16; ++e)
+                                if (col0 + e < cols) m[(int64_t)e * ldg] = reset ? v[e] : __fadd_rn(om[e], v[e]);
                         }
                     }
                 }
