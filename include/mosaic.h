@@ -410,8 +410,11 @@ int mosaic_compact_batch(const mosaic_compact_job *jobs, int64_t n_jobs, int dty
  *
  * Arithmetic: products exact, sums in fp32 on the tensor cores in token order
  * within a chunk, one fp32 add per chunk into G.  The result is deterministic
- * (independent of the grid) and differs from the exact sum by at most
- * (tokens/16 + 2) * 2^-24 * sum_t |X[t,j]| |X[t,l]| per call.
+ * (independent of the grid).  The tensor cores truncate when they add 16 tokens'
+ * products to the running sum, so the result of a call differs from the exact
+ * sum by at most (tokens/4 + 2) * 2^-24 * sum_t |X[t,j]| |X[t,l]| (measured: about
+ * tokens/16 * 2^-24 of the sum, low, on sums of one sign such as the diagonal;
+ * shorter calls lose proportionally less).
  * ------------------------------------------------------------------------- */
 int mosaic_gram_accumulate(const void *X, int64_t tokens, int64_t cols, int64_t ldx, int dtype, float *G,
                            int64_t ldg, int flags, int *status_dev, void *stream);

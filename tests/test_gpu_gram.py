@@ -2,8 +2,10 @@
 inverse-Hessian back-end of Section 4.1.2 is built from) against the fp64 oracle.
 
 The kernel sums exact bf16 products in fp32 on the tensor cores, so parity is a tolerance, derived
-from the arithmetic: one rounding of the running sum per 16-token MMA step plus the adds into G,
-each at most 2^-24 of sum_t |x_tj| |x_tl| (which the oracle returns beside the sum).
+from the arithmetic: every 16-token MMA step adds 16 exact products to the running sum and
+truncates - allow 2 units in the last place of the largest operand, i.e. 2^-22 of
+sum_t |x_tj| |x_tl| (which the oracle returns beside the sum) per step - plus the rounded add into G.
+Observed on sums of one sign (the diagonal): about a quarter of that, always low.
 """
 import numpy as np
 import pytest
@@ -18,7 +20,7 @@ ERR_INVALID_ARG, ERR_NULL_PTR, ERR_BAD_DTYPE, ERR_MISALIGNED, ERR_ALIASING = -1,
 
 
 def bound(tokens_per_call, calls, G_abs):
-    return (tokens_per_call / 16.0 + 2.0) * calls * 2.0 ** -24 * G_abs
+    return (tokens_per_call / 4.0 + 2.0) * calls * 2.0 ** -24 * G_abs
 
 
 def synth(tokens, cols, seed, outliers=True):
@@ -50,7 +52,7 @@ def test_gram_whole_matrix_against_oracle(tokens, cols):
     assert np.array_equal(G, G.T)                      # both triangles hold the same bits
     # diag(G) is the squared norm of Eq. 5
     ss = oracle.act_sumsq(wl.to_numpy(X), None, "bf16")
-    assert np.allclose(np.diag(G), ss, rtol=(tokens / 16.0 + 2.0) * 2.0 ** -24)
+    assert np.allclose(np.diag(G), ss, rtol=(tokens / 4.0 + 2.0) * 2.0 ** -24)
 
 
 def test_gram_accumulates_over_chunks_and_respects_ld():
