@@ -12,6 +12,7 @@ from __future__ import annotations
 import ctypes as C
 import os
 
+import numpy as np
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -345,13 +346,14 @@ def mosaic_allocate_sparsity(outlier_counts, numels, cols, n_layers: int, n_proj
                              lam: float = 0.08, mode: int = GLOBAL_NORM):
     """Host call: (sparsity[N*M] fp64, k[N*M] int64, infeasible flag) from the outlier counts."""
     n = n_layers * n_proj
-    I64 = C.c_int64 * n
-    oc, ne, cl = I64(*[int(v) for v in outlier_counts]), I64(*[int(v) for v in numels]), I64(*[int(v) for v in cols])
-    s, k = (C.c_double * n)(), I64()
-    st = _check(lib().mosaic_allocate_sparsity(C.addressof(oc), C.addressof(ne), C.addressof(cl), n_layers, n_proj,
-                                               float(p), float(lam), int(mode), C.addressof(s), C.addressof(k)),
+    oc, ne, cl = (np.ascontiguousarray(v, dtype=np.int64) for v in (outlier_counts, numels, cols))
+    if not (oc.shape == ne.shape == cl.shape == (n,)):
+        raise ValueError("outlier_counts, numels and cols need one entry per projection")
+    s, k = np.empty(n, dtype=np.float64), np.empty(n, dtype=np.int64)
+    st = _check(lib().mosaic_allocate_sparsity(oc.ctypes.data, ne.ctypes.data, cl.ctypes.data, n_layers, n_proj,
+                                               float(p), float(lam), int(mode), s.ctypes.data, k.ctypes.data),
                 "mosaic_allocate_sparsity", allow=(ERR_INFEASIBLE,))
-    return list(s), list(k), st == ERR_INFEASIBLE
+    return s.tolist(), k.tolist(), st == ERR_INFEASIBLE
 
 
 def _out_ptr(W_in: torch.Tensor, W_out: torch.Tensor | None, rows: int, cols: int, ldw: int):
@@ -424,8 +426,8 @@ class PruneBatch:
         if k is not None:
             if len(k) != len(self.jobs):
                 raise ValueError("one k per job")
-            for i, kk in enumerate(k):
-                self.arr[i].k = int(kk)
+            # (the k fields of all jobs in one strided write: a job is 8 words, k the seventh)
+            np.frombuffer(self.arr, dtype=np.int64).reshape(len(self.jobs), 8)[:, 6] = np.asarray(k, dtype=np.int64)
             self.ws_bytes = lib().mosaic_prune_unstructured_batch_workspace_bytes(C.addressof(self.arr), len(self.jobs), self.code)
         wp, wn = _ws(ws, self.device).get(self.ws_bytes)
         _check(lib().mosaic_prune_unstructured_batch(C.addressof(self.arr), len(self.jobs), self.code, wp, wn, _stream(stream)),

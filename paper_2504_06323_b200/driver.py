@@ -18,6 +18,7 @@ from __future__ import annotations
 
 from dataclasses import dataclass, field
 
+import numpy as np
 import torch
 
 from . import api
@@ -59,12 +60,9 @@ def plan_sparsity(cfg: ModelConfig, counts: list[int], p: float | None = None, l
                   mode: int = api.GLOBAL_NORM, n_layers: int | None = None):
     """normalize(R_LLM) + Projection Planner through the library's host call."""
     n_layers = cfg.n_layers if n_layers is None else n_layers
-    numels, cols = [], []
-    for _ in range(n_layers):
-        for pr in PROJECTIONS:
-            r, c = cfg.shape(pr)
-            numels.append(r * c)
-            cols.append(c)
+    shapes = [cfg.shape(pr) for pr in PROJECTIONS]
+    numels = np.tile(np.array([r * c for r, c in shapes], dtype=np.int64), n_layers)
+    cols = np.tile(np.array([c for _, c in shapes], dtype=np.int64), n_layers)
     return api.mosaic_allocate_sparsity(counts, numels, cols, n_layers, len(PROJECTIONS),
                                         cfg.p if p is None else p, cfg.lam if lam is None else lam, mode)
 
