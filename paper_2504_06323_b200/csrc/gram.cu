@@ -177,6 +177,7 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const int nk = (tokens + kGTok - 1) / kGTok;
+    uint32_t issued = 0;   // stages the loader thread has issued loads for
 
     if (warp == 0) {
         // ------------------------------------------------------------ loader
@@ -204,15 +205,7 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
                     }
                 }
             }
-            if (!ok) {
-                // gave up: let the loads already issued land before the CTA leaves (bounded)
-                for (uint32_t back = 1; back <= (uint32_t)kGStages && back <= it; ++back) {
-                    const uint32_t j = it - back, s = j % kGStages, ph = (j / kGStages) & 1u;
-                    const long long t0 = clock64();
-                    while (!mbar_try_wait(&full[s], ph) && clock64() - t0 < kGWaitCycles) {
-                    }
-                }
-            }
+            issued = it;
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issue
@@ -319,7 +312,17 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kGTmemCols) : "memory");
     }
-    if (threadIdx.x == 0 && *err != 0 && status != nullptr) atomicExch(status, 1);
+    if (threadIdx.x == 0 && *err != 0) {
+        // Some role gave up.  Every role has left its loop by now; let the loads of the last stages
+        // land before the CTA leaves its shared memory (a completed phase answers at once; bounded).
+        for (uint32_t back = 1; back <= (uint32_t)kGStages && back <= issued; ++back) {
+            const uint32_t j = issued - back, s = j % kGStages, ph = (j / kGStages) & 1u;
+            const long long t0 = clock64();
+            while (!mbar_try_wait(&full[s], ph) && clock64() - t0 < kGWaitCycles) {
+            }
+        }
+        if (status != nullptr) atomicExch(status, 1);
+    }
 }
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
