@@ -394,8 +394,10 @@ int mosaic_compact_batch(const mosaic_compact_job *jobs, int64_t n_jobs, int dty
  * calibration samples also give the pruning back-end its Hessian; Section 4.1.2:
  * that back-end ranks and updates weights with the inverse Hessian):
  *     G[j,l] += sum_t X[t,j] * X[t,l]        for all 0 <= j, l < cols.
- * The layer Hessian of the back-end is H = (2/T) * G over all T calibration
- * tokens; diag(G) is the squared norm of Eq. 5.  Call once per chunk of tokens.
+ * The layer Hessian of the back-end is a constant multiple of G (2 X X^T over
+ * the calibration tokens, divided by whatever the back-end averages by: (2/T) G
+ * per token; the constant changes none of its rankings); diag(G) is the squared
+ * norm of Eq. 5.  Call once per chunk of tokens.
  *
  *   X          device, [tokens, cols] row-major, ld = ldx, MOSAIC_BF16 only
  *              (bf16 products are exact in fp32; MOSAIC_F32 -> MOSAIC_ERR_BAD_DTYPE).
