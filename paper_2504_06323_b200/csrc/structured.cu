@@ -394,10 +394,14 @@ template <int DT, int NJ>
 __global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ CompactJobList<NJ> jobs, int64_t total_out_rows) {
     extern __shared__ __align__(16) unsigned char srow[];
     constexpr int esz = (DT == MOSAIC_F32) ? 4 : 2;
+    int job = 0;   // a CTA's rows ascend, so its job index only moves forward
     for (int64_t g = blockIdx.x; g < total_out_rows; g += gridDim.x) {
-        const CompactJob& J = jobs.job[find_job(jobs.n, g, [&](int i) { return jobs.job[i].out_row0; })];
+        while (job + 1 < jobs.n && jobs.job[job + 1].out_row0 <= g) ++job;
+        const CompactJob& J = jobs.job[job];
         const int64_t a = g - J.out_row0;
-        const int64_t src_row = clamp_unit(J.row_keep[a / J.row_group], J.n_ru) * J.row_group + a % J.row_group;
+        // (rows < 2^31: 32-bit division, and none at all for single rows)
+        const uint32_t rg = (uint32_t)J.row_group, a_unit = rg == 1u ? (uint32_t)a : (uint32_t)a / rg, a_in = rg == 1u ? 0u : (uint32_t)a % rg;
+        const int64_t src_row = clamp_unit(J.row_keep[a_unit], J.n_ru) * J.row_group + a_in;
         const int64_t cols = J.cols, out_cols = J.out_cols, col_group = J.col_group;
         const char* src = static_cast<const char*>(J.W_in) + (size_t)src_row * (size_t)J.ldw * esz;
         char* dst = static_cast<char*>(J.W_out) + (size_t)a * (size_t)out_cols * esz;
@@ -408,12 +412,13 @@ __global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ Co
             const int64_t nvec = out_cols / kVec;
             const bool dst_aligned = (out_cols % kVec) == 0;   // else only a whole-row copy with a ragged width gets here
             if (dst_aligned) {
-                for (int64_t v = threadIdx.x; v < nvec; v += blockDim.x) {
-                    const int64_t b0 = v * kVec;
-                    const int64_t j0 = (col_group == 1) ? b0 : clamp_unit(J.col_keep[b0 / col_group], J.n_cu) * col_group + b0 % col_group;
+                const uint32_t cg = (uint32_t)col_group;   // (columns < 2^31: 32-bit division)
+                for (int v = threadIdx.x; v < (int)nvec; v += blockDim.x) {
+                    const uint32_t b0 = (uint32_t)v * kVec;
+                    const int64_t j0 = (cg == 1u) ? (int64_t)b0 : clamp_unit(J.col_keep[b0 / cg], J.n_cu) * col_group + b0 % cg;
                     Raw8<DT> r;
                     r.template load<true>(src + j0 * esz);
-                    r.store(dst + b0 * esz);
+                    r.store(dst + (size_t)b0 * esz);
                 }
             } else {
                 for (int64_t b = threadIdx.x; b < out_cols; b += blockDim.x) {
@@ -449,7 +454,7 @@ __global__ void __launch_bounds__(256) compact_kernel(const __grid_constant__ Co
                 // the output matrix is dense: an odd row of odd width starts on the upper half of a word
                 const uint16_t* s16 = reinterpret_cast<const uint16_t*>(srow);
                 uint16_t* d16 = reinterpret_cast<uint16_t*>(dst);
-                const int head = (int)((a * out_cols) & 1);
+                const int head = (int)(a & out_cols & 1);   // parity of a * out_cols
                 const int pairs = (n_out - head) / 2;
                 uint32_t* d32 = reinterpret_cast<uint32_t*>(d16 + head);
                 for (int q = threadIdx.x; q < pairs; q += blockDim.x) {
