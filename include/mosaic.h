@@ -421,6 +421,19 @@ int mosaic_compact_batch(const mosaic_compact_job *jobs, int64_t n_jobs, int dty
 int mosaic_gram_accumulate(const void *X, int64_t tokens, int64_t cols, int64_t ldx, int dtype, float *G,
                            int64_t ldg, int flags, int *status_dev, void *stream);
 
+/* ---------------------------------------------------------------------------
+ * mosaic_bounded_wait_selftest - a diagnostic with no counterpart in the paper.
+ * The tensor-core kernel of mosaic_gram_accumulate synchronises its roles
+ * through mbarriers, and every such wait carries a cycle budget so that a
+ * fault in the pipeline ends as a status word instead of a hung GPU.  This
+ * call runs that wait alone: one thread waits on a barrier that nothing will
+ * complete, for at most budget_cycles (1 .. 2e9, i.e. up to about a second),
+ * and writes how the wait ended to status_dev (device, one int):
+ *   1  the wait gave up after the budget and raised the error word (expected)
+ *   2  the barrier completed (must not happen)   3  inconsistent
+ * ------------------------------------------------------------------------- */
+int mosaic_bounded_wait_selftest(int64_t budget_cycles, int *status_dev, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

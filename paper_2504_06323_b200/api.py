@@ -41,7 +41,7 @@ SYMBOLS = (
     "mosaic_rank_units", "mosaic_sum_unit_scores",
     "mosaic_unit_scores_batch_workspace_bytes", "mosaic_unit_scores_batch", "mosaic_add_unit_scores_batch",
     "mosaic_rank_units_batch", "mosaic_compact_batch",
-    "mosaic_gram_accumulate",
+    "mosaic_gram_accumulate", "mosaic_bounded_wait_selftest",
 )
 
 
@@ -67,6 +67,8 @@ def lib() -> C.CDLL:
         L.mosaic_version.restype = ci
         L.mosaic_status_string.restype = C.c_char_p
         L.mosaic_status_string.argtypes = [ci]
+        L.mosaic_bounded_wait_selftest.restype = ci
+        L.mosaic_bounded_wait_selftest.argtypes = [i64, vp, vp]
         L.mosaic_gram_accumulate.restype = ci
         L.mosaic_gram_accumulate.argtypes = [vp, i64, i64, i64, ci, vp, i64, ci, vp, vp]
         L.mosaic_act_norms_workspace_bytes.restype = sz
@@ -229,6 +231,15 @@ def mosaic_gram_accumulate(X: torch.Tensor, G: torch.Tensor, flags: int = 0, sta
         _dev(status, "status", torch.int32)
     _check(lib().mosaic_gram_accumulate(xp, tokens, cols, ldx, _dtype_code(X), G.data_ptr(), G.stride(0), int(flags),
                                         _ptr(status), _stream(stream)), "mosaic_gram_accumulate")
+
+
+def mosaic_bounded_wait_selftest(budget_cycles: int, status: torch.Tensor, stream=None) -> None:
+    """Diagnostic: the bounded mbarrier wait of the tensor-core kernel on its own, on a barrier that
+    nothing completes.  `status` (one int32 on the device) reads 1 after synchronisation if the wait
+    gave up after `budget_cycles` and raised the error word, as it must."""
+    _dev(status, "status", torch.int32)
+    _check(lib().mosaic_bounded_wait_selftest(int(budget_cycles), status.data_ptr(), _stream(stream)),
+           "mosaic_bounded_wait_selftest")
 
 
 def mosaic_score(W: torch.Tensor, norms: torch.Tensor, score_out: torch.Tensor, stream=None) -> None:

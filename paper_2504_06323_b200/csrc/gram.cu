@@ -69,11 +69,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Waits for the phase of the given parity to complete.  False if it gave up: after kGWaitCycles
 // (then it raises *err) or because another role raised *err.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* err, long long budget = kGWaitCycles) {
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
         if (*err != 0) return false;
-        if (clock64() - t0 > kGWaitCycles) {
+        if (clock64() - t0 > budget) {
             *err = 1;
             return false;
         }
@@ -325,6 +325,20 @@ __global__ void __launch_bounds__(kGThreads, 1) gram_kernel(const __grid_constan
     }
 }
 
+// The bounded wait on its own: one thread waits, for at most `budget` cycles, on a barrier that
+// nothing will ever complete, and reports how the wait ended.
+__global__ void bounded_wait_selftest_kernel(long long budget, int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int err;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1u);
+        err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool completed = mbar_wait(&bar, 0u, &err, budget);
+        *status = completed ? 2 : (err != 0 ? 1 : 3);   // 1: gave up after the budget and raised the error word
+    }
+}
+
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -400,6 +414,17 @@ extern "C" int mosaic_gram_accumulate(const void* X, int64_t tokens, int64_t col
     if (n_tiles > 0x7FFFFFFF) return MOSAIC_ERR_INVALID_ARG;
     const int grid = (int)(n_tiles < sm_count() ? n_tiles : sm_count());
     gram_kernel<<<grid, kGThreads, kGSmemBytes, st>>>(map, G, ldg, (int)cols, (int)tokens, n_blk, (int)n_tiles, reset ? 1 : 0, status_dev);
+    MOSAIC_LAUNCH_CHECK();
+    return MOSAIC_OK;
+}
+
+extern "C" int mosaic_bounded_wait_selftest(int64_t budget_cycles, int* status_dev, void* stream) {
+    if (status_dev == nullptr) return MOSAIC_ERR_NULL_PTR;
+    if ((reinterpret_cast<uintptr_t>(status_dev) & 3u) != 0) return MOSAIC_ERR_MISALIGNED;
+    if (budget_cycles < 1 || budget_cycles > 2000000000ll) return MOSAIC_ERR_INVALID_ARG;   // at most about a second
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MOSAIC_CUDA_TRY(cudaMemsetAsync(status_dev, 0, sizeof(int), st));
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>((long long)budget_cycles, status_dev);
     MOSAIC_LAUNCH_CHECK();
     return MOSAIC_OK;
 }

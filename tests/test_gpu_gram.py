@@ -144,6 +144,27 @@ def test_gram_full_size_widest_input_sampled_pairs():
     assert np.array_equal(Gs, Gt)
 
 
+def test_bounded_wait_gives_up_and_reports():
+    """The mbarrier wait every role of the kernel uses, alone, on a barrier nothing completes: it must
+    return after its cycle budget (2e6 cycles, about a millisecond) with the error word raised, and the
+    context must stay usable."""
+    import time
+    status = torch.full((1,), 7, device=DEV, dtype=torch.int32)
+    t0 = time.perf_counter()
+    api.mosaic_bounded_wait_selftest(2_000_000, status)
+    torch.cuda.synchronize()
+    assert time.perf_counter() - t0 < 5.0
+    assert int(status.item()) == 1
+    # the context is intact: a regular call still works
+    X = synth(64, 64, seed=2)
+    G = run(X)
+    assert torch.isfinite(G).all()
+    L = api.lib()
+    assert L.mosaic_bounded_wait_selftest(0, status.data_ptr(), None) == ERR_INVALID_ARG
+    assert L.mosaic_bounded_wait_selftest(3_000_000_000, status.data_ptr(), None) == ERR_INVALID_ARG
+    assert L.mosaic_bounded_wait_selftest(1000, None, None) == ERR_NULL_PTR
+
+
 def test_gram_argument_errors():
     L = api.lib()
     X = synth(64, 64, seed=1)
