@@ -38,6 +38,18 @@ constexpr int kOutUnroll = 8;
 constexpr int kOutTileRows = 64;
 constexpr int kOutBatch = 256;                 // matrices per launch (the list travels as a kernel parameter)
 
+// Single-sweep bookkeeping of one matrix (batched bf16 path): the estimate of its score sum from a
+// sample of rows, the count of its sure outliers, and whether the ladder settled its count.
+struct OutlierCtrl {
+    double est_sum;
+    unsigned long long sure;        // weights above their column's ladder
+    unsigned long long lad_count;   // ladder entries at or above the threshold, summed by the finishing CTAs
+    int valid;                      // 1: count_out holds the count
+    int invalid;                    // some column's threshold fell off its ladder
+    int done;                       // finishing CTAs that have reported
+};
+constexpr int kLadder = 32;   // bf16 magnitude patterns per column that the single sweep keeps apart
+
 struct OutlierJob {
     const void* W;
     const float* norms;
@@ -49,6 +61,8 @@ struct OutlierJob {
     int chunks;            // tiles per row band
     int ctile0;            // first global tile of the bf16 count sweep (taller tiles)
     int g_first, g_last;   // jobs of the launch that share this job's threshold (itself alone: Eq. 6; a layer: Eq. 3-4)
+    OutlierCtrl* ctrl;     // single-sweep mode: bookkeeping and [cols][kLadder] counters in the workspace; else nullptr
+    uint32_t* ladder;
 };
 template <int NJ>
 struct OutlierJobList {
@@ -309,6 +323,7 @@ __global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(cons
     int j = jobs.n - 1, j_tau = -1;
     float tau = 0.0f;
     unsigned int cnt = 0;
+    bool settled = false;
     auto flush = [&](int job) {   // add this CTA's count for `job` (block-uniform call)
         cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
         const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -327,11 +342,15 @@ __global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(cons
         while (tile < jobs.job[j].ctile0) --j;
         const OutlierJob& J = jobs.job[j];
         if (j != j_tau) {
-            if (j_tau >= 0) flush(j_tau);
-            const int last = J.ctile0 + (int)outlier_count_tiles(J.rows, J.cols) - 1;
-            tau = group_threshold<NJ>(jobs, j, tile == last, red, &tau_sh);   // the sum: once, by the CTA that owns the matrix's last tile
+            if (j_tau >= 0 && !settled) flush(j_tau);
+            settled = J.ctrl != nullptr && __ldcg(&J.ctrl->valid) != 0;   // the single sweep has this matrix's count already
+            if (!settled) {
+                const int last = J.ctile0 + (int)outlier_count_tiles(J.rows, J.cols) - 1;
+                tau = group_threshold<NJ>(jobs, j, tile == last, red, &tau_sh);   // the sum: once, by the CTA that owns the matrix's last tile
+            }
             j_tau = j;
         }
+        if (settled) continue;
         const int local = tile - J.ctile0;
         const int chunk = local % J.chunks, band = local / J.chunks;
         const int c0 = chunk * kOutChunk + (int)threadIdx.x * kVec;
@@ -355,7 +374,227 @@ __global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(cons
             for (; r < n_rows; ++r, p += stride) cnt += count_at_or_above(ld_stream16_ro(p), A4);
         }
     }
-    if (j_tau >= 0) flush(j_tau);
+    if (j_tau >= 0 && !settled) flush(j_tau);
+}
+
+// ------------------------------------------------------------------------------------------
+// Single sweep (batched bf16 path).  The count needs the threshold tau = alpha * mean, and the mean
+// needs the whole matrix - but for a fixed column the predicate score > tau is "magnitude pattern
+// >= A_j(tau)", and bf16 has few patterns: an estimate tau^ of the threshold (from a sample of
+// rows) is enough to know that A_j(tau) lies within kLadder patterns above A_j(0.97 tau^).  The
+// sweep that sums the scores therefore also counts, per column, the weights on each of those
+// kLadder patterns (a few per mille of all weights: one atomic each) and, in registers, the
+// weights above them.  Once the sum is known the exact count is the sure ones plus the ladder
+// entries from A_j(tau) up - the same number the count sweep would find, without a second read
+// of the matrix.  A matrix whose tau falls outside some column's ladder (a poor estimate) keeps
+// valid = 0 and is counted by the count sweep after all.
+// ------------------------------------------------------------------------------------------
+
+// est_sum of every matrix: the fp64 sum of the scores of about 128 evenly spaced rows, scaled to all
+// rows.  kEstParts CTAs per matrix (128 column lanes of 8 columns x kEstRowLanes row lanes each) add
+// their shares atomically: the estimate may differ in its last bits from run to run, which moves a
+// ladder by a pattern at most and never the count.  The bookkeeping block was zeroed with the ladders.
+constexpr int kEstRowLanes = 4, kEstParts = 8;
+template <int NJ>
+__global__ void __launch_bounds__(kOutThreads * kEstRowLanes) outlier_estimate_kernel(const __grid_constant__ OutlierJobList<NJ> jobs) {
+    __shared__ double red[32];
+    const OutlierJob& J = jobs.job[blockIdx.x];
+    const int64_t step = J.rows / 128 > 0 ? J.rows / 128 : 1;
+    const int64_t n_sampled = (J.rows - step / 2 + step - 1) / step;   // rows step/2, step/2 + step, ...
+    const int cl = threadIdx.x % kOutThreads, rl = threadIdx.x / kOutThreads;
+    const int lanes = kEstRowLanes * kEstParts, my = (int)blockIdx.y * kEstRowLanes + rl;
+    const size_t stride = (size_t)J.ldw * 2u;
+    double acc[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int c0 = cl * kVec; c0 < (int)J.cols; c0 += kOutChunk) {
+        float nrm[kVec];
+#pragma unroll
+        for (int e = 0; e < kVec; ++e) nrm[e] = __ldg(J.norms + c0 + e);
+        const char* base = static_cast<const char*>(J.W) + (size_t)c0 * 2u;
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {   // at most four sampled rows per thread (128 rows over 32 lanes)
+            const int64_t i = my + (int64_t)u * lanes;
+            v[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (i < n_sampled) v[u] = ld_stream16_ro(base + (size_t)(step / 2 + i * step) * stride);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) add_scores(v[u], nrm, acc);
+        for (int64_t i = my + 4ll * lanes; i < n_sampled; i += lanes)
+            add_scores(ld_stream16_ro(base + (size_t)(step / 2 + i * step) * stride), nrm, acc);
+    }
+    const double s = block_sum((acc[0] + acc[1]) + (acc[2] + acc[3]), red);
+    if (threadIdx.x == 0) {
+        atomicAdd(&J.ctrl->est_sum, s * ((double)J.rows / (double)n_sampled));
+        if (blockIdx.y == 0) *J.count_out = 0ull;
+    }
+}
+
+// Lower edge of the ladders of job j: a little under the estimated threshold of the jobs that share it.
+template <int NJ>
+__device__ float ladder_floor(const OutlierJobList<NJ>& jobs, int j, float* sh) {
+    if (threadIdx.x == 0) {
+        const OutlierJob& J = jobs.job[j];
+        double total = 0.0, numel = 0.0;
+        for (int g = J.g_first; g <= J.g_last; ++g) {
+            total = total + __ldcg(&jobs.job[g].ctrl->est_sum);
+            numel = numel + (double)(jobs.job[g].rows * jobs.job[g].cols);
+        }
+        *sh = __double2float_rd((double)jobs.alpha * (total / numel) * 0.96875);
+    }
+    __syncthreads();
+    const float v = *sh;
+    __syncthreads();
+    return v;
+}
+
+template <int NJ>
+__global__ void __launch_bounds__(kOutThreads, 8) score_sum_ladder_kernel(const __grid_constant__ OutlierJobList<NJ> jobs,
+                                                                          int n_ctiles) {
+    __shared__ double red[32];
+    __shared__ unsigned int cred[32];
+    __shared__ float floor_sh;
+    int t_begin, t_end;
+    tile_share(n_ctiles, &t_begin, &t_end);
+    int j = 0, j_floor = -1;
+    float tau_lo = 0.0f;
+    for (int tile = t_begin; tile < t_end; ++tile) {
+        while (j + 1 < jobs.n && tile >= jobs.job[j + 1].ctile0) ++j;
+        const OutlierJob& J = jobs.job[j];
+        if (j != j_floor) {
+            tau_lo = ladder_floor<NJ>(jobs, j, &floor_sh);
+            j_floor = j;
+        }
+        const int local = tile - J.ctile0;
+        const int chunk = local % J.chunks, band = local / J.chunks;
+        const int c0 = chunk * kOutChunk + (int)threadIdx.x * kVec;
+        const bool in_cols = c0 < (int)J.cols;
+        float nrm[kVec];
+        uint4 alo = make_uint4(0x80008000u, 0x80008000u, 0x80008000u, 0x80008000u), dep = make_uint4(0u, 0u, 0u, 0u);
+        if (in_cols) {
+            uint32_t a[kVec], d[kVec];
+#pragma unroll
+            for (int e = 0; e < kVec; ++e) {
+                nrm[e] = __ldg(J.norms + c0 + e);
+                a[e] = outlier_pattern(nrm[e], tau_lo);                                  // <= 0x8000
+                d[e] = (a[e] + kLadder <= 0x8000u ? a[e] + kLadder : 0x8000u) - a[e];   // the ladder ends at 0x8000 at the latest
+            }
+            alo = make_uint4(a[0] | (a[1] << 16), a[2] | (a[3] << 16), a[4] | (a[5] << 16), a[6] | (a[7] << 16));
+            dep = make_uint4(d[0] | (d[1] << 16), d[2] | (d[3] << 16), d[4] | (d[5] << 16), d[6] | (d[7] << 16));
+        }
+        uint32_t sure = 0u;
+        uint32_t* lad = J.ladder + (size_t)c0 * kLadder;
+        // One vector: its scores into the sum, its weights above the ladder counted, those on it noted.
+        auto take = [&](const uint4& v, double (&acc)[4]) {
+            add_scores(v, nrm, acc);
+            const uint32_t t0 = (v.x | 0x80008000u) - alo.x, t1 = (v.y | 0x80008000u) - alo.y, t2 = (v.z | 0x80008000u) - alo.z,
+                           t3 = (v.w | 0x80008000u) - alo.w;                         // bit 15 / 31: magnitude >= A_lo
+            const uint32_t u0 = t0 - dep.x, u1 = t1 - dep.y, u2 = t2 - dep.z, u3 = t3 - dep.w;   // ... >= A_hi
+            // flags of the eight elements on the top bits of the bytes of two words, merged into one for one popc
+            const uint32_t ua = __byte_perm(u0, u1, 0x7531), ub = __byte_perm(u2, u3, 0x7531);
+            sure += (uint32_t)__popc((ua & 0x80808080u) | ((ub >> 1) & 0x40404040u));
+            // on the ladder: at or above A_lo but not above A_hi
+            const uint32_t ta = __byte_perm(t0, t1, 0x7531), tb = __byte_perm(t2, t3, 0x7531);
+            uint32_t hits = ((ta & ~ua) & 0x80808080u) | (((tb & ~ub) >> 1) & 0x40404040u);   // element e < 4 on bit 8e+7, e >= 4 on bit 8(e-4)+6
+            while (hits != 0u) {   // a few per mille of the weights
+                const int b = __ffs(hits) - 1;
+                hits &= hits - 1u;
+                const int e = (b >> 3) + ((b & 1) ? 0 : 4);
+                const uint32_t tw = e < 2 ? t0 : (e < 4 ? t1 : (e < 6 ? t2 : t3));
+                const uint32_t idx = ((e & 1) ? (tw >> 16) : tw) & 0x7FFFu;                   // magnitude - A_lo
+                atomicAdd(&lad[e * kLadder + idx], 1u);
+            }
+        };
+        const size_t stride = (size_t)J.ldw * 2u;
+        // the tile's four bands of kOutTileRows rows give the same partial sums, in the same order, as the sum sweep
+        for (int sub = 0; sub < kCntTileRows / kOutTileRows; ++sub) {
+            const int64_t r0 = (int64_t)band * kCntTileRows + (int64_t)sub * kOutTileRows;
+            if (r0 >= J.rows) break;   // (block-uniform)
+            const int n_rows = (int)((r0 + kOutTileRows < J.rows ? r0 + kOutTileRows : J.rows) - r0);
+            double acc[4] = {0.0, 0.0, 0.0, 0.0};
+            if (in_cols) {
+                const char* p = static_cast<const char*>(J.W) + ((size_t)r0 * (size_t)J.ldw + (size_t)c0) * 2u;
+                int r = 0;
+                for (; r + 4 <= n_rows; r += 4, p += 4 * stride) {
+                    const uint4 v0 = ld_stream16_ro(p), v1 = ld_stream16_ro(p + stride), v2 = ld_stream16_ro(p + 2 * stride),
+                                v3 = ld_stream16_ro(p + 3 * stride);
+                    take(v0, acc);
+                    take(v1, acc);
+                    take(v2, acc);
+                    take(v3, acc);
+                }
+                for (; r < n_rows; ++r, p += stride) take(ld_stream16_ro(p), acc);
+            }
+            const double blk = block_sum((acc[0] + acc[1]) + (acc[2] + acc[3]), red);
+            if (threadIdx.x == 0) J.partial[(band * (kCntTileRows / kOutTileRows) + sub) * J.chunks + chunk] = blk;
+        }
+        // the tile's sure outliers
+        sure = __reduce_add_sync(0xFFFFFFFFu, sure);
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) cred[threadIdx.x >> 5] = sure;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long tot = 0;
+            for (int i = 0; i < kOutThreads / 32; ++i) tot += cred[i];
+            if (tot) atomicAdd(&J.ctrl->sure, tot);
+        }
+    }
+}
+
+// After the sweep, one CTA per matrix and chunk of kOutChunk columns: the threshold from the partial
+// sums, then per column the ladder entries from A_j(tau) up.  The CTA that reports last writes the
+// count and valid = 1 - iff tau lies on every column's ladder.
+template <int NJ>
+__global__ void __launch_bounds__(kOutThreads) outlier_finish_kernel(const __grid_constant__ OutlierJobList<NJ> jobs) {
+    __shared__ double red[32];
+    __shared__ float tau_sh, floor_sh;
+    __shared__ unsigned long long total_sh;
+    const int j = blockIdx.x, chunk = blockIdx.y;
+    const OutlierJob& J = jobs.job[j];
+    if (chunk >= J.chunks) return;
+    const float tau = group_threshold<NJ>(jobs, j, chunk == 0, red, &tau_sh);
+    const float tau_lo = ladder_floor<NJ>(jobs, j, &floor_sh);
+    if (threadIdx.x == 0) total_sh = 0ull;
+    __syncthreads();
+    unsigned long long cnt = 0ull;
+    bool ok = true;
+    const int c_end = (chunk + 1) * kOutChunk < (int)J.cols ? (chunk + 1) * kOutChunk : (int)J.cols;
+    for (int c = chunk * kOutChunk + (int)threadIdx.x; c < c_end; c += kOutThreads) {
+        const float n = __ldg(J.norms + c);
+        const uint32_t a_lo = outlier_pattern(n, tau_lo);
+        const uint32_t a_hi = a_lo + kLadder <= 0x8000u ? a_lo + kLadder : 0x8000u;
+        const uint32_t a_star = outlier_pattern(n, tau);
+        if (a_star < a_lo || a_star > a_hi) {
+            ok = false;
+        } else {
+            // the column's whole ladder in flight, then the entries from A(tau) up
+            const uint4* lad4 = reinterpret_cast<const uint4*>(J.ladder + (size_t)c * kLadder);
+            uint4 q[kLadder / 4];
+#pragma unroll
+            for (int i = 0; i < kLadder / 4; ++i) q[i] = __ldcg(&lad4[i]);
+            const uint32_t first = a_star - a_lo, n_used = a_hi - a_lo;
+#pragma unroll
+            for (int i = 0; i < kLadder / 4; ++i) {
+                const uint32_t w[4] = {q[i].x, q[i].y, q[i].z, q[i].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if ((uint32_t)(4 * i + e) >= first && (uint32_t)(4 * i + e) < n_used) cnt += w[e];
+            }
+        }
+    }
+    if (cnt) atomicAdd(&total_sh, cnt);
+    const bool all_ok = __syncthreads_and(ok ? 1 : 0) != 0;
+    if (threadIdx.x == 0) {
+        if (total_sh) atomicAdd(&J.ctrl->lad_count, total_sh);
+        if (!all_ok) atomicOr(&J.ctrl->invalid, 1);
+        __threadfence();
+        if (atomicAdd(&J.ctrl->done, 1) == J.chunks - 1) {   // every chunk has reported
+            __threadfence();
+            if (atomicOr(&J.ctrl->invalid, 0) == 0) {
+                *J.count_out = __ldcg(&J.ctrl->sure) + atomicAdd(&J.ctrl->lad_count, 0ull);
+                J.ctrl->valid = 1;
+            }
+        }
+    }
 }
 
 template <int DT>
@@ -428,9 +667,25 @@ static int cached_occupancy(DeviceCache& cache, K kernel) {
 template <int NJ>
 static int launch_outlier(const OutlierJobList<NJ>& list, int64_t n_tiles, int64_t n_ctiles, int dtype, bool lean,
                           cudaStream_t st) {
-    static DeviceCache occ[6];   // occupancy is a property of one device's copy of a kernel
+    static DeviceCache occ[7];   // occupancy is a property of one device's copy of a kernel
     int64_t g1, g2;
-    if (lean) {
+    if (lean && list.job[0].ctrl != nullptr) {
+        // single sweep: estimates, the summing sweep with its ladders, the per-matrix finish; the count
+        // sweep follows for the matrices the ladders did not settle (its CTAs skip the others at once)
+        g1 = (int64_t)sm_count() * cached_occupancy(occ[6], score_sum_ladder_kernel<NJ>);
+        g2 = (int64_t)sm_count() * cached_occupancy(occ[1], outlier_count_bf16_kernel<NJ>);
+        if (g1 > n_ctiles) g1 = n_ctiles;
+        if (g2 > n_ctiles) g2 = n_ctiles;
+        outlier_estimate_kernel<NJ><<<dim3((unsigned)list.n, kEstParts), kOutThreads * kEstRowLanes, 0, st>>>(list);
+        MOSAIC_LAUNCH_CHECK();
+        score_sum_ladder_kernel<NJ><<<(unsigned)g1, kOutThreads, 0, st>>>(list, (int)n_ctiles);
+        MOSAIC_LAUNCH_CHECK();
+        int max_chunks = 1;
+        for (int m = 0; m < list.n; ++m) max_chunks = list.job[m].chunks > max_chunks ? list.job[m].chunks : max_chunks;
+        outlier_finish_kernel<NJ><<<dim3((unsigned)list.n, (unsigned)max_chunks), kOutThreads, 0, st>>>(list);
+        MOSAIC_LAUNCH_CHECK();
+        outlier_count_bf16_kernel<NJ><<<(unsigned)g2, kOutThreads, 0, st>>>(list, (int)n_ctiles);
+    } else if (lean) {
         g1 = (int64_t)sm_count() * cached_occupancy(occ[0], score_sum_bf16_kernel<NJ>);
         g2 = (int64_t)sm_count() * cached_occupancy(occ[1], outlier_count_bf16_kernel<NJ>);
         if (g1 > n_tiles) g1 = n_tiles;
@@ -476,15 +731,22 @@ extern "C" int mosaic_outlier_ratio(const void* W, int64_t rows, int64_t cols, i
     one.n = 1;
     one.alpha = alpha;
     one.job[0] = OutlierJob{W, norms, reinterpret_cast<unsigned long long*>(outlier_count_out), score_sum_out,
-                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk), 0, 0, 0};
+                            static_cast<double*>(ws), rows, cols, ldw, 0, (int)((cols + kOutChunk - 1) / kOutChunk), 0, 0, 0,
+                            nullptr, nullptr};
     return launch_outlier<1>(one, outlier_tiles(rows, cols), outlier_count_tiles(rows, cols), dtype,
                              dtype == MOSAIC_BF16 && cols % kVec == 0, static_cast<cudaStream_t>(stream));
+}
+
+// Single-sweep scratch of one matrix: its bookkeeping block and kLadder counters per column.
+static size_t ladder_bytes(int64_t cols) {
+    return cols > 0 ? align_up(256 + sizeof(uint32_t) * (size_t)kLadder * (size_t)cols, 256) : 256;
 }
 
 extern "C" size_t mosaic_outlier_ratio_batch_workspace_bytes(const mosaic_outlier_job* jobs, int64_t n_jobs) {
     size_t total = 256;
     if (jobs == nullptr) return total;
-    for (int64_t i = 0; i < n_jobs; ++i) total += mosaic_outlier_ratio_workspace_bytes(jobs[i].rows, jobs[i].cols);
+    for (int64_t i = 0; i < n_jobs; ++i)
+        total += mosaic_outlier_ratio_workspace_bytes(jobs[i].rows, jobs[i].cols) + ladder_bytes(jobs[i].cols);
     return total;
 }
 
@@ -519,11 +781,15 @@ static int outlier_batch(const mosaic_outlier_job* jobs, const int32_t* group_of
     char* wsp = static_cast<char*>(ws);
     bool lean = dtype == MOSAIC_BF16;
     for (int64_t m = 0; m < n_jobs; ++m) lean = lean && jobs[m].cols % kVec == 0;
+    // the single-sweep scratch lies behind all partial sums
+    char* lad = static_cast<char*>(ws);
+    for (int64_t m = 0; m < n_jobs; ++m) lad += mosaic_outlier_ratio_workspace_bytes(jobs[m].rows, jobs[m].cols);
     int64_t i = 0;
     while (i < n_jobs) {
         list.n = 0;
         list.alpha = alpha;
         int64_t tiles = 0, ctiles = 0;
+        char* lad_begin = lad;
         while (i < n_jobs) {
             const int64_t e = group_end(i);
             int64_t g_tiles = 0;
@@ -535,7 +801,9 @@ static int outlier_batch(const mosaic_outlier_job* jobs, const int32_t* group_of
                 list.job[list.n++] = OutlierJob{j.W, j.norms, reinterpret_cast<unsigned long long*>(j.outlier_count_out),
                                                 j.score_sum_out, reinterpret_cast<double*>(wsp), j.rows, j.cols, j.ldw,
                                                 (int)tiles, (int)((j.cols + kOutChunk - 1) / kOutChunk), (int)ctiles,
-                                                g_first, g_last};
+                                                g_first, g_last, lean ? reinterpret_cast<OutlierCtrl*>(lad) : nullptr,
+                                                lean ? reinterpret_cast<uint32_t*>(lad + 256) : nullptr};
+                lad += ladder_bytes(j.cols);
                 wsp += mosaic_outlier_ratio_workspace_bytes(j.rows, j.cols);
                 tiles += outlier_tiles(j.rows, j.cols);
                 ctiles += outlier_count_tiles(j.rows, j.cols);
@@ -543,6 +811,7 @@ static int outlier_batch(const mosaic_outlier_job* jobs, const int32_t* group_of
             i = e;
         }
         if (list.n == 0) return MOSAIC_ERR_INVALID_ARG;   // a single group too large for one launch
+        if (lean) MOSAIC_CUDA_TRY(cudaMemsetAsync(lad_begin, 0, (size_t)(lad - lad_begin), st));   // the ladders start at zero
         const int rc = launch_outlier<kOutBatch>(list, tiles, ctiles, dtype, lean, st);
         if (rc != MOSAIC_OK) return rc;
     }

@@ -183,6 +183,49 @@ def test_outlier_ratio_uneven_rows_and_dense_threshold(dtype):
     assert ref["certified"] and cnt.item() == ref["count"] and 0 < ref["count"] < 600 * 2048
 
 
+def test_outlier_batch_single_sweep_and_its_fallback():
+    """The batched bf16 call counts in ONE sweep from an estimate of the threshold taken on a sample of
+    rows (about every rows/128-th), and falls back to the count sweep where the estimate misleads it.
+    Matrices whose sampled rows are unlike the rest, in both directions, non-finite weights, dead
+    channels and a constant matrix must all give the oracle's count and the single call's sum."""
+    cols = 2048
+    cases = []
+    for kind in ("plain", "sample_small", "sample_large", "inf", "nan", "dead_channels", "constant", "tall"):
+        rows = 3000 if kind == "tall" else 512
+        W = make(rows, cols, "bf16", seed=4000 + len(cases), heavy=(kind == "tall")).clone()
+        n = norms_for(cols, 400 + len(cases))
+        step = max(rows // 128, 1)
+        if kind == "sample_small":
+            W[step // 2::step] *= 0.001          # the sampled rows say "small scores": the ladders sit far too low
+        elif kind == "sample_large":
+            W[step // 2::step] *= 1000.0         # ... "large scores": far too high
+        elif kind == "inf":
+            W[7, 9] = float("inf")
+        elif kind == "nan":
+            W[300, 2000] = float("nan")
+        elif kind == "dead_channels":
+            n = n * (torch.rand(cols, device=DEV) > 0.5)
+        elif kind == "constant":
+            W.fill_(0.5)
+            n = torch.ones(cols, device=DEV)
+        cases.append((kind, W, n))
+    counts = torch.full((len(cases),), -5, dtype=torch.int64, device=DEV)
+    sums = torch.full((len(cases),), -1.0, dtype=torch.float64, device=DEV)
+    api.mosaic_outlier_ratio_batch([(W, n, counts[i:i + 1], sums[i:i + 1]) for i, (_, W, n) in enumerate(cases)], 4.0)
+    torch.cuda.synchronize()
+    for i, (kind, W, n) in enumerate(cases):
+        ref = oracle.outlier_ratio(host(W), n.cpu().numpy(), 4.0, "bf16")
+        assert counts[i].item() == ref["count"], kind
+        if kind not in ("inf", "nan"):
+            assert ref["certified"], kind
+            c1 = torch.zeros(1, dtype=torch.int64, device=DEV)
+            s1 = torch.zeros(1, dtype=torch.float64, device=DEV)
+            api.mosaic_outlier_ratio(W, n, 4.0, c1, s1)
+            assert c1.item() == counts[i].item(), kind
+            assert s1.cpu().numpy().tobytes() == sums[i:i + 1].cpu().numpy().tobytes(), kind   # same partial sums, same order
+    assert counts[[k for k, _, _ in cases].index("constant")].item() == 0
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_outlier_ratio_grouped_matches_oracle(dtype):
     # Eq. 3-4: the matrices of a group are counted against ONE threshold; three groups of different sizes
