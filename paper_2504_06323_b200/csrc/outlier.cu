@@ -390,7 +390,7 @@ __global__ void __launch_bounds__(kOutThreads, 8) outlier_count_bf16_kernel(cons
 // valid = 0 and is counted by the count sweep after all.
 // ------------------------------------------------------------------------------------------
 
-// est_sum of every matrix: the fp64 sum of the scores of about 128 evenly spaced rows, scaled to all
+// est_sum of every matrix: the fp64 sum of the scores of about 256 evenly spaced rows, scaled to all
 // rows.  kEstParts CTAs per matrix (128 column lanes of 8 columns x kEstRowLanes row lanes each) add
 // their shares atomically: the estimate may differ in its last bits from run to run, which moves a
 // ladder by a pattern at most and never the count.  The bookkeeping block was zeroed with the ladders.
@@ -399,7 +399,7 @@ template <int NJ>
 __global__ void __launch_bounds__(kOutThreads * kEstRowLanes) outlier_estimate_kernel(const __grid_constant__ OutlierJobList<NJ> jobs) {
     __shared__ double red[32];
     const OutlierJob& J = jobs.job[blockIdx.x];
-    const int64_t step = J.rows / 128 > 0 ? J.rows / 128 : 1;
+    const int64_t step = J.rows / 256 > 0 ? J.rows / 256 : 1;
     const int64_t n_sampled = (J.rows - step / 2 + step - 1) / step;   // rows step/2, step/2 + step, ...
     const int cl = threadIdx.x % kOutThreads, rl = threadIdx.x / kOutThreads;
     const int lanes = kEstRowLanes * kEstParts, my = (int)blockIdx.y * kEstRowLanes + rl;
@@ -410,16 +410,16 @@ __global__ void __launch_bounds__(kOutThreads * kEstRowLanes) outlier_estimate_k
 #pragma unroll
         for (int e = 0; e < kVec; ++e) nrm[e] = __ldg(J.norms + c0 + e);
         const char* base = static_cast<const char*>(J.W) + (size_t)c0 * 2u;
-        uint4 v[4];
+        uint4 v[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {   // at most four sampled rows per thread (128 rows over 32 lanes)
+        for (int u = 0; u < 8; ++u) {   // at most eight sampled rows per thread (256 rows over 32 lanes)
             const int64_t i = my + (int64_t)u * lanes;
             v[u] = make_uint4(0u, 0u, 0u, 0u);
             if (i < n_sampled) v[u] = ld_stream16_ro(base + (size_t)(step / 2 + i * step) * stride);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) add_scores(v[u], nrm, acc);
-        for (int64_t i = my + 4ll * lanes; i < n_sampled; i += lanes)
+        for (int u = 0; u < 8; ++u) add_scores(v[u], nrm, acc);
+        for (int64_t i = my + 8ll * lanes; i < n_sampled; i += lanes)
             add_scores(ld_stream16_ro(base + (size_t)(step / 2 + i * step) * stride), nrm, acc);
     }
     const double s = block_sum((acc[0] + acc[1]) + (acc[2] + acc[3]), red);
