@@ -129,8 +129,15 @@ double mosaic_ratio_from_count(int64_t outlier_count, int64_t numel);
 
 /* ---------------------------------------------------------------------------
  * mosaic_outlier_ratio_batch - mosaic_outlier_ratio for a list of projections
- * (Algorithm 1 loops over all N*M of them) in two launches instead of two per
- * projection.  Results are bit for bit those of the single call.
+ * (Algorithm 1 loops over all N*M of them) in a handful of launches instead of
+ * two per projection.  Results are bit for bit those of the single call.
+ * bf16 matrices with cols % 8 == 0 are read ONCE: an estimate of the threshold
+ * from a sample of rows fixes, per column, a ladder of 32 bf16 magnitude patterns
+ * around the pattern the threshold will fall on; the sweep that sums the scores
+ * counts the weights above the ladder and, per pattern, those on it, and the
+ * exact count follows when the sum is known.  A matrix whose threshold falls off
+ * a ladder (rows unlike the sampled ones) is counted by a second sweep after
+ * all.  The workspace holds the ladders (128 bytes per column and matrix).
  *   jobs   HOST array of n_jobs descriptors (read during the call only); the
  *          pointers inside are device pointers with the meaning of the
  *          single call's arguments (score_sum_out may be NULL)
