@@ -34,6 +34,22 @@ def test_every_declared_symbol_is_exported(lib):
     assert lib.mosaic_version() == 100
 
 
+def test_outlier_batch_workspace_holds_partials_and_ladders(lib):
+    # per matrix: one fp64 partial per 64 x 1024 tile (256-byte aligned) + a bookkeeping block and
+    # 32 counters of 4 bytes per column for the single-sweep count
+    jobs = (api.OutlierJob * 2)()
+    jobs[0].rows, jobs[0].cols = 4096, 4096
+    jobs[1].rows, jobs[1].cols = 11008, 4096
+    import ctypes as C
+    got = lib.mosaic_outlier_ratio_batch_workspace_bytes(C.addressof(jobs), 2)
+    want = 256
+    for rows, cols in ((4096, 4096), (11008, 4096)):
+        want += lib.mosaic_outlier_ratio_workspace_bytes(rows, cols)
+        want += (256 + 128 * cols + 255) // 256 * 256
+    assert got == want
+    assert lib.mosaic_outlier_ratio_workspace_bytes(4096, 4096) == 8 * 64 * 4     # 64 bands x 4 chunks of doubles
+
+
 def test_status_strings(lib):
     seen = set()
     for s in range(0, -11, -1):
