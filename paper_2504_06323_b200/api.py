@@ -338,7 +338,8 @@ class OutlierBatch:
 
 def mosaic_outlier_ratio_batch(jobs, alpha: float, ws: Workspace | None = None, stream=None) -> None:
     """mosaic_outlier_ratio over a list of (W, norms, outlier_count_out[1], score_sum_out[1] or None)
-    in two launches; the count tensors may be one-element views of a larger int64 tensor."""
+    in a handful of launches (bf16: one sweep over the weights); the count tensors may be one-element
+    views of a larger int64 tensor."""
     if jobs:
         OutlierBatch(jobs).run(alpha, ws, stream)
 

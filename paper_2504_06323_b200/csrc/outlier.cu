@@ -24,6 +24,10 @@
 //                             bisection on that very predicate - with  score > tau  <=>  |w| >= A_j,
 //                             and a row is counted two weights per integer subtract:
 //                             (w | 0x8000) - A_j has bit 15 set iff the magnitude is >= A_j.
+// The batched call reads such matrices only once: score_sum_ladder_kernel is the first sweep with a
+// ladder of bf16 patterns per column around an estimated threshold, from which the exact count
+// follows when the sum is known (see "Single sweep" below); the second sweep remains as the
+// fallback for matrices whose threshold falls off a ladder.
 #include <atomic>
 #include <memory>
 #include <new>

@@ -190,7 +190,7 @@ def _cached_batch(st: ModelState, name: str, jobs: list, make):
 
 
 def count_outliers_all(st: ModelState, alpha: float | None = None) -> int:
-    """Outlier counts of every owned projection through the batched call (two launches).  The job
+    """Outlier counts of every owned projection through the batched call (a handful of launches).  The job
     list is marshalled once and reused while the tensors of the ModelState stay the same objects."""
     cfg = st.cfg
     a = cfg.alpha if alpha is None else alpha
