@@ -115,3 +115,42 @@ def test_gram_random_cases(seed):
             ref = ref_abs = np.zeros((cols, cols))
         assert int(status.item()) == 0
         assert (np.abs(G.cpu().numpy() - ref) <= (tokens / 4.0 + 2.0) * 2.0 ** -24 * ref_abs + 1e-30).all(), dict(tokens=tokens, cols=cols)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_outlier_batch_random_cases(seed):
+    """The batched call (one sweep with per-column ladders, count sweep as the fallback) over lists of
+    random matrices, each with its own threshold or grouped: counts equal to the oracle's wherever it
+    certifies them, sums within what the order of fp64 additions can move them."""
+    rng = np.random.default_rng(400 + seed)
+    for _ in range(6):
+        n_jobs = int(rng.integers(1, 7))
+        alpha = float(rng.choice([1.0, 2.5, 5.0, 9.0]))
+        grouped = bool(rng.integers(2))
+        Ws, ns = [], []
+        for _j in range(n_jobs):
+            rows = int(rng.choice([1, 7, 64, 65, 255, 256, 257, int(rng.integers(1, 1500))]))
+            cols = int(rng.choice([8, 1024, 1032, 2048, 4096, int(rng.integers(1, 700)) * 8]))
+            Ws.append(rand_weights(rng, rows, cols, str(rng.choice(["t3", "ties", "sparse", "scales"]))))
+            ns.append(rand_norms(rng, cols, str(rng.choice(["spread", "equal", "ones", "zeros", "octaves"]))))
+        counts = torch.full((n_jobs,), -3, dtype=torch.int64, device=DEV)
+        sums = torch.full((n_jobs,), -1.0, dtype=torch.float64, device=DEV)
+        jobs = [(W, n, counts[i:i + 1], sums[i:i + 1]) for i, (W, n) in enumerate(zip(Ws, ns))]
+        if grouped:
+            groups = np.sort(rng.integers(0, 3, n_jobs)).tolist()
+            api.mosaic_outlier_ratio_grouped(jobs, groups, alpha)
+        else:
+            groups = list(range(n_jobs))
+            api.mosaic_outlier_ratio_batch(jobs, alpha)
+        torch.cuda.synchronize()
+        got_c, got_s = counts.cpu().tolist(), sums.cpu().numpy()
+        for g in sorted(set(groups)):
+            idx = [i for i in range(n_jobs) if groups[i] == g]
+            ref = oracle.outlier_ratio_group([wl.to_numpy(Ws[i]) for i in idx], [ns[i].cpu().numpy() for i in idx], alpha, "bf16")
+            for pos, i in enumerate(idx):
+                case = dict(seed=seed, shape=tuple(Ws[i].shape), alpha=alpha, grouped=grouped)
+                own = oracle.outlier_ratio(wl.to_numpy(Ws[i]), ns[i].cpu().numpy(), alpha, "bf16")["sum"]   # a matrix's own score sum
+                # another order of the fp64 additions: at most numel * 2^-53 of the sum of these non-negative terms
+                assert abs(got_s[i] - own) <= Ws[i].numel() * 2.0 ** -52 * abs(own) + 1e-300 or not np.isfinite(own), case
+                if ref["certified"]:
+                    assert got_c[i] == ref["counts"][pos], case
